@@ -1,0 +1,165 @@
+/*
+ * vgg19_b200 - the VGG19 forward and backward pass as one device program for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The computation is the one the paper offloads as a single executable
+ * (section 7.2 "VGG19 forward pass", section 7.3 "VGG19 backward pass"):
+ * 16 convolutions 3x3 / pad 1 / stride 1 with bias and ReLU, five 2x2
+ * max-pools, three dense layers (section 7.1, dense(W,x,b) = W*x .+ b),
+ * softmax (section 7.1), and the gradient of a scalar loss with respect to
+ * every parameter.  The loss is the mean cross-entropy of the softmax output
+ * against integer labels.
+ *
+ * Conventions
+ *  - Every function returns VGG19_OK (0) or a negative vgg19_status.  No C++
+ *    exception crosses this boundary.  vgg19_last_error() gives text.
+ *  - "device" pointers are CUDA device pointers of the current device, owned
+ *    by the caller, and must stay valid until the work enqueued on the stream
+ *    has finished.  "host" pointers are ordinary host memory.
+ *  - Work is enqueued on the given cudaStream_t (passed as void*; NULL = the
+ *    legacy default stream) and returns without waiting for it.
+ *  - Layouts: images and activations are NHWC (channel fastest); a conv weight
+ *    is [Cout][3][3][Cin]; a dense weight is [out][in] with `in` enumerating
+ *    the flattened (h, w, c) activation, c fastest; a bias is [out].
+ *  - The flat parameter / gradient buffer holds, for layer 1..19 in network
+ *    order, the weight then the bias, as fp32.
+ */
+#ifndef VGG19_B200_H_
+#define VGG19_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct vgg19 vgg19_t;
+
+typedef enum {
+  VGG19_OK = 0,
+  VGG19_ERR_ARG = -1,             /* null pointer, bad enum, batch out of range */
+  VGG19_ERR_SHAPE = -2,           /* height/width not a positive multiple of 32 */
+  VGG19_ERR_WORKSPACE = -3,       /* no workspace bound, or too small */
+  VGG19_ERR_CUDA = -4,            /* a CUDA runtime/driver call failed */
+  VGG19_ERR_DEVICE_TIMEOUT = -5,  /* a bounded device-side wait ran out */
+  VGG19_ERR_UNSUPPORTED_ARCH = -6 /* the device is not compute capability 10.x */
+} vgg19_status;
+
+typedef enum {
+  VGG19_FP32 = 0, /* fp32 storage and fp32 FMA arithmetic throughout */
+  VGG19_BF16 = 1  /* bf16 activations/weights, fp32 accumulation, fp32 gradients */
+} vgg19_dtype;
+
+enum {
+  VGG19_FLAG_NO_GRAPH = 1,        /* enqueue kernels directly instead of replaying a CUDA graph */
+  VGG19_FLAG_NO_TENSOR_CORES = 2  /* bf16 only: use the CUDA-core kernels for every layer */
+};
+
+typedef enum { VGG19_MODE_FORWARD = 0, VGG19_MODE_BACKWARD = 1 } vgg19_mode;
+
+typedef struct {
+  int32_t height;    /* input height, multiple of 32 */
+  int32_t width;     /* input width, multiple of 32 */
+  int32_t batch_max; /* largest batch any later call will use */
+  int32_t dtype;     /* vgg19_dtype */
+  uint32_t flags;    /* VGG19_FLAG_* */
+} vgg19_config;
+
+/* Build a network whose parameters are the seeded He-normal set (weights
+ * N(0, 2/fan_in), biases 0) drawn on the host from `seed` and uploaded.  The
+ * library owns the parameters.  (North-star entry point "vgg19_create from a
+ * seeded weight set"; the paper itself used trained weights, section 7.2.) */
+int vgg19_create(const vgg19_config *cfg, uint64_t seed, vgg19_t **out);
+
+/* Same, from a caller-supplied flat fp32 HOST buffer of vgg19_param_count()
+ * elements in the order given above.  The buffer is copied. */
+int vgg19_create_from_params(const vgg19_config *cfg, const float *host_params, vgg19_t **out);
+
+/* Frees everything the library allocated (parameters, graphs).  Never frees
+ * the workspace.  NULL is allowed. */
+void vgg19_destroy(vgg19_t *net);
+
+/* Number of parameter tensors (38) and of fp32 elements in the flat buffer. */
+int vgg19_param_count(const vgg19_t *net, int32_t *n_tensors, size_t *n_elems);
+
+/* Tensor i (0..37): element offset in the flat buffer, rank and dims
+ * ([Cout,3,3,Cin], [out,in] or [out]). */
+int vgg19_param_info(const vgg19_t *net, int32_t i, size_t *offset, int32_t *rank, int64_t dims[4]);
+
+/* Copy the fp32 master parameters to / from a HOST buffer (synchronous). */
+int vgg19_get_params(const vgg19_t *net, float *host_params);
+int vgg19_set_params(vgg19_t *net, const float *host_params);
+
+/* Bytes of device scratch a call in `mode` at `batch` needs (saved
+ * activations, gradients in flight, split-K partials).  0 on bad arguments. */
+size_t vgg19_workspace_bytes(const vgg19_t *net, int32_t batch, int32_t mode);
+
+/* Hand the library a DEVICE buffer (256-byte aligned) to use as scratch.  The
+ * caller keeps ownership and must keep it alive while calls are in flight. */
+int vgg19_bind_workspace(vgg19_t *net, void *device_workspace, size_t bytes);
+
+/* Forward pass (section 7.2).  images: device, [batch][H][W][3], fp32 or bf16
+ * per the config, already normalised.  logits: device fp32 [batch][1000], the
+ * input of the softmax.  probs: device fp32 [batch][1000] = softmax(logits)
+ * (section 7.1), or NULL to skip it.  The first call for a given (batch,
+ * pointers) records the whole pass into one CUDA graph; later calls replay
+ * it - the counterpart of the paper's single offloaded executable. */
+int vgg19_forward(vgg19_t *net, const void *images, int32_t batch, float *logits, float *probs,
+                  void *stream);
+
+/* Forward + loss + backward (section 7.3) as one graph.  labels: device int32
+ * [batch] in [0,1000).  grads: device fp32, vgg19_param_count() elements,
+ * fully overwritten with d(loss)/d(parameter), loss = mean cross-entropy.
+ * loss: device fp32 scalar or NULL.  logits: device fp32 [batch][1000] or
+ * NULL.  The batch argument is an addition to the spec signature, which
+ * leaves the batch size implicit. */
+int vgg19_backward(vgg19_t *net, const void *images, const int32_t *labels, int32_t batch,
+                   float *grads, float *loss, float *logits, void *stream);
+
+/* HOST-buffer convenience wrappers: copy images (and labels) to the device,
+ * run the pass, copy the results back and wait for the stream.  The bound
+ * workspace must hold vgg19_workspace_bytes(net, batch, mode) +
+ * vgg19_io_bytes(net, batch, mode) bytes; the staging area is its tail.
+ * Host buffers should be page-locked for full copy bandwidth.  Any result
+ * pointer may be NULL to skip that copy. */
+size_t vgg19_io_bytes(const vgg19_t *net, int32_t batch, int32_t mode);
+int vgg19_forward_host(vgg19_t *net, const void *host_images, int32_t batch, float *host_logits,
+                       float *host_probs, void *stream);
+int vgg19_backward_host(vgg19_t *net, const void *host_images, const int32_t *host_labels,
+                        int32_t batch, float *host_grads, float *host_loss, void *stream);
+
+/* Single convolution layer (3x3, pad 1, stride 1) + bias + ReLU, optionally
+ * followed by the 2x2 max-pool, on caller-supplied device tensors in the
+ * config's dtype; the per-layer building block of section 7.2, exposed for
+ * per-layer parity and timing.  layer in 1..16 selects shape and weights;
+ * x: [batch][h][w][Cin]; y: [batch][h][w][Cout]; pooled (or NULL):
+ * [batch][h/2][w/2][Cout]. */
+int vgg19_conv_layer_forward(vgg19_t *net, int32_t layer, const void *x, int32_t batch,
+                             void *y, void *pooled, void *stream);
+
+/* Gradients of that layer given dz = d(loss)/d(pre-activation) already
+ * masked by the ReLU: dw fp32 [Cout][3][3][Cin], db fp32 [Cout], and (unless
+ * NULL) dx in the config's dtype [batch][h][w][Cin] (section 7.3). */
+int vgg19_conv_layer_backward(vgg19_t *net, int32_t layer, const void *x, const void *dz,
+                              int32_t batch, float *dw, float *db, void *dx, void *stream);
+
+/* Wait for the stream and report any device-side error recorded so far. */
+int vgg19_sync_status(vgg19_t *net, void *stream);
+
+/* Number of kernel launches (graph nodes) one forward / backward call makes. */
+int vgg19_launch_count(const vgg19_t *net, int32_t mode, int32_t *n_kernels);
+
+/* Human-readable layer table and kernel list (the counterpart of the paper's
+ * @code_xla introspection macro, section 7.1).  Writes at most n bytes,
+ * NUL-terminated; returns the length needed. */
+int vgg19_describe(const vgg19_t *net, char *buf, size_t n);
+
+/* Text of the last error on this handle (or of the last failed create when
+ * net is NULL).  Never NULL. */
+const char *vgg19_last_error(const vgg19_t *net);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VGG19_B200_H_ */

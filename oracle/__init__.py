@@ -66,6 +66,7 @@ def _load():
             "oracle_cross_entropy": ([d, i32, I, I, I], ctypes.c_double),
             "oracle_softmax_ce_bwd": ([d, i32, d, I, I, I], None),
             "oracle_softmax_bwd": ([d, d, d, I, I], None),
+            "oracle_round_bf16": ([d, L], None),
         }
         for name, (args, res) in sig.items():
             fn = getattr(lib, name)
@@ -211,6 +212,22 @@ def softmax_bwd(p, g):
     return dl
 
 
+def round_bf16(x):
+    """Nearest-bfloat16 (ties to even) of every element, returned as fp64."""
+    x = np.array(x, dtype=np.float64, order="C", copy=True)
+    _load().oracle_round_bf16(_d(x), x.size)
+    return x
+
+
+def _store(x, storage):
+    """Model the storage format of a tensor the configuration keeps in memory:
+    exact for fp64, rounded to bf16 for the bf16 configurations."""
+    if storage is None:
+        return x
+    assert storage == "bf16"
+    return round_bf16(x)
+
+
 # ------------------------------------------------------------------ networks
 
 def vgg19_steps():
@@ -250,9 +267,16 @@ def split_params(flat_params, shapes):
     return out
 
 
-def forward(steps, params, images, keep=False):
+def forward(steps, params, images, keep=False, storage=None):
     """Logits [N, classes] (pre-softmax).  With keep=True also returns the
-    list of saved tensors the backward pass needs."""
+    list of saved tensors the backward pass needs.
+
+    storage=None: every intermediate stays fp64.  storage="bf16": the
+    configuration "bf16 activations, fp32 accumulate" - all arithmetic is still
+    fp64, but each activation the configuration keeps in memory (the output of
+    every conv+ReLU and dense+ReLU) is rounded to bf16 where it is stored, so
+    that ReLU masks and pool arg-maxima are decided on the same stored values
+    on which the device decides them.  Logits stay unrounded."""
     x = _c(images)
     shapes = param_shapes(steps, x.shape[1], x.shape[2], x.shape[3])
     P = split_params(_c(params), shapes)
@@ -261,8 +285,8 @@ def forward(steps, params, images, keep=False):
         if st[0] == "conv":
             Wt, b = P[pi]; pi += 1
             z = conv3x3_fwd(x, Wt, b)
-            y = relu_fwd(z)
-            saved.append(("conv", x, z))
+            y = _store(relu_fwd(z), storage)
+            saved.append(("conv", x, y))  # y > 0 exactly where z > 0
             x = y
         elif st[0] == "pool":
             p = maxpool2x2_fwd(x)
@@ -273,18 +297,20 @@ def forward(steps, params, images, keep=False):
             shp = x.shape
             xf = x.reshape(x.shape[0], -1)
             z = dense_fwd(xf, Wt, b)
-            saved.append(("fc", xf, z, shp, st[2]))
-            x = relu_fwd(z) if st[2] else z
+            x = _store(relu_fwd(z), storage) if st[2] else z
+            saved.append(("fc", xf, x, shp, st[2]))
     return (x, saved) if keep else x
 
 
-def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_kind="ce"):
+def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_kind="ce", storage=None):
     """Gradient of the loss with respect to every parameter, flat, in the
     parameter order.  loss_kind "ce": mean cross-entropy of softmax(logits)
     (dlogits = (p - onehot) / n_total).  loss_kind "sum": the paper's
     stand-in sum(softmax(logits)) (section 7.3).  When `grads` is given the
-    result is accumulated into it (chunked batches).  Returns
-    (loss, grads, logits)."""
+    result is accumulated into it (chunked batches).  With storage="bf16"
+    the gradients the configuration keeps in memory between layers (dlogits
+    and every activation gradient) are rounded to bf16 where they are stored;
+    parameter gradients are never rounded.  Returns (loss, grads, logits)."""
     params = _c(params)
     images = _c(images)
     N = images.shape[0]
@@ -294,11 +320,11 @@ def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_
     if grads is None:
         grads = np.zeros_like(params)
     G = split_params(grads, shapes)
-    logits, saved = forward(steps, params, images, keep=True)
+    logits, saved = forward(steps, params, images, keep=True, storage=storage)
     p = softmax(logits)
     if loss_kind == "ce":
         loss = cross_entropy(logits, labels, n_total)
-        g = softmax_ce_bwd(p, labels, n_total)
+        g = _store(softmax_ce_bwd(p, labels, n_total), storage)
     else:
         loss = float(p.sum())
         g = softmax_bwd(p, np.ones_like(p))
@@ -307,32 +333,32 @@ def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_
     for si in range(len(steps) - 1, -1, -1):
         st, sv = steps[si], saved[si]
         if st[0] == "fc":
-            _, xf, z, shp, relu = sv
+            _, xf, y, shp, relu = sv
             if relu:
-                g = relu_bwd(z, g)
+                g = relu_bwd(y, g)
             Wt, _ = P[pi]
             dW, db = G[pi]; pi -= 1
             dx, _, _ = dense_bwd(xf, Wt, g, dW, db, need_dx=si != first_param_step)
-            g = None if dx is None else dx.reshape(shp)
+            g = None if dx is None else _store(dx.reshape(shp), storage)
         elif st[0] == "pool":
             g = maxpool2x2_bwd(sv[1], g)
         else:
-            _, xin, z = sv
-            dz = relu_bwd(z, g)
+            _, xin, y = sv
+            dz = relu_bwd(y, g)
             Wt, _ = P[pi]
             dW, db = G[pi]; pi -= 1
             conv3x3_wgrad(xin, dz, dW, db)
             # the derivative is with respect to the model only: the first
             # layer's input gradient is never needed (47, not 48, convolutions)
-            g = conv3x3_dgrad(dz, Wt) if si != first_param_step else None
+            g = _store(conv3x3_dgrad(dz, Wt), storage) if si != first_param_step else None
     return loss, grads, logits
 
 
-def vgg19_forward(params, images):
-    return forward(vgg19_steps(), params, images)
+def vgg19_forward(params, images, storage=None):
+    return forward(vgg19_steps(), params, images, storage=storage)
 
 
-def vgg19_backward(params, images, labels, chunk=4):
+def vgg19_backward(params, images, labels, chunk=4, storage=None):
     """Whole-batch VGG19 loss, gradients and logits, processed `chunk` images
     at a time to bound memory (the loss and gradient are sums over images)."""
     steps = vgg19_steps()
@@ -340,7 +366,8 @@ def vgg19_backward(params, images, labels, chunk=4):
     grads = np.zeros(np.asarray(params).size)
     loss, logits = 0.0, []
     for s in range(0, N, chunk):
-        l, _, lg = backward(steps, params, images[s:s + chunk], labels[s:s + chunk], n_total=N, grads=grads)
+        l, _, lg = backward(steps, params, images[s:s + chunk], labels[s:s + chunk], n_total=N, grads=grads,
+                            storage=storage)
         loss += l
         logits.append(lg)
     return loss, grads, np.concatenate(logits)

@@ -264,3 +264,21 @@ void oracle_softmax_bwd(const double *p, const double *g, double *dl, int N, int
       dl[(idx)n * C + j] = p[(idx)n * C + j] * (g[(idx)n * C + j] - dot);
   }
 }
+
+/* Storage format of the bf16 configurations ("bf16 activations/weights with
+ * fp32 accumulate"): round every element to the nearest bfloat16 (8 significant
+ * bits, ties to even), keeping it as a double.  A value v = m * 2^e with
+ * 0.5 <= |m| < 1 lies in a binade whose bf16 spacing is 2^(e-8); below the
+ * smallest normal the spacing stays at 2^-133.  rint() rounds ties to even in
+ * the default rounding mode and the scaling by a power of two is exact.      */
+void oracle_round_bf16(double *x, idx n) {
+  for (idx i = 0; i < n; ++i) {
+    double v = x[i];
+    if (v == 0.0 || !isfinite(v)) continue;
+    int e;
+    frexp(v, &e);
+    int q = e - 8;
+    if (q < -133) q = -133;
+    x[i] = ldexp(rint(ldexp(v, -q)), q);
+  }
+}

@@ -1,0 +1,90 @@
+// Shared declarations of the VGG19 device library: status codes, small
+// device helpers, and the host-side launch functions each .cu file exports
+// to the pass scheduler in vgg19_api.cu.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace vgg {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// Device-side error word (one per network).  A kernel whose bounded wait ran
+// out stores a nonzero code here and returns; the host reads it at
+// vgg19_sync_status().
+enum DeviceError : int {
+  kDevOk = 0,
+  kDevTimeoutTmaFull = 1,   // consumer waited too long for a TMA stage
+  kDevTimeoutStageFree = 2, // producer waited too long for a free stage
+  kDevTimeoutAccum = 3,     // epilogue waited too long for the accumulator
+  kDevTimeoutTmemFree = 4,  // MMA issuer waited too long for a drained accumulator
+};
+
+// ---- CUDA-core kernels (simt_kernels.cu) ---------------------------------
+// T is the storage type of activations and weights (float or bf16); every
+// sum is accumulated in fp32.
+
+struct ConvShape {
+  int N, H, W, Cin, Cout;
+};
+
+// out = [relu](conv3x3(in, wt) + bias) [* (mask > 0)], NHWC, wt [Cout][3][3][Cin].
+template <typename T>
+cudaError_t simt_conv3x3(const T* in, const T* wt, const float* bias, const T* mask, T* out,
+                         ConvShape s, bool relu, cudaStream_t st);
+
+// dW[k][r][s][c] = sum_p dz[p][k] x[p+(r-1,s-1)][c]; db[k] = sum_p dz[p][k].
+// partial: fp32 scratch of simt_wgrad_scratch_elems() elements.
+size_t simt_wgrad_scratch_elems(ConvShape s);
+template <typename T>
+cudaError_t simt_conv3x3_wgrad(const T* x, const T* dz, float* dW, float* db, float* partial,
+                               ConvShape s, cudaStream_t st);
+
+// y = max over 2x2 windows (stride 2) of x, NHWC.
+template <typename T>
+cudaError_t simt_maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st);
+
+// dy[pos] = dp[window] where pos is the window's first maximum of y and
+// y[pos] > 0, else 0 (pool scatter fused with the ReLU mask of the layer that
+// produced y).
+template <typename T>
+cudaError_t simt_maxpool_bwd_relu(const T* y, const T* dp, T* dy, int N, int H, int W, int C,
+                                  cudaStream_t st);
+
+// C[m][n] = epilogue(sum_k A[m][k] * B[n][k]); A [M][K] and B [N][K] row-major.
+// Epilogue: + bias[n], ReLU, * (mask[m][n] > 0); written as T (out_t) and/or fp32 (out_f).
+template <typename T>
+cudaError_t simt_dense_nt(const T* A, const T* B, const float* bias, const T* mask, T* out_t,
+                          float* out_f, int M, int N, int K, bool relu, cudaStream_t st);
+
+// dX[m][i] = (sum_o dY[m][o] * W[o][i]) * (mask[m][i] > 0)      (W [Out][In] row-major)
+template <typename T>
+cudaError_t simt_dense_dx(const T* dY, const T* W, const T* mask, T* dX, int M, int In, int Out,
+                          cudaStream_t st);
+
+// dW[o][i] = sum_m dY[m][o] * X[m][i];  db[o] = sum_m dY[m][o]   (fp32 out)
+template <typename T>
+cudaError_t simt_dense_dw(const T* dY, const T* X, float* dW, float* db, int M, int In, int Out,
+                          cudaStream_t st);
+
+// Row-wise softmax of fp32 logits (probs may be null), and for the backward
+// pass the per-row loss and dlogits = (p - onehot(label)) / rows, stored as T.
+template <typename T>
+cudaError_t softmax_xent(const float* logits, const int32_t* labels, float* probs, T* dlogits,
+                         float* row_loss, float* loss, int rows, int classes, cudaStream_t st);
+
+// fp32 -> T copy (weights), and the dgrad filter: wt_t[c][r][s][k] = w[k][2-r][2-s][c].
+template <typename T>
+cudaError_t convert_f32(const float* src, T* dst, size_t n, cudaStream_t st);
+template <typename T>
+cudaError_t make_dgrad_filter(const float* w, T* wt_t, int Cin, int Cout, cudaStream_t st);
+
+}  // namespace vgg

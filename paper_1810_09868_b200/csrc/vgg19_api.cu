@@ -1,0 +1,692 @@
+// C-ABI of the VGG19 device library: the static layer table, the workspace
+// plan, the order in which kernels are enqueued for a forward or a
+// forward+backward pass, and the CUDA-graph cache that turns a pass into one
+// launch (the counterpart of the paper's single offloaded executable,
+// section 7.2).
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/vgg19_b200.h"
+#include "../../seeded_inputs/seeded_inputs.h"
+#include "common.cuh"
+#include "tc_kernels.cuh"
+
+using namespace vgg;
+
+namespace {
+
+constexpr int kConvLayers = 16, kFcLayers = 3, kLayers = 19, kClasses = 1000;
+const int kConvOut[kConvLayers] = {64, 64, 128, 128, 256, 256, 256, 256,
+                                   512, 512, 512, 512, 512, 512, 512, 512};
+const bool kPoolAfter[kConvLayers] = {false, true, false, true, false, false, false, true,
+                                      false, false, false, true, false, false, false, true};
+
+struct ConvLayer {
+  int H, W, Cin, Cout;  // input spatial size = output spatial size
+  bool pool_after;
+  size_t w_off, b_off;  // element offsets in the flat parameter buffer
+  size_t dgrad_off;     // element offset of the rotated filter in the dgrad filter buffer
+};
+struct FcLayer {
+  int In, Out;
+  bool relu;
+  size_t w_off, b_off;
+};
+
+std::string g_create_error;
+
+size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+struct GraphEntry {
+  int mode, batch;
+  const void *p[6];
+  cudaGraphExec_t exec;
+  int n_kernels;
+};
+
+}  // namespace
+
+struct vgg19 {
+  vgg19_config cfg;
+  size_t elt;  // bytes per activation element
+  ConvLayer conv[kConvLayers];
+  int pool_idx[kConvLayers];  // which of the five pools follows layer l, or -1
+  FcLayer fc[kFcLayers];
+  size_t n_params, n_dgrad;
+  float *params = nullptr;   // fp32 master, device
+  void *params_t = nullptr;  // copy in the storage dtype (aliases params in fp32 mode)
+  void *dgrad_w = nullptr;   // rotated filters for layers 2..16, storage dtype
+  int *dev_error = nullptr;
+  void *ws = nullptr;
+  size_t ws_bytes = 0;
+  std::vector<GraphEntry> graphs;
+  int launches[2] = {0, 0};
+  std::string err;
+  bool use_tc = false;
+};
+
+namespace {
+
+int fail(vgg19 *n, int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (n) n->err = buf; else g_create_error = buf;
+  return code;
+}
+
+#define CUDA_TRY(n, expr)                                                                   \
+  do {                                                                                      \
+    cudaError_t e_ = (expr);                                                                \
+    if (e_ != cudaSuccess)                                                                  \
+      return fail((n), VGG19_ERR_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e_), \
+                  __FILE__, __LINE__);                                                      \
+  } while (0)
+
+// ---- workspace plan ---------------------------------------------------------
+// All offsets in bytes from the workspace base, each 256-byte aligned.
+struct Plan {
+  size_t act[kConvLayers];  // y_l = relu(conv_l + b): [B][H][W][Cout]
+  size_t pooled[5];         // outputs of the five pools
+  size_t a1, a2;            // dense activations [B][4096]
+  size_t logits, probs;     // fp32 [B][1000] (used when the caller passes none)
+  size_t dl, dz2, dz1, dflat;  // backward: dlogits, dense pre-activation grads, d(flatten)
+  size_t dza, dzb, dxlow;   // conv backward ping-pong and the pooled-resolution dx
+  size_t partial;           // fp32 split-K partials
+  size_t row_loss, loss;
+  size_t total;
+  size_t io_images, io_labels, io_logits, io_probs, io_grads, io_loss, io_total;
+};
+
+Plan make_plan(const vgg19 *n, int B, int mode) {
+  Plan p{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  int pi = 0;
+  size_t max_act = 0, max_low = 0, max_partial = 0;
+  for (int l = 0; l < kConvLayers; ++l) {
+    const ConvLayer &c = n->conv[l];
+    size_t a = (size_t)B * c.H * c.W * c.Cout;
+    p.act[l] = take(a * n->elt);
+    if (a > max_act) max_act = a;
+    if (c.pool_after) {
+      p.pooled[pi++] = take(a / 4 * n->elt);
+      if (a / 4 > max_low) max_low = a / 4;
+    }
+    ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
+    size_t pe = simt_wgrad_scratch_elems(s);
+    size_t te = tc_wgrad_scratch_elems(s);
+    if (te > pe) pe = te;
+    if (pe > max_partial) max_partial = pe;
+  }
+  p.a1 = take((size_t)B * 4096 * n->elt);
+  p.a2 = take((size_t)B * 4096 * n->elt);
+  p.logits = take((size_t)B * kClasses * 4);
+  p.probs = take((size_t)B * kClasses * 4);
+  if (mode == VGG19_MODE_BACKWARD) {
+    p.dl = take((size_t)B * kClasses * n->elt);
+    p.dz2 = take((size_t)B * 4096 * n->elt);
+    p.dz1 = take((size_t)B * 4096 * n->elt);
+    p.dflat = take((size_t)B * n->fc[0].In * n->elt);
+    p.dza = take(max_act * n->elt);
+    p.dzb = take(max_act * n->elt);
+    p.dxlow = take(max_low * n->elt);
+    p.partial = take(max_partial * 4);
+    p.row_loss = take((size_t)B * 4);
+    p.loss = take(256);
+  }
+  p.total = off;
+  size_t io = off;
+  auto take_io = [&](size_t bytes) { size_t o = io; io += align_up(bytes); return o; };
+  p.io_images = take_io((size_t)B * n->cfg.height * n->cfg.width * 3 * n->elt);
+  p.io_logits = take_io((size_t)B * kClasses * 4);
+  p.io_probs = take_io((size_t)B * kClasses * 4);
+  if (mode == VGG19_MODE_BACKWARD) {
+    p.io_labels = take_io((size_t)B * 4);
+    p.io_grads = take_io(n->n_params * 4);
+    p.io_loss = take_io(256);
+  }
+  p.io_total = io - off;
+  return p;
+}
+
+// ---- enqueueing a pass ------------------------------------------------------
+
+struct PassArgs {
+  const void *images;
+  const int32_t *labels;
+  float *logits, *probs, *grads, *loss;
+  int batch;
+};
+
+template <typename T>
+struct Pass {
+  vgg19 *n;
+  Plan p;
+  cudaStream_t st;
+  int launches = 0;
+  cudaError_t err = cudaSuccess;
+
+  T *buf(size_t off) const { return reinterpret_cast<T *>(static_cast<char *>(n->ws) + off); }
+  float *fbuf(size_t off) const { return reinterpret_cast<float *>(static_cast<char *>(n->ws) + off); }
+  const T *wt(size_t off) const { return static_cast<const T *>(n->params_t) + off; }
+  void ok(cudaError_t e, int k) { if (err == cudaSuccess) err = e; launches += k; }
+
+  bool tc_conv_ok(const ConvShape &s) const { return n->use_tc && tc_conv3x3_supported(s); }
+
+  // y = relu(conv(x) + b), optionally pooled
+  void conv_forward(int l, const T *x, int B, T *y, T *pooled) {
+    const ConvLayer &c = n->conv[l];
+    ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
+    if (tc_conv_ok(s))
+      ok(tc_conv3x3((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
+                    (bf16 *)y, s, true, n->dev_error, st), 1);
+    else
+      ok(simt_conv3x3<T>(x, wt(c.w_off), n->params + c.b_off, nullptr, y, s, true, st), 1);
+    if (pooled) ok(simt_maxpool_fwd<T>(y, pooled, B, c.H, c.W, c.Cout, st), 1);
+  }
+
+  // dW, db from (x, dz); dx = dgrad(dz) [* (mask > 0)] unless dx is null
+  void conv_backward(int l, const T *x, const T *dz, int B, float *dW, float *db, T *dx,
+                     const T *mask) {
+    const ConvLayer &c = n->conv[l];
+    ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
+    if (n->use_tc && tc_wgrad_supported(s))
+      ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, db, fbuf(p.partial), s,
+                          n->dev_error, st), tc_wgrad_launches(s));
+    else
+      ok(simt_conv3x3_wgrad<T>(x, dz, dW, db, fbuf(p.partial), s, st), 4);
+    if (dx) {
+      ConvShape t{B, c.H, c.W, c.Cout, c.Cin};  // a 3x3 correlation from Cout to Cin channels
+      const T *wr = static_cast<const T *>(n->dgrad_w) + c.dgrad_off;
+      if (tc_conv_ok(t))
+        ok(tc_conv3x3((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
+                      t, false, n->dev_error, st), 1);
+      else
+        ok(simt_conv3x3<T>(dz, wr, nullptr, mask, dx, t, false, st), 1);
+    }
+  }
+
+  void forward(const PassArgs &a) {
+    const int B = a.batch;
+    const T *x = static_cast<const T *>(a.images);
+    int pi = 0;
+    for (int l = 0; l < kConvLayers; ++l) {
+      T *y = buf(p.act[l]);
+      T *pooled = n->conv[l].pool_after ? buf(p.pooled[pi++]) : nullptr;
+      conv_forward(l, x, B, y, pooled);
+      x = pooled ? pooled : y;
+    }
+    float *logits = a.logits ? a.logits : fbuf(p.logits);
+    const FcLayer *f = n->fc;
+    ok(simt_dense_nt<T>(x, wt(f[0].w_off), n->params + f[0].b_off, nullptr, buf(p.a1), nullptr, B,
+                        f[0].Out, f[0].In, true, st), 1);
+    ok(simt_dense_nt<T>(buf(p.a1), wt(f[1].w_off), n->params + f[1].b_off, nullptr, buf(p.a2),
+                        nullptr, B, f[1].Out, f[1].In, true, st), 1);
+    ok(simt_dense_nt<T>(buf(p.a2), wt(f[2].w_off), n->params + f[2].b_off, nullptr, nullptr, logits,
+                        B, f[2].Out, f[2].In, false, st), 1);
+    if (a.probs && !a.grads)
+      ok(softmax_xent<T>(logits, nullptr, a.probs, nullptr, nullptr, nullptr, B, kClasses, st), 1);
+  }
+
+  void backward(const PassArgs &a) {
+    const int B = a.batch;
+    forward(a);
+    float *logits = a.logits ? a.logits : fbuf(p.logits);
+    float *loss = a.loss ? a.loss : fbuf(p.loss);
+    float *g = a.grads;
+    const FcLayer *f = n->fc;
+    ok(softmax_xent<T>(logits, a.labels, a.probs, buf(p.dl), fbuf(p.row_loss), loss, B, kClasses,
+                       st), 2);
+    const T *flat = buf(p.pooled[4]);
+    // dense 3, 2, 1: filter gradient, then input gradient masked by the ReLU below
+    ok(simt_dense_dw<T>(buf(p.dl), buf(p.a2), g + f[2].w_off, g + f[2].b_off, B, f[2].In, f[2].Out, st), 2);
+    ok(simt_dense_dx<T>(buf(p.dl), wt(f[2].w_off), buf(p.a2), buf(p.dz2), B, f[2].In, f[2].Out, st), 1);
+    ok(simt_dense_dw<T>(buf(p.dz2), buf(p.a1), g + f[1].w_off, g + f[1].b_off, B, f[1].In, f[1].Out, st), 2);
+    ok(simt_dense_dx<T>(buf(p.dz2), wt(f[1].w_off), buf(p.a1), buf(p.dz1), B, f[1].In, f[1].Out, st), 1);
+    ok(simt_dense_dw<T>(buf(p.dz1), flat, g + f[0].w_off, g + f[0].b_off, B, f[0].In, f[0].Out, st), 2);
+    ok(simt_dense_dx<T>(buf(p.dz1), wt(f[0].w_off), nullptr, buf(p.dflat), B, f[0].In, f[0].Out, st), 1);
+    // convolutions 16..1.  `dz` is the gradient at layer l's pre-activation.
+    T *dz = buf(p.dza), *other = buf(p.dzb);
+    {
+      const ConvLayer &c = n->conv[15];
+      ok(simt_maxpool_bwd_relu<T>(buf(p.act[15]), buf(p.dflat), dz, B, c.H, c.W, c.Cout, st), 1);
+    }
+    for (int l = kConvLayers - 1; l >= 0; --l) {
+      const ConvLayer &c = n->conv[l];
+      const bool in_is_pool = l > 0 && n->conv[l - 1].pool_after;
+      const T *x = l == 0 ? static_cast<const T *>(a.images)
+                          : (in_is_pool ? buf(p.pooled[n->pool_idx[l - 1]]) : buf(p.act[l - 1]));
+      float *dW = g + c.w_off, *db = g + c.b_off;
+      if (l == 0) {
+        conv_backward(l, x, dz, B, dW, db, nullptr, nullptr);
+      } else if (in_is_pool) {
+        const ConvLayer &below = n->conv[l - 1];
+        conv_backward(l, x, dz, B, dW, db, buf(p.dxlow), nullptr);
+        ok(simt_maxpool_bwd_relu<T>(buf(p.act[l - 1]), buf(p.dxlow), other, B, below.H, below.W,
+                                    below.Cout, st), 1);
+      } else {
+        conv_backward(l, x, dz, B, dW, db, other, buf(p.act[l - 1]));
+      }
+      T *t = dz; dz = other; other = t;
+    }
+  }
+};
+
+int check_batch(vgg19 *n, int batch, int mode, size_t extra) {
+  if (batch < 1 || batch > n->cfg.batch_max)
+    return fail(n, VGG19_ERR_ARG, "batch %d outside [1, %d]", batch, n->cfg.batch_max);
+  Plan p = make_plan(n, batch, mode);
+  if (!n->ws) return fail(n, VGG19_ERR_WORKSPACE, "no workspace bound");
+  if (n->ws_bytes < p.total + extra)
+    return fail(n, VGG19_ERR_WORKSPACE, "workspace has %zu bytes, this call needs %zu", n->ws_bytes,
+                p.total + extra);
+  return VGG19_OK;
+}
+
+template <typename T>
+int enqueue(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st, int *launches) {
+  Pass<T> pass{n, make_plan(n, a.batch, mode), st};
+  if (mode == VGG19_MODE_FORWARD) pass.forward(a); else pass.backward(a);
+  if (launches) *launches = pass.launches;
+  n->launches[mode] = pass.launches;
+  if (pass.err != cudaSuccess)
+    return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(pass.err));
+  return VGG19_OK;
+}
+
+int enqueue_any(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st, int *launches) {
+  return n->cfg.dtype == VGG19_BF16 ? enqueue<bf16>(n, mode, a, st, launches)
+                                    : enqueue<float>(n, mode, a, st, launches);
+}
+
+// Run the pass: replay its CUDA graph when there is one for these pointers,
+// else record it first.  The legacy default stream cannot be captured, so work
+// given to it is enqueued directly.
+int run_pass(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st) {
+  if ((n->cfg.flags & VGG19_FLAG_NO_GRAPH) || st == nullptr || st == cudaStreamLegacy)
+    return enqueue_any(n, mode, a, st, nullptr);
+  const void *key[6] = {a.images, a.labels, a.logits, a.probs, a.grads, a.loss};
+  for (auto &g : n->graphs)
+    if (g.mode == mode && g.batch == a.batch && !memcmp(g.p, key, sizeof key)) {
+      CUDA_TRY(n, cudaGraphLaunch(g.exec, st));
+      return VGG19_OK;
+    }
+  cudaGraph_t graph = nullptr;
+  CUDA_TRY(n, cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+  int launches = 0;
+  int rc = enqueue_any(n, mode, a, st, &launches);
+  cudaError_t ce = cudaStreamEndCapture(st, &graph);
+  if (rc != VGG19_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+  CUDA_TRY(n, ce);
+  GraphEntry e{};
+  e.mode = mode; e.batch = a.batch; memcpy(e.p, key, sizeof key); e.n_kernels = launches;
+  cudaError_t ie = cudaGraphInstantiate(&e.exec, graph, 0);
+  cudaGraphDestroy(graph);
+  CUDA_TRY(n, ie);
+  if (n->graphs.size() >= 8) { cudaGraphExecDestroy(n->graphs.front().exec); n->graphs.erase(n->graphs.begin()); }
+  n->graphs.push_back(e);
+  CUDA_TRY(n, cudaGraphLaunch(e.exec, st));
+  return VGG19_OK;
+}
+
+void drop_graphs(vgg19 *n) {
+  for (auto &g : n->graphs) cudaGraphExecDestroy(g.exec);
+  n->graphs.clear();
+}
+
+int upload_params(vgg19 *n, const float *host) {
+  CUDA_TRY(n, cudaMemcpy(n->params, host, n->n_params * 4, cudaMemcpyHostToDevice));
+  const bool h = n->cfg.dtype == VGG19_BF16;
+  if (h) CUDA_TRY(n, convert_f32<bf16>(n->params, (bf16 *)n->params_t, n->n_params, 0));
+  for (int l = 1; l < kConvLayers; ++l) {
+    const ConvLayer &c = n->conv[l];
+    if (h)
+      CUDA_TRY(n, make_dgrad_filter<bf16>(n->params + c.w_off, (bf16 *)n->dgrad_w + c.dgrad_off, c.Cin, c.Cout, 0));
+    else
+      CUDA_TRY(n, make_dgrad_filter<float>(n->params + c.w_off, (float *)n->dgrad_w + c.dgrad_off, c.Cin, c.Cout, 0));
+  }
+  CUDA_TRY(n, cudaDeviceSynchronize());
+  return VGG19_OK;
+}
+
+int create_common(const vgg19_config *cfg, vgg19 **out) {
+  if (!cfg || !out) return fail(nullptr, VGG19_ERR_ARG, "null argument");
+  *out = nullptr;
+  if (cfg->dtype != VGG19_FP32 && cfg->dtype != VGG19_BF16)
+    return fail(nullptr, VGG19_ERR_ARG, "dtype %d is neither VGG19_FP32 nor VGG19_BF16", cfg->dtype);
+  if (cfg->height < 32 || cfg->width < 32 || cfg->height % 32 || cfg->width % 32)
+    return fail(nullptr, VGG19_ERR_SHAPE, "height %d / width %d must be positive multiples of 32",
+                cfg->height, cfg->width);
+  if (cfg->batch_max < 1) return fail(nullptr, VGG19_ERR_ARG, "batch_max %d < 1", cfg->batch_max);
+  int dev = 0;
+  cudaDeviceProp prop;
+  CUDA_TRY(nullptr, cudaGetDevice(&dev));
+  CUDA_TRY(nullptr, cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10)
+    return fail(nullptr, VGG19_ERR_UNSUPPORTED_ARCH, "device is sm_%d%d; this library is built for sm_100a only",
+                prop.major, prop.minor);
+  vgg19 *n = new (std::nothrow) vgg19();
+  if (!n) return fail(nullptr, VGG19_ERR_ARG, "out of host memory");
+  n->cfg = *cfg;
+  n->elt = cfg->dtype == VGG19_BF16 ? 2 : 4;
+  n->use_tc = cfg->dtype == VGG19_BF16 && !(cfg->flags & VGG19_FLAG_NO_TENSOR_CORES);
+  size_t off = 0, doff = 0;
+  int h = cfg->height, w = cfg->width, cin = 3, n_pool = 0;
+  for (int l = 0; l < kConvLayers; ++l) {
+    ConvLayer &c = n->conv[l];
+    n->pool_idx[l] = kPoolAfter[l] ? n_pool++ : -1;
+    c.H = h; c.W = w; c.Cin = cin; c.Cout = kConvOut[l]; c.pool_after = kPoolAfter[l];
+    c.w_off = off; off += (size_t)c.Cout * 9 * c.Cin;
+    c.b_off = off; off += c.Cout;
+    c.dgrad_off = doff;
+    if (l > 0) doff += (size_t)c.Cout * 9 * c.Cin;
+    cin = c.Cout;
+    if (c.pool_after) { h /= 2; w /= 2; }
+  }
+  const int fc_dims[4] = {512 * h * w, 4096, 4096, kClasses};
+  for (int i = 0; i < kFcLayers; ++i) {
+    FcLayer &f = n->fc[i];
+    f.In = fc_dims[i]; f.Out = fc_dims[i + 1]; f.relu = i < 2;
+    f.w_off = off; off += (size_t)f.In * f.Out;
+    f.b_off = off; off += f.Out;
+  }
+  n->n_params = off;
+  n->n_dgrad = doff;
+  cudaError_t e = cudaMalloc(&n->params, n->n_params * 4);
+  if (e == cudaSuccess) {
+    if (cfg->dtype == VGG19_BF16) e = cudaMalloc(&n->params_t, n->n_params * 2);
+    else n->params_t = n->params;
+  }
+  if (e == cudaSuccess) e = cudaMalloc(&n->dgrad_w, n->n_dgrad * n->elt);
+  if (e == cudaSuccess) e = cudaMalloc(&n->dev_error, 256);
+  if (e == cudaSuccess) e = cudaMemset(n->dev_error, 0, 256);
+  if (e != cudaSuccess) {
+    int rc = fail(nullptr, VGG19_ERR_CUDA, "allocating parameters failed: %s", cudaGetErrorString(e));
+    vgg19_destroy(n);
+    return rc;
+  }
+  *out = n;
+  return VGG19_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int vgg19_create_from_params(const vgg19_config *cfg, const float *host_params, vgg19_t **out) {
+  if (!host_params) return fail(nullptr, VGG19_ERR_ARG, "null host_params");
+  int rc = create_common(cfg, out);
+  if (rc != VGG19_OK) return rc;
+  rc = upload_params(*out, host_params);
+  if (rc != VGG19_OK) { g_create_error = (*out)->err; vgg19_destroy(*out); *out = nullptr; }
+  return rc;
+}
+
+int vgg19_create(const vgg19_config *cfg, uint64_t seed, vgg19_t **out) {
+  int rc = create_common(cfg, out);
+  if (rc != VGG19_OK) return rc;
+  std::vector<float> host;
+  try { host.resize((*out)->n_params); } catch (...) {
+    vgg19_destroy(*out); *out = nullptr;
+    return fail(nullptr, VGG19_ERR_ARG, "out of host memory");
+  }
+  seeded_vgg19_params(host.data(), cfg->height, cfg->width, seed, 0.0, 0);
+  rc = upload_params(*out, host.data());
+  if (rc != VGG19_OK) { g_create_error = (*out)->err; vgg19_destroy(*out); *out = nullptr; }
+  return rc;
+}
+
+void vgg19_destroy(vgg19_t *n) {
+  if (!n) return;
+  drop_graphs(n);
+  if (n->params_t && n->params_t != (void *)n->params) cudaFree(n->params_t);
+  if (n->params) cudaFree(n->params);
+  if (n->dgrad_w) cudaFree(n->dgrad_w);
+  if (n->dev_error) cudaFree(n->dev_error);
+  delete n;
+}
+
+int vgg19_param_count(const vgg19_t *n, int32_t *n_tensors, size_t *n_elems) {
+  if (!n) return VGG19_ERR_ARG;
+  if (n_tensors) *n_tensors = 2 * kLayers;
+  if (n_elems) *n_elems = n->n_params;
+  return VGG19_OK;
+}
+
+int vgg19_param_info(const vgg19_t *n, int32_t i, size_t *offset, int32_t *rank, int64_t dims[4]) {
+  if (!n || i < 0 || i >= 2 * kLayers) return VGG19_ERR_ARG;
+  int l = i / 2;
+  bool bias = i & 1;
+  int64_t d[4] = {0, 0, 0, 0};
+  int r;
+  size_t off;
+  if (l < kConvLayers) {
+    const ConvLayer &c = n->conv[l];
+    if (bias) { r = 1; d[0] = c.Cout; off = c.b_off; }
+    else { r = 4; d[0] = c.Cout; d[1] = 3; d[2] = 3; d[3] = c.Cin; off = c.w_off; }
+  } else {
+    const FcLayer &f = n->fc[l - kConvLayers];
+    if (bias) { r = 1; d[0] = f.Out; off = f.b_off; }
+    else { r = 2; d[0] = f.Out; d[1] = f.In; off = f.w_off; }
+  }
+  if (offset) *offset = off;
+  if (rank) *rank = r;
+  if (dims) memcpy(dims, d, sizeof d);
+  return VGG19_OK;
+}
+
+int vgg19_get_params(const vgg19_t *n, float *host) {
+  if (!n || !host) return VGG19_ERR_ARG;
+  return cudaMemcpy(host, n->params, n->n_params * 4, cudaMemcpyDeviceToHost) == cudaSuccess
+             ? VGG19_OK : VGG19_ERR_CUDA;
+}
+
+int vgg19_set_params(vgg19_t *n, const float *host) {
+  if (!n || !host) return VGG19_ERR_ARG;
+  CUDA_TRY(n, cudaDeviceSynchronize());
+  return upload_params(n, host);
+}
+
+size_t vgg19_workspace_bytes(const vgg19_t *n, int32_t batch, int32_t mode) {
+  if (!n || batch < 1 || batch > n->cfg.batch_max || (mode != 0 && mode != 1)) return 0;
+  return make_plan(n, batch, mode).total;
+}
+
+size_t vgg19_io_bytes(const vgg19_t *n, int32_t batch, int32_t mode) {
+  if (!n || batch < 1 || batch > n->cfg.batch_max || (mode != 0 && mode != 1)) return 0;
+  return make_plan(n, batch, mode).io_total;
+}
+
+int vgg19_bind_workspace(vgg19_t *n, void *ws, size_t bytes) {
+  if (!n) return VGG19_ERR_ARG;
+  if (ws && (reinterpret_cast<uintptr_t>(ws) & 255))
+    return fail(n, VGG19_ERR_ARG, "workspace must be 256-byte aligned");
+  drop_graphs(n);
+  n->ws = ws;
+  n->ws_bytes = ws ? bytes : 0;
+  return VGG19_OK;
+}
+
+int vgg19_forward(vgg19_t *n, const void *images, int32_t batch, float *logits, float *probs,
+                  void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!images || !logits) return fail(n, VGG19_ERR_ARG, "images and logits must not be null");
+  int rc = check_batch(n, batch, VGG19_MODE_FORWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  PassArgs a{images, nullptr, logits, probs, nullptr, nullptr, batch};
+  return run_pass(n, VGG19_MODE_FORWARD, a, static_cast<cudaStream_t>(stream));
+}
+
+int vgg19_backward(vgg19_t *n, const void *images, const int32_t *labels, int32_t batch,
+                   float *grads, float *loss, float *logits, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!images || !labels || !grads)
+    return fail(n, VGG19_ERR_ARG, "images, labels and grads must not be null");
+  int rc = check_batch(n, batch, VGG19_MODE_BACKWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  PassArgs a{images, labels, logits, nullptr, grads, loss, batch};
+  return run_pass(n, VGG19_MODE_BACKWARD, a, static_cast<cudaStream_t>(stream));
+}
+
+int vgg19_forward_host(vgg19_t *n, const void *host_images, int32_t batch, float *host_logits,
+                       float *host_probs, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!host_images) return fail(n, VGG19_ERR_ARG, "host_images must not be null");
+  int rc = check_batch(n, batch, VGG19_MODE_FORWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  Plan p = make_plan(n, batch, VGG19_MODE_FORWARD);
+  rc = check_batch(n, batch, VGG19_MODE_FORWARD, p.io_total);
+  if (rc != VGG19_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char *base = static_cast<char *>(n->ws);
+  size_t img_bytes = (size_t)batch * n->cfg.height * n->cfg.width * 3 * n->elt;
+  CUDA_TRY(n, cudaMemcpyAsync(base + p.io_images, host_images, img_bytes, cudaMemcpyHostToDevice, st));
+  float *logits = reinterpret_cast<float *>(base + p.io_logits);
+  float *probs = host_probs ? reinterpret_cast<float *>(base + p.io_probs) : nullptr;
+  PassArgs a{base + p.io_images, nullptr, logits, probs, nullptr, nullptr, batch};
+  rc = run_pass(n, VGG19_MODE_FORWARD, a, st);
+  if (rc != VGG19_OK) return rc;
+  size_t out_bytes = (size_t)batch * kClasses * 4;
+  if (host_logits) CUDA_TRY(n, cudaMemcpyAsync(host_logits, logits, out_bytes, cudaMemcpyDeviceToHost, st));
+  if (host_probs) CUDA_TRY(n, cudaMemcpyAsync(host_probs, probs, out_bytes, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(n, cudaStreamSynchronize(st));
+  return VGG19_OK;
+}
+
+int vgg19_backward_host(vgg19_t *n, const void *host_images, const int32_t *host_labels,
+                        int32_t batch, float *host_grads, float *host_loss, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!host_images || !host_labels) return fail(n, VGG19_ERR_ARG, "host_images and host_labels must not be null");
+  int rc = check_batch(n, batch, VGG19_MODE_BACKWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  Plan p = make_plan(n, batch, VGG19_MODE_BACKWARD);
+  rc = check_batch(n, batch, VGG19_MODE_BACKWARD, p.io_total);
+  if (rc != VGG19_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char *base = static_cast<char *>(n->ws);
+  size_t img_bytes = (size_t)batch * n->cfg.height * n->cfg.width * 3 * n->elt;
+  CUDA_TRY(n, cudaMemcpyAsync(base + p.io_images, host_images, img_bytes, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(n, cudaMemcpyAsync(base + p.io_labels, host_labels, (size_t)batch * 4, cudaMemcpyHostToDevice, st));
+  float *grads = reinterpret_cast<float *>(base + p.io_grads);
+  float *loss = reinterpret_cast<float *>(base + p.io_loss);
+  PassArgs a{base + p.io_images, reinterpret_cast<const int32_t *>(base + p.io_labels), nullptr,
+             nullptr, grads, loss, batch};
+  rc = run_pass(n, VGG19_MODE_BACKWARD, a, st);
+  if (rc != VGG19_OK) return rc;
+  if (host_grads) CUDA_TRY(n, cudaMemcpyAsync(host_grads, grads, n->n_params * 4, cudaMemcpyDeviceToHost, st));
+  if (host_loss) CUDA_TRY(n, cudaMemcpyAsync(host_loss, loss, 4, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(n, cudaStreamSynchronize(st));
+  return VGG19_OK;
+}
+
+int vgg19_conv_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t batch, void *y,
+                             void *pooled, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (layer < 1 || layer > kConvLayers || !x || !y || batch < 1)
+    return fail(n, VGG19_ERR_ARG, "bad layer (%d), batch (%d) or null tensor", layer, batch);
+  if (pooled && !n->conv[layer - 1].pool_after) {
+    // pooling after any layer is well defined; only the fused schedule is per-layer
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  if (n->cfg.dtype == VGG19_BF16) {
+    Pass<bf16> ps{n, Plan{}, st};
+    ps.conv_forward(layer - 1, (const bf16 *)x, batch, (bf16 *)y, (bf16 *)pooled);
+    e = ps.err;
+  } else {
+    Pass<float> ps{n, Plan{}, st};
+    ps.conv_forward(layer - 1, (const float *)x, batch, (float *)y, (float *)pooled);
+    e = ps.err;
+  }
+  if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  return VGG19_OK;
+}
+
+int vgg19_conv_layer_backward(vgg19_t *n, int32_t layer, const void *x, const void *dz,
+                              int32_t batch, float *dw, float *db, void *dx, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (layer < 1 || layer > kConvLayers || !x || !dz || !dw || !db || batch < 1)
+    return fail(n, VGG19_ERR_ARG, "bad layer (%d), batch (%d) or null tensor", layer, batch);
+  if (dx && layer == 1) return fail(n, VGG19_ERR_ARG, "layer 1 has no input gradient");
+  int rc = check_batch(n, batch, VGG19_MODE_BACKWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Plan p = make_plan(n, batch, VGG19_MODE_BACKWARD);
+  cudaError_t e;
+  if (n->cfg.dtype == VGG19_BF16) {
+    Pass<bf16> ps{n, p, st};
+    ps.conv_backward(layer - 1, (const bf16 *)x, (const bf16 *)dz, batch, dw, db, (bf16 *)dx, nullptr);
+    e = ps.err;
+  } else {
+    Pass<float> ps{n, p, st};
+    ps.conv_backward(layer - 1, (const float *)x, (const float *)dz, batch, dw, db, (float *)dx, nullptr);
+    e = ps.err;
+  }
+  if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  return VGG19_OK;
+}
+
+int vgg19_sync_status(vgg19_t *n, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  CUDA_TRY(n, cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  int code = 0;
+  CUDA_TRY(n, cudaMemcpy(&code, n->dev_error, sizeof code, cudaMemcpyDeviceToHost));
+  if (code != 0) {
+    cudaMemset(n->dev_error, 0, 256);
+    return fail(n, VGG19_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (code %d)", code);
+  }
+  return VGG19_OK;
+}
+
+int vgg19_launch_count(const vgg19_t *n, int32_t mode, int32_t *n_kernels) {
+  if (!n || !n_kernels || (mode != 0 && mode != 1)) return VGG19_ERR_ARG;
+  *n_kernels = n->launches[mode];
+  return VGG19_OK;
+}
+
+int vgg19_describe(const vgg19_t *n, char *out, size_t cap) {
+  if (!n) return VGG19_ERR_ARG;
+  std::string s;
+  char line[256];
+  snprintf(line, sizeof line, "vgg19 %dx%dx3 dtype=%s batch_max=%d params=%zu\n", n->cfg.height,
+           n->cfg.width, n->cfg.dtype == VGG19_BF16 ? "bf16" : "fp32", n->cfg.batch_max, n->n_params);
+  s += line;
+  for (int l = 0; l < kConvLayers; ++l) {
+    const ConvLayer &c = n->conv[l];
+    ConvShape sh{n->cfg.batch_max, c.H, c.W, c.Cin, c.Cout};
+    ConvShape sd{n->cfg.batch_max, c.H, c.W, c.Cout, c.Cin};
+    snprintf(line, sizeof line, "conv%-2d %3dx%-3d %3d->%-3d +bias +relu%s  fwd=%s dgrad=%s wgrad=%s\n",
+             l + 1, c.H, c.W, c.Cin, c.Cout, c.pool_after ? " +maxpool2x2" : "",
+             n->use_tc && tc_conv3x3_supported(sh) ? "tcgen05" : "simt",
+             l == 0 ? "none" : (n->use_tc && tc_conv3x3_supported(sd) ? "tcgen05" : "simt"),
+             n->use_tc && tc_wgrad_supported(sh) ? "tcgen05" : "simt");
+    s += line;
+  }
+  for (int i = 0; i < kFcLayers; ++i) {
+    const FcLayer &f = n->fc[i];
+    snprintf(line, sizeof line, "dense%d %5d->%-4d +bias%s\n", i + 1, f.In, f.Out, f.relu ? " +relu" : "");
+    s += line;
+  }
+  s += "softmax 1000\n";
+  snprintf(line, sizeof line, "counts: convolution=16 reduce-window=5 dot=3 relu=18 softmax=1 rng=0\n");
+  s += line;
+  if (out && cap) {
+    size_t k = s.size() < cap - 1 ? s.size() : cap - 1;
+    memcpy(out, s.data(), k);
+    out[k] = 0;
+  }
+  return (int)s.size();
+}
+
+const char *vgg19_last_error(const vgg19_t *n) { return n ? n->err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

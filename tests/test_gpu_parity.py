@@ -1,0 +1,206 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU
+checker on the same seeded inputs.
+
+Tolerances.  fp32 configuration: relative L2 error of the logits <= 1e-4 (the
+stated bar); gradients <= 2e-4 (fp32 FMA sums of up to ~25k terms, two passes
+through the network).  bf16 configurations (fp32 accumulation): relative L2
+<= 2e-2 on the logits and on each of the 38 gradient tensors, against the
+checker run with the configuration's storage format (activations and
+activation gradients rounded to bf16 where they are stored, arithmetic in
+fp64), so that ReLU masks and pool arg-maxima are decided on the same stored
+values on both sides.  The logits are also held to 2e-2 against the checker
+with nothing rounded.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import seeded_inputs as si
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def pkg():
+    import paper_1810_09868_b200 as p
+    return p
+
+
+def rel_l2(a, b):
+    a, b = np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def make_inputs(H, W, B, bf16, bias_std=0.0):
+    params = si.vgg19_params(H, W, seed=0, bias_std=bias_std, bf16_exact=bf16)
+    images = si.images(B, H, W, seed=1, bf16_exact=bf16)
+    labels = si.labels(B, seed=2)
+    return params, images, labels
+
+
+def run_backward(net, images, labels):
+    x = torch.from_numpy(images).to(DEV).to(net.act_dtype)
+    y = torch.from_numpy(labels).to(DEV)
+    logits = torch.empty(images.shape[0], 1000, dtype=torch.float32, device=DEV)
+    grads, loss = net.backward(x, y, logits=logits)
+    net.sync_status()
+    return logits.cpu().numpy(), grads.cpu().numpy(), float(loss.item())
+
+
+def check_grads(net, grads, o_grads, tol):
+    worst = []
+    for i, (off, dims) in enumerate(net.param_slices()):
+        n = int(np.prod(dims))
+        e = rel_l2(grads[off:off + n], o_grads[off:off + n])
+        worst.append((e, i, dims))
+    bad = [w for w in worst if not w[0] <= tol]
+    assert not bad, f"gradient tensors above {tol}: {bad}"
+    return max(w[0] for w in worst)
+
+
+def test_config1_fp32_forward_32x32_batch1():
+    p = pkg()
+    params, images, _ = make_inputs(32, 32, 1, False)
+    net = p.Net(32, 32, 1, p.VGG19_FP32, params=params, mode=p.VGG19_MODE_FORWARD)
+    x = torch.from_numpy(images).to(DEV)
+    probs = torch.empty(1, 1000, dtype=torch.float32, device=DEV)
+    logits = net.forward(x, probs=probs)
+    net.sync_status()
+    o = oracle.vgg19_forward(params.astype(np.float64), images)
+    assert rel_l2(logits.cpu().numpy(), o) <= 1e-4
+    assert rel_l2(probs.cpu().numpy(), oracle.softmax(o)) <= 1e-4
+    assert int(logits.argmax()) == int(o.argmax())
+    net.close()
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_fp32_backward_32x32(flags):
+    p = pkg()
+    B = 3
+    params, images, labels = make_inputs(32, 32, B, False, bias_std=0.05)
+    net = p.Net(32, 32, B, p.VGG19_FP32, params=params, flags=flags)
+    logits, grads, loss = run_backward(net, images, labels)
+    o_loss, o_grads, o_logits = oracle.vgg19_backward(params.astype(np.float64), images, labels, chunk=B)
+    assert rel_l2(logits, o_logits) <= 1e-4
+    assert abs(loss - o_loss) <= 1e-4 * abs(o_loss)
+    check_grads(net, grads, o_grads, 2e-4)
+    net.close()
+
+
+@pytest.mark.parametrize("flags", [0, 2])
+def test_bf16_backward_32x32(flags):
+    p = pkg()
+    B = 5
+    params, images, labels = make_inputs(32, 32, B, True, bias_std=0.05)
+    net = p.Net(32, 32, B, p.VGG19_BF16, params=params, flags=flags)
+    logits, grads, loss = run_backward(net, images, labels)
+    o_loss, o_grads, o_logits = oracle.vgg19_backward(params.astype(np.float64), images, labels, chunk=B,
+                                                      storage="bf16")
+    assert rel_l2(logits, o_logits) <= 2e-2
+    assert rel_l2(logits, oracle.vgg19_forward(params.astype(np.float64), images)) <= 2e-2
+    assert abs(loss - o_loss) <= 2e-2 * abs(o_loss)
+    worst = check_grads(net, grads, o_grads, 2e-2)
+    print(f"bf16 32x32 B={B} flags={flags}: logits {rel_l2(logits, o_logits):.2e} worst grad {worst:.2e}")
+    net.close()
+
+
+def test_smaller_batch_than_batch_max_and_ragged_sizes():
+    p = pkg()
+    params, images, labels = make_inputs(64, 32, 3, True)
+    net = p.Net(64, 32, 7, p.VGG19_BF16, params=params)
+    logits, grads, loss = run_backward(net, images, labels)
+    o_loss, o_grads, o_logits = oracle.vgg19_backward(params.astype(np.float64), images, labels, chunk=3,
+                                                      storage="bf16")
+    assert rel_l2(logits, o_logits) <= 2e-2
+    check_grads(net, grads, o_grads, 2e-2)
+    net.close()
+
+
+def test_graph_replay_is_bit_identical_and_matches_direct_launch():
+    p = pkg()
+    params, images, _ = make_inputs(32, 32, 2, True)
+    x = torch.from_numpy(images).to(DEV).to(torch.bfloat16)
+    outs = []
+    for flags in (0, p.VGG19_FLAG_NO_GRAPH):
+        net = p.Net(32, 32, 2, p.VGG19_BF16, params=params, flags=flags, mode=p.VGG19_MODE_FORWARD)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            a = net.forward(x, stream=s).clone()
+            b = net.forward(x, stream=s).clone()
+            c = net.forward(x, stream=s).clone()
+        net.sync_status(s)
+        assert torch.equal(a, b) and torch.equal(b, c)
+        outs.append(a.cpu())
+        assert p.vgg19_launch_count(net.handle, p.VGG19_MODE_FORWARD) >= 16 + 5 + 3
+        net.close()
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_seeded_create_matches_the_generator_and_get_set_params():
+    p = pkg()
+    h = p.vgg19_create(32, 32, 1, p.VGG19_FP32, 0)
+    n_t, n_e = p.vgg19_param_count(h)
+    assert n_t == 38 and n_e == 43003944
+    host = np.empty(n_e, dtype=np.float32)
+    p.vgg19_get_params(h, host)
+    assert np.array_equal(host, si.vgg19_params(32, 32, seed=0))
+    other = si.vgg19_params(32, 32, seed=5)
+    p.vgg19_set_params(h, other)
+    p.vgg19_get_params(h, host)
+    assert np.array_equal(host, other)
+    off, dims = p.vgg19_param_info(h, 0)
+    assert off == 0 and dims == (64, 3, 3, 3)
+    off, dims = p.vgg19_param_info(h, 32)
+    assert dims == (4096, 512)
+    text = p.vgg19_describe(h)
+    assert text.count("conv") >= 16 and "convolution=16 reduce-window=5 dot=3" in text
+    p.vgg19_destroy(h)
+
+
+def test_error_codes_on_a_device():
+    p = pkg()
+    h = p.vgg19_create(32, 32, 2, p.VGG19_BF16, 0)
+    x = torch.zeros(2, 32, 32, 3, dtype=torch.bfloat16, device=DEV)
+    out = torch.zeros(2, 1000, device=DEV)
+    with pytest.raises(p.binding.Vgg19Error) as e:
+        p.vgg19_forward(h, x, 2, out)
+    assert e.value.code == p.VGG19_ERR_WORKSPACE
+    need = p.vgg19_workspace_bytes(h, 2, p.VGG19_MODE_FORWARD)
+    assert need > 0 and p.vgg19_workspace_bytes(h, 3, p.VGG19_MODE_FORWARD) == 0
+    ws = torch.empty(need - 256, dtype=torch.uint8, device=DEV)
+    p.vgg19_bind_workspace(h, ws, need - 256)
+    with pytest.raises(p.binding.Vgg19Error) as e:
+        p.vgg19_forward(h, x, 2, out)
+    assert e.value.code == p.VGG19_ERR_WORKSPACE
+    with pytest.raises(p.binding.Vgg19Error) as e:
+        p.vgg19_forward(h, x, 3, out)
+    assert e.value.code == p.VGG19_ERR_ARG
+    with pytest.raises(p.binding.Vgg19Error) as e:
+        p.vgg19_forward(h, None, 2, out)
+    assert e.value.code == p.VGG19_ERR_ARG
+    p.vgg19_destroy(h)
+
+
+def test_host_buffer_entry_points():
+    p = pkg()
+    B = 2
+    params, images, labels = make_inputs(32, 32, B, True)
+    net = p.Net(32, 32, B, p.VGG19_BF16, params=params, host_io=True)
+    x_host = torch.from_numpy(images).to(torch.bfloat16).pin_memory()
+    logits_host = torch.empty(B, 1000, dtype=torch.float32).pin_memory()
+    probs_host = torch.empty(B, 1000, dtype=torch.float32).pin_memory()
+    s = torch.cuda.Stream()
+    p.vgg19_forward_host(net.handle, x_host, B, logits_host, probs_host, s)
+    dev_logits = net.forward(x_host.to(DEV))
+    torch.cuda.synchronize()
+    assert torch.equal(dev_logits.cpu(), logits_host)
+    np.testing.assert_allclose(probs_host.sum(1).numpy(), 1.0, rtol=1e-5)
+    grads_host = torch.empty(net.n_params, dtype=torch.float32).pin_memory()
+    loss_host = torch.empty(1, dtype=torch.float32).pin_memory()
+    p.vgg19_backward_host(net.handle, x_host, torch.from_numpy(labels), B, grads_host, loss_host, s)
+    grads, loss = net.backward(x_host.to(DEV), torch.from_numpy(labels).to(DEV))
+    torch.cuda.synchronize()
+    assert torch.equal(grads.cpu(), grads_host) and float(loss) == float(loss_host)
+    net.close()

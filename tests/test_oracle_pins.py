@@ -232,6 +232,38 @@ def test_softmax_jacobian_of_sum_vanishes():
     np.testing.assert_allclose(oracle.softmax_bwd(pr, g), tl.grad.numpy(), rtol=1e-12, atol=1e-15)
 
 
+def test_round_bf16_against_torch_and_on_ties():
+    v = np.concatenate([rng.standard_normal(20000) * 10.0 ** rng.integers(-30, 30, 20000),
+                        np.array([0.0, -0.0, 1.0, -1.0, 2.0 ** -126, 2.0 ** -133, 3.0 * 2.0 ** -134])])
+    v = v.astype(np.float32)  # torch rounds from fp32; these are exact doubles too
+    ref = torch.from_numpy(v).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(oracle.round_bf16(v.astype(np.float64)), ref)
+    # ties go to the even 8-bit significand: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert oracle.round_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert oracle.round_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+    assert oracle.round_bf16(np.array([1.0 + 2.0 ** -8 + 2.0 ** -40]))[0] == 1.0 + 2.0 ** -7
+    # a value that fp32 double rounding would get wrong is rounded once, from fp64
+    x = 1.0 + 2.0 ** -8 + 2.0 ** -30  # fp32 would first drop 2^-30, then tie to even -> 1.0
+    assert oracle.round_bf16(np.array([x]))[0] == 1.0 + 2.0 ** -7
+    r = oracle.round_bf16(rng.standard_normal(1000))
+    assert np.array_equal(oracle.round_bf16(r), r)
+
+
+def test_bf16_storage_model_only_rounds_what_is_stored():
+    params, x, labels = tiny_inputs()
+    params, x = oracle.round_bf16(params), oracle.round_bf16(x)
+    l64 = oracle.forward(TINY, params, x)
+    l16, saved = oracle.forward(TINY, params, x, keep=True, storage="bf16")
+    assert 0 < np.abs(l16 - l64).max() < 0.05 * np.abs(l64).max()
+    for sv in saved:
+        if sv[0] == "conv":
+            assert np.array_equal(oracle.round_bf16(sv[2]), sv[2])
+    _, g64, _ = oracle.backward(TINY, params, x, labels)
+    _, g16, _ = oracle.backward(TINY, params, x, labels, storage="bf16")
+    rel = np.linalg.norm(g16 - g64) / np.linalg.norm(g64)
+    assert 0 < rel < 0.1
+
+
 # ------------------------------------------------------------- whole networks
 
 TINY = [("conv", 3), ("conv", 4), ("pool",), ("conv", 2), ("pool",), ("fc", 6, True), ("fc", 5, True), ("fc", 3, False)]
