@@ -144,6 +144,17 @@ int vgg19_conv_layer_forward(vgg19_t *net, int32_t layer, const void *x, int32_t
 int vgg19_conv_layer_backward(vgg19_t *net, int32_t layer, const void *x, const void *dz,
                               int32_t batch, float *dw, float *db, void *dx, void *stream);
 
+/* Where a pass at `batch` in `mode` leaves the activations it stores, as a
+ * byte offset into the bound workspace, so that a caller can inspect the
+ * forward state a backward pass differentiated (the ReLU masks and pool
+ * arg-maxima of section 7.3 are decided on exactly these stored values).
+ * index 0..15: output of conv layer index+1 after bias and ReLU,
+ * [batch][h][w][Cout]; 16..20: outputs of the five max-pools; 21, 22: outputs
+ * of dense layers 1 and 2 after ReLU, [batch][4096] (dims[2] = dims[3] = 1).
+ * Element type is the config's dtype. */
+int vgg19_saved_tensor(const vgg19_t *net, int32_t batch, int32_t mode, int32_t index,
+                       size_t *offset_bytes, int64_t dims[4]);
+
 /* Wait for the stream and report any device-side error recorded so far. */
 int vgg19_sync_status(vgg19_t *net, void *stream);
 

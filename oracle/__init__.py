@@ -302,7 +302,29 @@ def forward(steps, params, images, keep=False, storage=None):
     return (x, saved) if keep else x
 
 
-def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_kind="ce", storage=None):
+def state_from_outputs(steps, images, outputs):
+    """Rebuild the saved forward state from the stored output of every step
+    (conv: y after ReLU; pool: pooled tensor; fc: activation, logits for the
+    last), e.g. as read back from a device.  Returns (logits, saved) in the
+    form forward(keep=True) returns, so that backward() can differentiate the
+    network at exactly that state: given the stored activations, the ReLU
+    masks and pool arg-maxima are fixed and the gradient is unique."""
+    x = _c(images)
+    saved = []
+    for st, out in zip(steps, outputs):
+        out = _c(out)
+        if st[0] == "conv":
+            saved.append(("conv", x, out))
+        elif st[0] == "pool":
+            saved.append(("pool", x))
+        else:
+            saved.append(("fc", x.reshape(x.shape[0], -1), out, x.shape, st[2]))
+        x = out
+    return x, saved
+
+
+def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_kind="ce", storage=None,
+             state=None):
     """Gradient of the loss with respect to every parameter, flat, in the
     parameter order.  loss_kind "ce": mean cross-entropy of softmax(logits)
     (dlogits = (p - onehot) / n_total).  loss_kind "sum": the paper's
@@ -310,7 +332,9 @@ def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_
     result is accumulated into it (chunked batches).  With storage="bf16"
     the gradients the configuration keeps in memory between layers (dlogits
     and every activation gradient) are rounded to bf16 where they are stored;
-    parameter gradients are never rounded.  Returns (loss, grads, logits)."""
+    parameter gradients are never rounded.  With state=(logits, saved) the
+    forward pass is not run and the network is differentiated at that given
+    forward state.  Returns (loss, grads, logits)."""
     params = _c(params)
     images = _c(images)
     N = images.shape[0]
@@ -320,7 +344,10 @@ def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_
     if grads is None:
         grads = np.zeros_like(params)
     G = split_params(grads, shapes)
-    logits, saved = forward(steps, params, images, keep=True, storage=storage)
+    if state is None:
+        logits, saved = forward(steps, params, images, keep=True, storage=storage)
+    else:
+        logits, saved = state
     p = softmax(logits)
     if loss_kind == "ce":
         loss = cross_entropy(logits, labels, n_total)

@@ -55,6 +55,15 @@ class Net:
         binding.vgg19_backward(self.handle, images, labels, B, grads, loss, logits, stream)
         return grads, loss
 
+    def saved_tensor(self, batch, mode, index):
+        """View of a stored activation inside the workspace (no copy)."""
+        off, dims = binding.vgg19_saved_tensor(self.handle, batch, mode, index)
+        n = 1
+        for d in dims:
+            n *= d
+        elt = 2 if self.dtype == binding.VGG19_BF16 else 4
+        return self.workspace[off:off + n * elt].view(self.act_dtype).view(*dims)
+
     def param_slices(self):
         """[(offset, dims)] of the 38 tensors in the flat parameter buffer."""
         return [binding.vgg19_param_info(self.handle, i) for i in range(self.n_tensors)]

@@ -635,6 +635,29 @@ int vgg19_conv_layer_backward(vgg19_t *n, int32_t layer, const void *x, const vo
   return VGG19_OK;
 }
 
+int vgg19_saved_tensor(const vgg19_t *n, int32_t batch, int32_t mode, int32_t index,
+                       size_t *offset_bytes, int64_t dims[4]) {
+  if (!n || !offset_bytes || !dims || batch < 1 || batch > n->cfg.batch_max || (mode != 0 && mode != 1) ||
+      index < 0 || index > 22)
+    return VGG19_ERR_ARG;
+  Plan p = make_plan(n, batch, mode);
+  if (index < kConvLayers) {
+    const ConvLayer &c = n->conv[index];
+    *offset_bytes = p.act[index];
+    dims[0] = batch; dims[1] = c.H; dims[2] = c.W; dims[3] = c.Cout;
+  } else if (index < kConvLayers + 5) {
+    int l = 0;
+    while (n->pool_idx[l] != index - kConvLayers) ++l;
+    const ConvLayer &c = n->conv[l];
+    *offset_bytes = p.pooled[index - kConvLayers];
+    dims[0] = batch; dims[1] = c.H / 2; dims[2] = c.W / 2; dims[3] = c.Cout;
+  } else {
+    *offset_bytes = index == 21 ? p.a1 : p.a2;
+    dims[0] = batch; dims[1] = 4096; dims[2] = 1; dims[3] = 1;
+  }
+  return VGG19_OK;
+}
+
 int vgg19_sync_status(vgg19_t *n, void *stream) {
   if (!n) return VGG19_ERR_ARG;
   CUDA_TRY(n, cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));

@@ -264,6 +264,24 @@ def test_bf16_storage_model_only_rounds_what_is_stored():
     assert 0 < rel < 0.1
 
 
+def test_backward_at_a_given_forward_state_reproduces_backward():
+    params, x, labels = tiny_inputs()
+    loss, grads, logits = oracle.backward(TINY, params, x, labels)
+    _, saved = oracle.forward(TINY, params, x, keep=True)
+    outputs = []
+    for st, sv in zip(TINY, saved):
+        outputs.append(sv[2] if st[0] in ("conv", "fc") else None)
+    # pool outputs are the next step's input
+    for i, st in enumerate(TINY):
+        if st[0] == "pool":
+            nxt = saved[i + 1]
+            outputs[i] = nxt[1] if nxt[0] == "conv" else nxt[1].reshape(nxt[3])
+    lg2, state = oracle.state_from_outputs(TINY, x, outputs)
+    assert np.array_equal(lg2, logits)
+    loss2, grads2, _ = oracle.backward(TINY, params, x, labels, state=(lg2, state))
+    assert loss2 == loss and np.array_equal(grads2, grads)
+
+
 # ------------------------------------------------------------- whole networks
 
 TINY = [("conv", 3), ("conv", 4), ("pool",), ("conv", 2), ("pool",), ("fc", 6, True), ("fc", 5, True), ("fc", 3, False)]
