@@ -1,0 +1,327 @@
+"""Benchmark of the VGG19 pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One "step" is one forward pass of the whole network on a batch of 100
+224x224x3 bf16 images (the paper's headline shape, figure "Timings for the
+VGG19 forward pass", N=100).  Rank 0 prints ONE JSON line: images/s with the
+inputs resident in HBM (`value`), the same through the host-buffer entry point
+with copies inside the timed region (`e2e`), the forward+backward training-step
+throughput (`fwd_bwd`), the roofline of the dominant kernel (the tensor-core
+implicit-GEMM convolution, timed per layer with CUDA events), and the fp64 CPU
+checker timed on a bounded sample (`cpu_baseline`).
+
+With N > 1 (torchrun) every rank runs the same batch-100 pass on its own GPU:
+the path shards over the batch with no collective in the forward pass, so the
+aggregate is N * 100 images per step over the slowest rank's time.
+
+--impl reference times the CPU checker itself (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "VGG19 fwd images/s @batch 100, 224x224 bf16"
+WORKLOAD = "configs[3]: full VGG19 forward, 224x224x3, batch 100, bf16 storage, fp32 accumulate"
+H = W = 224
+BATCH = 100
+CONV = [(224, 3, 64), (224, 64, 64), (112, 64, 128), (112, 128, 128), (56, 128, 256), (56, 256, 256),
+        (56, 256, 256), (56, 256, 256), (28, 256, 512), (28, 512, 512), (28, 512, 512), (28, 512, 512),
+        (14, 512, 512), (14, 512, 512), (14, 512, 512), (14, 512, 512)]
+FWD_FLOP_PER_IMAGE = sum(2 * s * s * co * 9 * ci for s, ci, co in CONV) + 2 * (25088 * 4096 + 4096 * 4096 + 4096 * 1000)
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_forward_rate(n_images, seed_offset=0):
+    """images/s of the fp64 CPU checker's forward pass on n_images of the workload."""
+    import numpy as np
+    import oracle
+    import seeded_inputs as si
+    params = si.vgg19_params(H, W, seed=0, bf16_exact=True).astype(np.float64)
+    images = si.images(BATCH, H, W, seed=1, bf16_exact=True)[seed_offset:seed_offset + n_images]
+    oracle.vgg19_forward(params, images[:1])  # page in code and weights
+    t0 = time.perf_counter()
+    oracle.vgg19_forward(params, images)
+    dt = time.perf_counter() - t0
+    return n_images / dt, dt
+
+
+def run_reference(args):
+    """The CPU checker as it stands, timed on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    import seeded_inputs as si
+    per_step = 1
+    params = si.vgg19_params(H, W, seed=0, bf16_exact=True).astype(np.float64)
+    images = si.images(BATCH, H, W, seed=1, bf16_exact=True)
+    for i in range(args.warmup):
+        oracle.vgg19_forward(params, images[i % BATCH:i % BATCH + per_step])
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        j = (args.warmup + i) % BATCH
+        oracle.vgg19_forward(params, images[j:j + per_step])
+    dt = time.perf_counter() - t0
+    value = per_step * args.steps / dt
+    cores = os.cpu_count()
+    sample = f"{per_step} image(s) of the batch of 100 per step, {args.steps} steps, forward only"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "note": "fp64 CPU checker, OpenMP over rows; bounded sample"},
+        "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def time_conv_layers(pkg, net, torch, stream, reps=5):
+    """Per-layer CUDA-event timing of the convolution kernel on the batch-100 activations
+    left in the workspace by a forward pass.  Returns [(layer, ms, flop, path)]."""
+    out = []
+    desc = pkg.vgg19_describe(net.handle).splitlines()
+    scratch = torch.empty(BATCH * 224 * 224 * 64, dtype=torch.bfloat16, device=net.device)
+    for l, (s, ci, co) in enumerate(CONV):
+        if l == 0:
+            continue  # 3 input channels: HBM-bound CUDA-core kernel, not the tensor-core one
+        prev = l - 1
+        x = net.saved_tensor(BATCH, pkg.VGG19_MODE_BACKWARD, prev)
+        if x.shape[1] != s:  # a pool sits between: input is the pooled tensor
+            pool_index = {1: 16, 3: 17, 7: 18, 11: 19, 15: 20}[prev]
+            x = net.saved_tensor(BATCH, pkg.VGG19_MODE_BACKWARD, pool_index)
+        path = "tcgen05" if "fwd=tcgen05" in desc[1 + l] else "simt"
+        with torch.cuda.stream(stream):
+            for _ in range(2):
+                pkg.vgg19_conv_layer_forward(net.handle, l + 1, x, BATCH, scratch, None, stream)
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+            for a, b in evs:
+                a.record(stream)
+                pkg.vgg19_conv_layer_forward(net.handle, l + 1, x, BATCH, scratch, None, stream)
+                b.record(stream)
+        stream.synchronize()
+        ms = sum(a.elapsed_time(b) for a, b in evs) / reps
+        out.append((l + 1, ms, 2.0 * BATCH * s * s * co * 9 * ci, path))
+    return out
+
+
+def run_native(args):
+    import numpy as np
+    import torch
+    import seeded_inputs as si
+    import paper_1810_09868_b200 as pkg
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    params = si.vgg19_params(H, W, seed=0, bf16_exact=True)
+    images = si.images(BATCH, H, W, seed=1, bf16_exact=True)
+    labels = si.labels(BATCH, seed=2)
+    net = pkg.Net(H, W, BATCH, pkg.VGG19_BF16, params=params, host_io=True, device=f"cuda:{local}")
+    x = torch.from_numpy(images).to(dev).to(torch.bfloat16)
+    y = torch.from_numpy(labels).to(dev)
+    logits = torch.empty(BATCH, 1000, dtype=torch.float32, device=dev)
+    grads = torch.empty(net.n_params, dtype=torch.float32, device=dev)
+    loss = torch.empty(1, dtype=torch.float32, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def timed(fn, steps, warmup):
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                fn()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            a.record(stream)
+            for _ in range(steps):
+                fn()
+            b.record(stream)
+        barrier()
+        return max_over_ranks(a.elapsed_time(b))
+
+    fwd = lambda: pkg.vgg19_forward(net.handle, x, BATCH, logits, None, stream)
+    bwd = lambda: pkg.vgg19_backward(net.handle, x, y, BATCH, grads, loss, None, stream)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    fwd_ms = timed(fwd, args.steps, args.warmup)
+    clocks = sampler.stop() if sampler else None
+    net.sync_status(stream)
+    bwd_steps = max(3, args.steps // 2)
+    bwd_ms = timed(bwd, bwd_steps, max(3, args.warmup))
+    net.sync_status(stream)
+
+    # end to end: pinned host images in, logits out, through the host-buffer entry point
+    x_host = torch.from_numpy(images).to(torch.bfloat16).pin_memory()
+    logits_host = torch.empty(BATCH, 1000, dtype=torch.float32).pin_memory()
+    for _ in range(max(3, args.warmup)):
+        pkg.vgg19_forward_host(net.handle, x_host, BATCH, logits_host, None, stream)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        pkg.vgg19_forward_host(net.handle, x_host, BATCH, logits_host, None, stream)
+    e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0))
+    barrier()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    # roofline of the dominant kernel: the convolution layers after the first
+    with torch.cuda.stream(stream):
+        bwd()  # leaves the batch-100 activations of every layer in the workspace
+    stream.synchronize()
+    layers = time_conv_layers(pkg, net, torch, stream)
+    conv_ms = sum(ms for _, ms, _, _ in layers)
+    conv_flop = sum(f for _, _, f, _ in layers)
+    achieved = conv_flop / (conv_ms * 1e-3) / 1e12
+    peak = pk["bf16_tflops"]
+    per_layer = {f"conv{l}": {"ms": round(ms, 4), "tflops": round(f / (ms * 1e-3) / 1e12, 1), "path": path}
+                 for l, ms, f, path in layers}
+
+    n_fwd = pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_FORWARD)
+    cpu_rate, cpu_dt = oracle_forward_rate(args.cpu_images)
+    value = world * BATCH * args.steps / (fwd_ms * 1e-3)
+    fwd_tflops = value * FWD_FLOP_PER_IMAGE / 1e12 / world
+    out = {
+        "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": fwd_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "image": [H, W, 3],
+                   "l2": "no explicit flush: each step writes and re-reads 3.4 GB of activations, 27x the 126 MB L2",
+                   "weights": "He-normal seed 0, biases 0", "graph": "one CUDA graph per pass"},
+        "clocks": clocks,
+        "e2e": {"value": world * BATCH * args.steps / (e2e_ms * 1e-3), "unit": "images/s",
+                "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": logits_host.numel() * 4,
+                "api": "vgg19_forward_host"},
+        "gpu_launches": n_fwd * args.steps,
+        "fwd_tflops_per_gpu": fwd_tflops,
+        "fwd_frac_of_bf16_peak": fwd_tflops / peak,
+        "fwd_bwd": {"value": world * BATCH * bwd_steps / (bwd_ms * 1e-3), "unit": "images/s", "steps": bwd_steps,
+                    "ms_per_step": bwd_ms / bwd_steps,
+                    "launches_per_step": pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_BACKWARD)},
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "traffic": None,
+                     "kernel": "3x3 convolution forward (implicit GEMM), layers 2..16, flop-weighted",
+                     "peak_source": f"{pk['source']} burst bf16 GEMM (kernel timed alone per layer)",
+                     "per_layer": per_layer},
+        "cpu_baseline": {"value": cpu_rate, "unit": "images/s", "cores": os.cpu_count(), "kind": "oracle",
+                         "sample": f"forward of {args.cpu_images} of the 100 images, {cpu_dt:.1f} s"},
+        "context": {"paper_tpuv2_core_s_per_batch100": 0.23, "paper_xeon_4114_flux_cpu_s_per_batch100": 52.4},
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--cpu-images", type=int, default=8, help="images the CPU checker is timed on")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_native(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,14 +1,343 @@
+// Tensor-core 3x3 convolution for sm_100a: an implicit GEMM on tcgen05 with the
+// accumulator in tensor memory, fed by TMA.
+//
+//   D[pixel][cout] = sum over (r, s, c) of  X[pixel shifted by (r-1, s-1)][c] * Wt[cout][r][s][c]
+//
+// GEMM view: M = N*H*W output pixels, N = Cout, K = 9*Cin walked as nine filter
+// taps times Cin/64 channel blocks.  One CTA computes a 128 (pixels) x BN
+// (output channels) tile:
+//   warp 0  : TMA producer.  Per K block it issues one im2col load (128 pixels
+//             x 64 channels of the NHWC input at tap (r, s); zero padding comes
+//             from the hardware's out-of-bounds fill) and one tiled load of the
+//             BN x 64 filter slice, into a ring of shared-memory stages.
+//   warp 1  : allocates tensor memory; one thread issues tcgen05.mma
+//             (128 x BN x 16 per instruction, four per K block) and commits each
+//             stage back to the producer and each finished tile to the epilogue.
+//   warps 2-5: epilogue.  Each thread owns one pixel row of the tile: it reads
+//             the fp32 accumulator from tensor memory 32 columns at a time, adds
+//             the bias, applies ReLU and/or the ReLU mask of the layer below,
+//             rounds to bf16 and stores to the NHWC output.
+// The accumulator is double buffered (2 x BN columns of tensor memory) so the
+// epilogue of one tile overlaps the main loop of the next; CTAs are persistent
+// and walk the tile list with a fixed stride.  Every wait has a time limit.
 #include "tc_kernels.cuh"
+
+#include <mutex>
+
+#include "tc_common.cuh"
 
 namespace vgg {
 
-bool tc_conv3x3_supported(ConvShape) { return false; }
-cudaError_t tc_conv3x3(const bf16*, const bf16*, const float*, const bf16*, bf16*, ConvShape, bool,
-                       int*, cudaStream_t) { return cudaErrorNotSupported; }
+// ---- tensor-map plumbing ------------------------------------------------------
+
+const TensorMapApi& tensor_map_api() {
+  static TensorMapApi api;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return;
+    api.encode_tiled = reinterpret_cast<decltype(api.encode_tiled)>(fn);
+    fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return;
+    api.encode_im2col = reinterpret_cast<decltype(api.encode_im2col)>(fn);
+    api.ok = true;
+  });
+  return api;
+}
+
+bool make_tiled_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  const TensorMapApi& api = tensor_map_api();
+  if (!api.ok) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return api.encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_im2col_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, uint32_t pixels) {
+  const TensorMapApi& api = tensor_map_api();
+  if (!api.ok) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+  cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+  // 3x3 window, padding 1: the window's first tap sits one pixel up/left of the
+  // output pixel, and the last tap (first + 2) must still be allowed to reach
+  // one pixel past the far edge.
+  int lower[2] = {-1, -1};
+  int upper[2] = {-1, -1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return api.encode_im2col(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, lower,
+                           upper, 64, pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128;             // pixels per tile (TMEM lanes)
+constexpr int BK = 64;              // channels per K block (one 128-byte swizzle row)
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int kThreads = 192;
+constexpr int kSmemLimit = 227 * 1024;
+
+template <int BN>
+struct ConvTile {
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = (kSmemLimit - 2048) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 2048) / STAGE_BYTES;
+  static constexpr int TMEM_COLS = 2 * BN;  // 128, 256 or 512: powers of two
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct ConvArgs {
+  int pixels;     // N*H*W
+  int H, W;
+  int cin_blocks; // Cin / 64
+  int Cout;
+  int m_tiles, n_tiles;
+  int relu;
+  const float* bias;
+  const bf16* mask;
+  bf16* out;
+  int* dev_error;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, ConvArgs a) {
+  using T = ConvTile<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = smem_base + T::STAGES * T::STAGE_BYTES;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (T::STAGES + s); };
+  auto acc_full_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + b); };
+  auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + 2 + b); };
+  const uint32_t drain_bar = bars + 8u * (2 * T::STAGES + 4);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k_blocks = 9 * a.cin_blocks;
+  const int total_tiles = a.m_tiles * a.n_tiles;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < T::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 128); }
+    mbar_init(drain_bar, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&map_x);
+    tma_prefetch_desc(&map_w);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), T::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      uint32_t fills[T::STAGES];
+#pragma unroll
+      for (int s = 0; s < T::STAGES; ++s) fills[s] = 0;
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
+        const int p0 = m_tile * BM;
+        const int w0 = p0 % a.W, t = p0 / a.W;
+        const int h0 = t % a.H, n0 = t / a.H;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          const int rs = kb / a.cin_blocks, cb = kb - rs * a.cin_blocks;
+          const int r = rs / 3, s = rs - r * 3;
+          if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
+          const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
+          mbar_expect_tx(full_bar(stage), T::STAGE_BYTES);
+          tma_load_im2col_4d(sa, &map_x, full_bar(stage), cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
+          tma_load_2d(sb, &map_w, full_bar(stage), kb * BK, n_tile * BN);
+          ++fills[stage];
+          if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        // let every copy already in flight land before the CTA may exit
+        for (int s = 0; s < T::STAGES; ++s)
+          if (fills[s]) {
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(full_bar(s), (fills[s] - 1) & 1) && global_timer_ns() - t0 < 100000000ull) {}
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+        const int buf = local & 1;
+        const uint32_t use = (uint32_t)(local >> 1);  // how many times this buffer was used before
+        if (!mbar_wait(acc_empty_bar(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = smem_desc_sw128(sa + k * 32, 16);
+            const uint64_t db = smem_desc_sw128(sb + k * 32, 16);
+            umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(acc_full_bar(buf));
+      }
+      if (!ok) {
+        // wait for the MMAs already issued before shared and tensor memory go away
+        umma_commit(drain_bar);
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else {
+    // -------------------------------- epilogue --------------------------------
+    const int quarter = warp & 3;  // the TMEM lane quarter this warp may read
+    const int row = quarter * 32 + lane;
+    int local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+      const int buf = local & 1;
+      const uint32_t use = (uint32_t)(local >> 1);
+      const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
+      if (!mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum)) { ok = false; break; }
+      tc_fence_after();
+      const long pixel = (long)m_tile * BM + row;
+      const bool valid = pixel < a.pixels;
+      const int c_base = n_tile * BN;
+      bf16* out_row = a.out + pixel * a.Cout + c_base;
+      const bf16* mask_row = a.mask ? a.mask + pixel * a.Cout + c_base : nullptr;
+#pragma unroll 1
+      for (int cc = 0; cc < BN; cc += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+        tmem_ld_wait();
+        if (valid) {
+          uint32_t packed[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
+            if (a.bias) { x0 += __ldg(a.bias + c_base + cc + j); x1 += __ldg(a.bias + c_base + cc + j + 1); }
+            if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
+            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+            packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          if (mask_row) {
+            const uint4* mp = reinterpret_cast<const uint4*>(mask_row + cc);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 m = __ldg(mp + q);
+              const uint32_t mw[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                // a bf16 is > 0 iff its sign bit is clear and it is not zero
+                const uint32_t lo = mw[e] & 0xFFFFu, hi = mw[e] >> 16;
+                uint32_t keep = 0;
+                if (lo != 0 && !(lo & 0x8000u)) keep |= 0x0000FFFFu;
+                if (hi != 0 && !(hi & 0x8000u)) keep |= 0xFFFF0000u;
+                packed[q * 4 + e] &= keep;
+              }
+            }
+          }
+          uint4* op = reinterpret_cast<uint4*>(out_row + cc);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty_bar(buf));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, T::TMEM_COLS);
+  }
+}
+
+template <int BN>
+cudaError_t launch_conv(const CUtensorMap& mx, const CUtensorMap& mw, ConvArgs a, cudaStream_t st) {
+  using T = ConvTile<BN>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int tiles = a.m_tiles * a.n_tiles;
+  const int grid = tiles < sms ? tiles : sms;
+  conv3x3_tc_kernel<BN><<<grid, kThreads, T::SMEM_BYTES, st>>>(mx, mw, a);
+  return cudaGetLastError();
+}
+
+int pick_bn(int Cout) { return Cout % 256 == 0 ? 256 : (Cout % 128 == 0 ? 128 : 64); }
+
+}  // namespace
+
+bool tc_conv3x3_supported(ConvShape s) {
+  return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.H >= 2 && s.W >= 2 && s.N >= 1 &&
+         (long)s.N * s.H * s.W < (1L << 31) - 256;
+}
+
+cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out, ConvShape s,
+                       bool relu, int* dev_error, cudaStream_t st) {
+  if (!tc_conv3x3_supported(s)) return cudaErrorInvalidValue;
+  const int BN = pick_bn(s.Cout);
+  CUtensorMap mx, mw;
+  if (!make_im2col_map(&mx, in, s.N, s.H, s.W, s.Cin, BM)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
+  ConvArgs a;
+  a.pixels = s.N * s.H * s.W;
+  a.H = s.H; a.W = s.W;
+  a.cin_blocks = s.Cin / 64;
+  a.Cout = s.Cout;
+  a.m_tiles = (a.pixels + BM - 1) / BM;
+  a.n_tiles = s.Cout / BN;
+  a.relu = relu ? 1 : 0;
+  a.bias = bias; a.mask = mask; a.out = out; a.dev_error = dev_error;
+  switch (BN) {
+    case 256: return launch_conv<256>(mx, mw, a, st);
+    case 128: return launch_conv<128>(mx, mw, a, st);
+    default: return launch_conv<64>(mx, mw, a, st);
+  }
+}
+
 bool tc_wgrad_supported(ConvShape) { return false; }
 size_t tc_wgrad_scratch_elems(ConvShape) { return 0; }
 int tc_wgrad_launches(ConvShape) { return 0; }
-cudaError_t tc_conv3x3_wgrad(const bf16*, const bf16*, float*, float*, float*, ConvShape, int*,
-                             cudaStream_t) { return cudaErrorNotSupported; }
+cudaError_t tc_conv3x3_wgrad(const bf16*, const bf16*, float*, float*, float*, ConvShape, int*, cudaStream_t) {
+  return cudaErrorNotSupported;
+}
 
 }  // namespace vgg
