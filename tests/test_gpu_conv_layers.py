@@ -1,0 +1,91 @@
+"""Per-layer parity of the convolution kernels (forward, input gradient, filter
+and bias gradient) at the layer shapes of the 224x224 network, on a small
+batch, against the fp64 CPU checker fed the same bf16-exact tensors.
+
+Tolerance: the device accumulates in fp32 and stores bf16.  Against the
+checker's result rounded to bf16 the only differences are rare one-ulp
+rounding flips (relative L2 ~1e-4): bar 1e-3.  fp32 gradient outputs are not
+rounded: bar 1e-3 as well (sums of up to ~10^5 bf16 products in fp32).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import seeded_inputs as si
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+# (layer, H=W at a 224x224 input, Cin, Cout): the nine distinct shapes
+SHAPES = [(1, 224, 3, 64), (2, 224, 64, 64), (3, 112, 64, 128), (4, 112, 128, 128), (5, 56, 128, 256),
+          (6, 56, 256, 256), (9, 28, 256, 512), (10, 28, 512, 512), (13, 14, 512, 512)]
+
+
+def rel_l2(a, b):
+    a, b = np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+@pytest.fixture(scope="module")
+def net224():
+    import paper_1810_09868_b200 as p
+    params = si.vgg19_params(224, 224, seed=0, bias_std=0.1, bf16_exact=True)
+    net = p.Net(224, 224, 3, p.VGG19_BF16, params=params)
+    yield p, net, params
+    net.close()
+
+
+def layer_params(p, net, params, layer):
+    (woff, wdims), (boff, bdims) = p.vgg19_param_info(net.handle, 2 * (layer - 1)), p.vgg19_param_info(net.handle, 2 * layer - 1)
+    Wt = params[woff:woff + int(np.prod(wdims))].reshape(wdims).astype(np.float64)
+    b = params[boff:boff + int(np.prod(bdims))].astype(np.float64)
+    return Wt, b
+
+
+def layer_input(layer, B, S, Cin):
+    if Cin == 3:
+        return si.images(B, S, S, seed=1, bf16_exact=True)
+    return si.normal(B * S * S * Cin, seed=100 + layer, take_abs=True, bf16_exact=True).reshape(B, S, S, Cin)
+
+
+@pytest.mark.parametrize("layer,S,Cin,Cout", SHAPES)
+def test_conv_layer_forward(net224, layer, S, Cin, Cout):
+    p, net, params = net224
+    B = 3 if S <= 28 else 1  # 14x14x3 = 588 pixels: a ragged last tile
+    x = layer_input(layer, B, S, Cin)
+    Wt, b = layer_params(p, net, params, layer)
+    xd = torch.from_numpy(x).to(DEV).to(torch.bfloat16)
+    y = torch.full((B, S, S, Cout), float("nan"), dtype=torch.bfloat16, device=DEV)
+    pooled = torch.full((B, S // 2, S // 2, Cout), float("nan"), dtype=torch.bfloat16, device=DEV)
+    p.vgg19_conv_layer_forward(net.handle, layer, xd, B, y, pooled, torch.cuda.current_stream())
+    net.sync_status()
+    ref = oracle.round_bf16(oracle.relu_fwd(oracle.conv3x3_fwd(x, Wt, b)))
+    got = y.float().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert rel_l2(got, ref) <= 1e-3
+    assert np.array_equal(pooled.float().cpu().numpy(), oracle.maxpool2x2_fwd(got))
+
+
+@pytest.mark.parametrize("layer,S,Cin,Cout", SHAPES)
+def test_conv_layer_backward(net224, layer, S, Cin, Cout):
+    p, net, params = net224
+    B = 3 if S <= 28 else 1
+    x = layer_input(layer, B, S, Cin)
+    # a ReLU-masked upstream gradient: about half the entries are exactly zero
+    dz = si.normal(B * S * S * Cout, seed=200 + layer, stddev=1e-3, bf16_exact=True).reshape(B, S, S, Cout)
+    dz = dz * (si.uniform(dz.size, seed=300 + layer).reshape(dz.shape) < 0.5)
+    Wt, _ = layer_params(p, net, params, layer)
+    xd = torch.from_numpy(x).to(DEV).to(torch.bfloat16)
+    dzd = torch.from_numpy(dz).to(DEV).to(torch.bfloat16)
+    dw = torch.full((Cout, 3, 3, Cin), float("nan"), dtype=torch.float32, device=DEV)
+    db = torch.full((Cout,), float("nan"), dtype=torch.float32, device=DEV)
+    dx = None if layer == 1 else torch.full((B, S, S, Cin), float("nan"), dtype=torch.bfloat16, device=DEV)
+    p.vgg19_conv_layer_backward(net.handle, layer, xd, dzd, B, dw, db, dx, torch.cuda.current_stream())
+    net.sync_status()
+    o_dw, o_db = oracle.conv3x3_wgrad(x, dz)
+    assert rel_l2(dw.cpu().numpy(), o_dw) <= 1e-3
+    assert rel_l2(db.cpu().numpy(), o_db) <= 1e-3
+    if dx is not None:
+        ref = oracle.round_bf16(oracle.conv3x3_dgrad(dz, Wt))
+        assert rel_l2(dx.float().cpu().numpy(), ref) <= 1e-3
