@@ -155,6 +155,42 @@ int vgg19_conv_layer_backward(vgg19_t *net, int32_t layer, const void *x, const 
 int vgg19_saved_tensor(const vgg19_t *net, int32_t batch, int32_t mode, int32_t index,
                        size_t *offset_bytes, int64_t dims[4]);
 
+/* Filter and bias gradient of one 3x3 / pad 1 / stride 1 convolution without
+ * any allocation.  (The paper has no counterpart: this entry point exists for
+ * the library's users, not for the method.)
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained -
+ * a plugin or callback invoked inside someone else's framework after that
+ * framework has claimed the whole GPU for its own pool, or a process whose
+ * memory budget was fixed at start-up - cannot create a network handle or
+ * provide a workspace, because both need cudaMalloc.  This function needs
+ * neither: it takes no handle, and the split-K scratch its kernel uses is a
+ * fixed array of VGG19_STATIC_SCRATCH_BYTES compiled into the library (every
+ * GPU that loads the library carries that array until the process exits).  It
+ * calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   x  : device, [batch][height][width][cin]   layer input
+ *   dz : device, [batch][height][width][cout]  gradient at the pre-activation
+ *   dtype : VGG19_FP32 or VGG19_BF16, the element type of x and dz
+ *   dw : device fp32 [cout][3][3][cin], db : device fp32 [cout]; overwritten
+ *   needed_bytes : if not NULL, receives the scratch this shape needs
+ * Same arithmetic as the CUDA-core path of vgg19_conv_layer_backward.
+ *
+ * Returns VGG19_ERR_WORKSPACE, and launches nothing, when the shape needs more
+ * scratch than VGG19_STATIC_SCRATCH_BYTES (*needed_bytes says how much);
+ * VGG19_ERR_ARG for null pointers or non-positive sizes.
+ *
+ * The first call on each device looks up the array's device address (that
+ * device must be current); make that first call outside any stream capture.
+ * All calls share the one array and it keeps whatever the last call left in
+ * it; the kernels never rely on its previous contents.  Two calls that overlap
+ * on the GPU (different streams) race on it: keep calls on one stream, or
+ * order them with events. */
+#define VGG19_STATIC_SCRATCH_BYTES (8u << 20)
+int vgg19_conv_wgrad_static(const void *x, const void *dz, int32_t batch, int32_t height, int32_t width,
+                            int32_t cin, int32_t cout, int32_t dtype, float *dw, float *db,
+                            size_t *needed_bytes, void *stream);
+
 /* Wait for the stream and report any device-side error recorded so far. */
 int vgg19_sync_status(vgg19_t *net, void *stream);
 

@@ -22,7 +22,7 @@ EXPORTS = (
     "vgg19_create", "vgg19_create_from_params", "vgg19_destroy", "vgg19_param_count", "vgg19_param_info",
     "vgg19_get_params", "vgg19_set_params", "vgg19_workspace_bytes", "vgg19_bind_workspace",
     "vgg19_forward", "vgg19_backward", "vgg19_io_bytes", "vgg19_forward_host", "vgg19_backward_host",
-    "vgg19_conv_layer_forward", "vgg19_conv_layer_backward", "vgg19_saved_tensor", "vgg19_sync_status", "vgg19_launch_count",
+    "vgg19_conv_layer_forward", "vgg19_conv_layer_backward", "vgg19_saved_tensor", "vgg19_conv_wgrad_static", "vgg19_sync_status", "vgg19_launch_count",
     "vgg19_describe", "vgg19_last_error",
 )
 
@@ -75,6 +75,7 @@ def load():
         "vgg19_conv_layer_forward": ([vp, i32, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_backward": ([vp, i32, vp, vp, i32, vp, vp, vp, vp], ctypes.c_int),
         "vgg19_saved_tensor": ([vp, i32, i32, i32, ctypes.POINTER(sz), ctypes.POINTER(ctypes.c_int64)], ctypes.c_int),
+        "vgg19_conv_wgrad_static": ([vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, ctypes.POINTER(sz), vp], ctypes.c_int),
         "vgg19_sync_status": ([vp, vp], ctypes.c_int),
         "vgg19_launch_count": ([vp, i32, ctypes.POINTER(i32)], ctypes.c_int),
         "vgg19_describe": ([vp, ctypes.c_char_p, sz], ctypes.c_int),
@@ -198,6 +199,17 @@ def vgg19_saved_tensor(net, batch, mode, index):
     dims = (ctypes.c_int64 * 4)()
     _check(net, load().vgg19_saved_tensor(net, batch, mode, index, ctypes.byref(off), dims))
     return off.value, tuple(dims)
+
+
+VGG19_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def vgg19_conv_wgrad_static(x, dz, batch, height, width, cin, cout, dtype, dw, db, stream=None):
+    """Allocation-free filter/bias gradient; returns (status, scratch bytes the shape needs)."""
+    need = ctypes.c_size_t()
+    rc = load().vgg19_conv_wgrad_static(_ptr(x), _ptr(dz), batch, height, width, cin, cout, dtype, _ptr(dw), _ptr(db),
+                                        ctypes.byref(need), _stream(stream))
+    return rc, need.value
 
 
 def vgg19_sync_status(net, stream=None):
