@@ -48,6 +48,13 @@ template <typename T>
 cudaError_t simt_conv3x3_wgrad(const T* x, const T* dz, float* dW, float* db, float* partial,
                                ConvShape s, cudaStream_t st);
 
+// db[c] = sum_p dz[p][c]; partial: fp32 scratch of at least 256 * C elements.
+template <typename T>
+cudaError_t simt_bias_grad(const T* dz, float* db, float* partial, long P, int C, cudaStream_t st);
+// db[o] = sum_m dY[m][o]
+template <typename T>
+cudaError_t simt_dense_db(const T* dY, float* db, int M, int Out, cudaStream_t st);
+
 // y = max over 2x2 windows (stride 2) of x, NHWC.
 template <typename T>
 cudaError_t simt_maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st);

@@ -235,6 +235,16 @@ cudaError_t simt_conv3x3_wgrad(const T* x, const T* dz, float* dW, float* db, fl
   return cudaGetLastError();
 }
 
+template <typename T>
+cudaError_t simt_bias_grad(const T* dz, float* db, float* partial, long P, int C, cudaStream_t st) {
+  int chunks = colsum_chunks(P);
+  long per = (P + chunks - 1) / chunks;
+  dim3 grid((C + 31) / 32, chunks), block(32, 8);
+  colsum_partial_kernel<T><<<grid, block, 0, st>>>(dz, partial, P, C, per);
+  reduce_splits_kernel<<<(C + 255) / 256, 256, 0, st>>>(partial, db, C, chunks);
+  return cudaGetLastError();
+}
+
 // ---- pooling ---------------------------------------------------------------
 
 template <typename T>
@@ -316,6 +326,12 @@ __global__ void dense_db_kernel(const T* dY, float* db, int M, int Out) {
   float s = 0.f;
   for (int m = 0; m < M; ++m) s += to_f32(dY[(long)m * Out + o]);
   db[o] = s;
+}
+
+template <typename T>
+cudaError_t simt_dense_db(const T* dY, float* db, int M, int Out, cudaStream_t st) {
+  dense_db_kernel<T><<<(Out + 127) / 128, 128, 0, st>>>(dY, db, M, Out);
+  return cudaGetLastError();
 }
 
 template <typename T>
@@ -431,6 +447,8 @@ cudaError_t make_dgrad_filter(const float* w, T* wt_t, int Cin, int Cout, cudaSt
                                         cudaStream_t);                                               \
   template cudaError_t simt_dense_dw<T>(const T*, const T*, float*, float*, int, int, int,           \
                                         cudaStream_t);                                               \
+  template cudaError_t simt_bias_grad<T>(const T*, float*, float*, long, int, cudaStream_t);           \
+  template cudaError_t simt_dense_db<T>(const T*, float*, int, int, cudaStream_t);                    \
   template cudaError_t softmax_xent<T>(const float*, const int32_t*, float*, T*, float*, float*,     \
                                        int, int, cudaStream_t);                                      \
   template cudaError_t convert_f32<T>(const float*, T*, size_t, cudaStream_t);                       \

@@ -1,0 +1,452 @@
+// Tensor-core GEMM for sm_100a (tcgen05 + TMEM + TMA) behind the dense layers
+// and the convolution filter gradient:
+//
+//   D[m][n] = sum_k A(m, k) * B(n, k),   bf16 operands, fp32 accumulation.
+//
+// Each operand can sit in memory either K-major (a row per m / n, k contiguous:
+// activations [batch][features], weights [out][in]) or MN-major (a row per k,
+// m / n contiguous: the same matrices used transposed, as the backward pass
+// does).  A third form of B reads an NHWC activation through a 3x3 window
+// (TMA im2col) with the pixel index as k: that is the filter gradient
+//   dW[cout][tap][c] = sum_pixels dz[pixel][cout] * x[pixel shifted by tap][c].
+//
+// One CTA computes one 128 x BN tile over its share of K (grid.y splits K):
+//   warp 0 TMA producer, warp 1 TMEM owner + single-thread MMA issuer, warps
+//   2-5 epilogue (one tile row per thread, straight from tensor memory).
+// With K split, tiles write raw fp32 partial sums and a second kernel adds the
+// splits in a fixed order and applies bias / ReLU / mask (deterministic).
+// All waits are time-limited (see tc_common.cuh).
+#include "tc_common.cuh"
+#include "tc_kernels.cuh"
+
+namespace vgg {
+namespace {
+
+using namespace tc;
+
+enum OperandMode { kKMajor = 0, kMnMajor = 1, kMnMajorIm2col = 2 };
+
+constexpr int BM = 128, BK = 64;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int GROUP_BYTES = 64 * BK * 2;  // one 64 x 64 box of an MN-major operand
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+
+struct GemmArgs {
+  int M, N;          // valid rows and columns of D
+  int k_blocks;      // ceil(K / 64)
+  int kb_per_split;
+  int n_tiles;
+  int stages;
+  int H, W, Cin;     // im2col form of B: column j of D is (tap = j / Cin, channel = j % Cin)
+  float* partial;    // split-K: raw sums at partial[(split * M + m) * N + n]; else null
+  float* out_f;      // direct epilogue outputs (either may be null), row stride ldc
+  bf16* out_h;
+  long ldc;
+  const float* bias; // per column, or null
+  const bf16* mask;  // same shape as the output, or null: keep where mask > 0
+  int relu;
+  int* dev_error;
+};
+
+template <int BN>
+__host__ __device__ constexpr int stage_bytes() { return A_BYTES + BN * BK * 2; }
+
+template <int BN, int AMODE, int BMODE>
+__global__ void __launch_bounds__(kThreads)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs g) {
+  constexpr int STAGE = stage_bytes<BN>();
+  constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = smem_base + g.stages * STAGE;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+  const uint32_t acc_bar = bars + 8u * (2 * kMaxStages);
+  const uint32_t drain_bar = bars + 8u * (2 * kMaxStages + 1);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tile = blockIdx.x / g.n_tiles, n_tile = blockIdx.x - m_tile * g.n_tiles;
+  const int m0 = m_tile * BM, n0 = n_tile * BN;
+  const int kb0 = blockIdx.y * g.kb_per_split;
+  const int kb1 = min(g.k_blocks, kb0 + g.kb_per_split);
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(acc_bar, 1);
+    mbar_init(drain_bar, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&map_a);
+    tma_prefetch_desc(&map_b);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t fills[kMaxStages];
+#pragma unroll
+      for (int s = 0; s < kMaxStages; ++s) fills[s] = 0;
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      int tap_s = 0, tap_r = 0, c0 = 0;
+      if (BMODE == kMnMajorIm2col) {
+        const int tap = n0 / g.Cin;
+        c0 = n0 - tap * g.Cin;
+        tap_r = tap / 3;
+        tap_s = tap - tap_r * 3;
+      }
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, g.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
+        const uint32_t sa = smem_base + stage * STAGE, sb = sa + A_BYTES;
+        mbar_expect_tx(full_bar(stage), STAGE);
+        if (AMODE == kKMajor) {
+          tma_load_2d(sa, &map_a, full_bar(stage), kb * BK, m0);
+        } else {
+          tma_load_2d(sa, &map_a, full_bar(stage), m0, kb * BK);
+          tma_load_2d(sa + GROUP_BYTES, &map_a, full_bar(stage), m0 + 64, kb * BK);
+        }
+        if (BMODE == kKMajor) {
+          tma_load_2d(sb, &map_b, full_bar(stage), kb * BK, n0);
+        } else if (BMODE == kMnMajor) {
+#pragma unroll
+          for (int q = 0; q < BN / 64; ++q) tma_load_2d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), n0 + 64 * q, kb * BK);
+        } else {
+          const int p0 = kb * BK;
+          const int w0 = p0 % g.W, t = p0 / g.W;
+          const int h0 = t % g.H, img = t / g.H;
+#pragma unroll
+          for (int q = 0; q < BN / 64; ++q)
+            tma_load_im2col_4d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), c0 + 64 * q, w0 - 1, h0 - 1, img,
+                               (uint16_t)tap_s, (uint16_t)tap_r);
+        }
+        ++fills[stage];
+        if (++stage == g.stages) { stage = 0; phase ^= 1; }
+      }
+      if (!ok) {
+        for (int s = 0; s < g.stages; ++s)
+          if (fills[s]) {
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(full_bar(s), (fills[s] - 1) & 1) && global_timer_ns() - t0 < 100000000ull) {}
+          }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, AMODE != kKMajor, BMODE != kKMajor);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(full_bar(stage), phase, &abort_flag, g.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_base + stage * STAGE, sb = sa + A_BYTES;
+#pragma unroll
+        for (int k = 0; k < BK / 16; ++k) {
+          // K-major: 16 k = 32 bytes along the swizzled row.  MN-major: 16 k = 16 rows = 2048 bytes.
+          const uint64_t da = AMODE == kKMajor ? smem_desc_sw128(sa + k * 32, 16) : smem_desc_sw128(sa + k * 2048, GROUP_BYTES);
+          const uint64_t db = BMODE == kKMajor ? smem_desc_sw128(sb + k * 32, 16) : smem_desc_sw128(sb + k * 2048, GROUP_BYTES);
+          umma_bf16(tmem_base, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(empty_bar(stage));
+        if (++stage == g.stages) { stage = 0; phase ^= 1; }
+      }
+      if (ok) {
+        umma_commit(acc_bar);
+      } else {
+        umma_commit(drain_bar);
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int m = m0 + quarter * 32 + lane;
+    const bool row_ok = m < g.M;
+    if (mbar_wait(acc_bar, 0, &abort_flag, g.dev_error, kDevTimeoutAccum)) {
+      tc_fence_after();
+#pragma unroll 1
+      for (int cc = 0; cc < BN; cc += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)cc, v);
+        tmem_ld_wait();
+        const int n = n0 + cc;
+        if (!row_ok || n >= g.N) continue;
+        if (g.partial) {
+          float* dst = g.partial + ((long)blockIdx.y * g.M + m) * g.N + n;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            if (n + j < g.N)
+              *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+        } else {
+          const long o = (long)m * g.ldc + n;
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            if (n + j >= g.N) break;
+            float x[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              x[e] = __uint_as_float(v[j + e]);
+              if (g.bias) x[e] += __ldg(g.bias + n + j + e);
+              if (g.relu) x[e] = fmaxf(x[e], 0.f);
+            }
+            if (g.mask) {
+              const uint4 mk = __ldg(reinterpret_cast<const uint4*>(g.mask + o + j));
+              const uint32_t mw[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t lo = mw[e] & 0xFFFFu, hi = mw[e] >> 16;
+                if (lo == 0 || (lo & 0x8000u)) x[2 * e] = 0.f;
+                if (hi == 0 || (hi & 0x8000u)) x[2 * e + 1] = 0.f;
+              }
+            }
+            if (g.out_f) {
+              *reinterpret_cast<float4*>(g.out_f + o + j) = make_float4(x[0], x[1], x[2], x[3]);
+              *reinterpret_cast<float4*>(g.out_f + o + j + 4) = make_float4(x[4], x[5], x[6], x[7]);
+            }
+            if (g.out_h) {
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(x[0], x[1]), h1 = __floats2bfloat162_rn(x[2], x[3]);
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(x[4], x[5]), h3 = __floats2bfloat162_rn(x[6], x[7]);
+              *reinterpret_cast<uint4*>(g.out_h + o + j) =
+                  make_uint4(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1),
+                             *reinterpret_cast<uint32_t*>(&h2), *reinterpret_cast<uint32_t*>(&h3));
+            }
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// out = epilogue(sum over splits of partial[split]), four columns per thread
+__global__ void splitk_finish_kernel(const float* __restrict__ partial, int splits, long MN, int N,
+                                     const float* __restrict__ bias, int relu, const bf16* __restrict__ mask,
+                                     bf16* out_h, float* out_f) {
+  const long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= MN) return;
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int z = 0; z < splits; ++z) {
+    const float4 p = *reinterpret_cast<const float4*>(partial + (long)z * MN + i);
+    s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+  }
+  float x[4] = {s.x, s.y, s.z, s.w};
+  const int n = (int)(i % N);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    if (bias) x[e] += bias[n + e];
+    if (relu) x[e] = fmaxf(x[e], 0.f);
+    if (mask && !(__bfloat162float(mask[i + e]) > 0.f)) x[e] = 0.f;
+  }
+  if (out_f) *reinterpret_cast<float4*>(out_f + i) = make_float4(x[0], x[1], x[2], x[3]);
+  if (out_h) {
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(x[0], x[1]), h1 = __floats2bfloat162_rn(x[2], x[3]);
+    *reinterpret_cast<uint2*>(out_h + i) = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
+  }
+}
+
+int sm_count() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
+  }
+  return sms;
+}
+
+// K split: aim at about two CTAs per SM in total, never an empty split.
+void plan_split(int mn_tiles, int k_blocks, int* splits, int* kb_per_split) {
+  int want = (2 * sm_count() + mn_tiles - 1) / mn_tiles;
+  if (want < 1) want = 1;
+  if (want > k_blocks) want = k_blocks;
+  int per = (k_blocks + want - 1) / want;
+  *kb_per_split = per;
+  *splits = (k_blocks + per - 1) / per;
+}
+
+template <int BN, int AMODE, int BMODE>
+cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArgs g, int m_tiles, int splits,
+                           cudaStream_t st) {
+  constexpr int STAGE = stage_bytes<BN>();
+  constexpr int max_stages = (227 * 1024 - 2048) / STAGE > kMaxStages ? kMaxStages : (227 * 1024 - 2048) / STAGE;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, AMODE, BMODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         max_stages * STAGE + 1024 + 256);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  g.stages = g.kb_per_split < max_stages ? g.kb_per_split : max_stages;
+  const size_t smem = (size_t)g.stages * STAGE + 1024 + 256;
+  dim3 grid(m_tiles * g.n_tiles, splits);
+  gemm_tc_kernel<BN, AMODE, BMODE><<<grid, kThreads, smem, st>>>(ma, mb, g);
+  return cudaGetLastError();
+}
+
+cudaError_t finish(const GemmArgs& g, int splits, const float* bias, bool relu, const bf16* mask, bf16* out_h,
+                   float* out_f, cudaStream_t st) {
+  const long MN = (long)g.M * g.N;
+  splitk_finish_kernel<<<(unsigned)((MN / 4 + 255) / 256), 256, 0, st>>>(g.partial, splits, MN, g.N, bias, relu ? 1 : 0,
+                                                                          mask, out_h, out_f);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// ---- dense layers ------------------------------------------------------------
+
+bool tc_dense_supported(int M, int In, int Out) {
+  return M >= 1 && In % 8 == 0 && Out % 8 == 0 && In >= 64 && Out >= 64;
+}
+
+size_t tc_dense_scratch_elems(int M, int In, int Out) {
+  // forward and input-gradient both split K; bound both
+  size_t worst = 0;
+  const int shapes[2][2] = {{Out, In}, {In, Out}};  // {N, K}
+  for (auto& s : shapes) {
+    int splits, per;
+    plan_split(((M + BM - 1) / BM) * ((s[0] + 127) / 128), (s[1] + BK - 1) / BK, &splits, &per);
+    size_t e = (size_t)splits * M * s[0];
+    if (e > worst) worst = e;
+  }
+  return worst;
+}
+
+// Y = [relu](X W^T + b): X [M][In], W [Out][In]
+cudaError_t tc_dense_forward(const bf16* X, const bf16* Wt, const float* bias, bf16* out_h, float* out_f,
+                             float* partial, int M, int In, int Out, bool relu, int* dev_error, cudaStream_t st) {
+  CUtensorMap ma, mb;
+  if (!make_tiled_map_2d(&ma, X, (uint64_t)M, (uint64_t)In, BM)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d(&mb, Wt, (uint64_t)Out, (uint64_t)In, 128)) return cudaErrorInvalidValue;
+  GemmArgs g{};
+  g.M = M; g.N = Out; g.k_blocks = (In + BK - 1) / BK; g.n_tiles = (Out + 127) / 128;
+  g.dev_error = dev_error; g.ldc = Out;
+  const int m_tiles = (M + BM - 1) / BM;
+  int splits;
+  plan_split(m_tiles * g.n_tiles, g.k_blocks, &splits, &g.kb_per_split);
+  if (splits == 1) {
+    g.bias = bias; g.relu = relu; g.out_h = out_h; g.out_f = out_f;
+    return launch_gemm_tc<128, kKMajor, kKMajor>(ma, mb, g, m_tiles, 1, st);
+  }
+  g.partial = partial;
+  cudaError_t e = launch_gemm_tc<128, kKMajor, kKMajor>(ma, mb, g, m_tiles, splits, st);
+  if (e != cudaSuccess) return e;
+  return finish(g, splits, bias, relu, nullptr, out_h, out_f, st);
+}
+
+// dX = (dY W) [* (mask > 0)]: dY [M][Out], W [Out][In]
+cudaError_t tc_dense_dx(const bf16* dY, const bf16* Wt, const bf16* mask, bf16* dX, float* partial, int M, int In,
+                        int Out, int* dev_error, cudaStream_t st) {
+  CUtensorMap ma, mb;
+  if (!make_tiled_map_2d(&ma, dY, (uint64_t)M, (uint64_t)Out, BM)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d(&mb, Wt, (uint64_t)Out, (uint64_t)In, 64)) return cudaErrorInvalidValue;
+  GemmArgs g{};
+  g.M = M; g.N = In; g.k_blocks = (Out + BK - 1) / BK; g.n_tiles = (In + 127) / 128;
+  g.dev_error = dev_error; g.ldc = In;
+  const int m_tiles = (M + BM - 1) / BM;
+  int splits;
+  plan_split(m_tiles * g.n_tiles, g.k_blocks, &splits, &g.kb_per_split);
+  if (splits == 1) {
+    g.mask = mask; g.out_h = dX;
+    return launch_gemm_tc<128, kKMajor, kMnMajor>(ma, mb, g, m_tiles, 1, st);
+  }
+  g.partial = partial;
+  cudaError_t e = launch_gemm_tc<128, kKMajor, kMnMajor>(ma, mb, g, m_tiles, splits, st);
+  if (e != cudaSuccess) return e;
+  return finish(g, splits, nullptr, false, mask, dX, nullptr, st);
+}
+
+// dW = dY^T X: dY [M][Out], X [M][In] -> dW fp32 [Out][In]
+cudaError_t tc_dense_dw(const bf16* dY, const bf16* X, float* dW, int M, int In, int Out, int* dev_error,
+                        cudaStream_t st) {
+  CUtensorMap ma, mb;
+  if (!make_tiled_map_2d(&ma, dY, (uint64_t)M, (uint64_t)Out, 64)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d(&mb, X, (uint64_t)M, (uint64_t)In, 64)) return cudaErrorInvalidValue;
+  GemmArgs g{};
+  g.M = Out; g.N = In; g.k_blocks = (M + BK - 1) / BK; g.kb_per_split = g.k_blocks;
+  g.dev_error = dev_error; g.ldc = In; g.out_f = dW;
+  const int m_tiles = (Out + BM - 1) / BM;
+  if (In % 256 == 0) {
+    g.n_tiles = In / 256;
+    return launch_gemm_tc<256, kMnMajor, kMnMajor>(ma, mb, g, m_tiles, 1, st);
+  }
+  g.n_tiles = (In + 127) / 128;
+  return launch_gemm_tc<128, kMnMajor, kMnMajor>(ma, mb, g, m_tiles, 1, st);
+}
+
+// ---- convolution filter gradient ----------------------------------------------
+
+namespace {
+int wgrad_bn(int Cin) { return Cin % 256 == 0 ? 256 : (Cin % 128 == 0 ? 128 : 64); }
+void wgrad_plan(ConvShape s, int* m_tiles, int* n_tiles, int* k_blocks, int* splits, int* per) {
+  const long P = (long)s.N * s.H * s.W;
+  *m_tiles = (s.Cout + BM - 1) / BM;
+  *n_tiles = 9 * s.Cin / wgrad_bn(s.Cin);
+  *k_blocks = (int)((P + BK - 1) / BK);
+  plan_split(*m_tiles * *n_tiles, *k_blocks, splits, per);
+}
+}  // namespace
+
+bool tc_wgrad_supported(ConvShape s) {
+  return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.H >= 2 && s.W >= 2 && (long)s.N * s.H * s.W < (1L << 31) - 256;
+}
+
+size_t tc_wgrad_scratch_elems(ConvShape s) {
+  if (!tc_wgrad_supported(s)) return 0;
+  int mt, nt, kb, splits, per;
+  wgrad_plan(s, &mt, &nt, &kb, &splits, &per);
+  return (size_t)splits * s.Cout * 9 * s.Cin;
+}
+
+int tc_wgrad_launches(ConvShape s) {
+  int mt, nt, kb, splits, per;
+  wgrad_plan(s, &mt, &nt, &kb, &splits, &per);
+  return splits > 1 ? 2 : 1;
+}
+
+// dW[k][tap][c] = sum_pixels dz[pixel][k] * x[pixel + tap][c]   (fp32 out, [Cout][9*Cin])
+cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* partial, ConvShape s, int* dev_error,
+                             cudaStream_t st) {
+  if (!tc_wgrad_supported(s)) return cudaErrorInvalidValue;
+  const long P = (long)s.N * s.H * s.W;
+  const int BN = wgrad_bn(s.Cin);
+  CUtensorMap ma, mb;
+  if (!make_tiled_map_2d(&ma, dz, (uint64_t)P, (uint64_t)s.Cout, 64)) return cudaErrorInvalidValue;
+  if (!make_im2col_map(&mb, x, s.N, s.H, s.W, s.Cin, 64)) return cudaErrorInvalidValue;
+  GemmArgs g{};
+  int m_tiles, splits;
+  wgrad_plan(s, &m_tiles, &g.n_tiles, &g.k_blocks, &splits, &g.kb_per_split);
+  g.M = s.Cout; g.N = 9 * s.Cin; g.H = s.H; g.W = s.W; g.Cin = s.Cin;
+  g.dev_error = dev_error; g.ldc = g.N;
+  if (splits == 1) g.out_f = dW; else g.partial = partial;
+  cudaError_t e;
+  switch (BN) {
+    case 256: e = launch_gemm_tc<256, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
+    case 128: e = launch_gemm_tc<128, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
+    default: e = launch_gemm_tc<64, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
+  }
+  if (e != cudaSuccess || splits == 1) return e;
+  return finish(g, splits, nullptr, false, nullptr, nullptr, dW, st);
+}
+
+}  // namespace vgg

@@ -17,12 +17,23 @@ bool tc_conv3x3_supported(ConvShape s);
 cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const bf16* mask,
                        bf16* out, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
 
-// Filter and bias gradient of the same convolution (M = Cout, N = 9*Cin,
-// K = pixels).
+// Filter gradient of the same convolution as a GEMM with M = Cout, N = 9*Cin,
+// K = pixels (both operands read transposed, x through the im2col window):
+// dW fp32 [Cout][3][3][Cin].  partial: fp32 scratch of tc_wgrad_scratch_elems().
 bool tc_wgrad_supported(ConvShape s);
 size_t tc_wgrad_scratch_elems(ConvShape s);
 int tc_wgrad_launches(ConvShape s);
-cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* db, float* partial,
-                             ConvShape s, int* dev_error, cudaStream_t st);
+cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* partial, ConvShape s, int* dev_error,
+                             cudaStream_t st);
+
+// Dense layers on the same GEMM kernel.  X [M][In], W [Out][In], dY [M][Out].
+bool tc_dense_supported(int M, int In, int Out);
+size_t tc_dense_scratch_elems(int M, int In, int Out);
+cudaError_t tc_dense_forward(const bf16* X, const bf16* W, const float* bias, bf16* out_h, float* out_f,
+                             float* partial, int M, int In, int Out, bool relu, int* dev_error, cudaStream_t st);
+cudaError_t tc_dense_dx(const bf16* dY, const bf16* W, const bf16* mask, bf16* dX, float* partial, int M, int In,
+                        int Out, int* dev_error, cudaStream_t st);
+cudaError_t tc_dense_dw(const bf16* dY, const bf16* X, float* dW, int M, int In, int Out, int* dev_error,
+                        cudaStream_t st);
 
 }  // namespace vgg

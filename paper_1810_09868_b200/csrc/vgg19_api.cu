@@ -131,6 +131,14 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
   p.a2 = take((size_t)B * 4096 * n->elt);
   p.logits = take((size_t)B * kClasses * 4);
   p.probs = take((size_t)B * kClasses * 4);
+  size_t dense_partial = 0;
+  for (int i = 0; i < kFcLayers; ++i) {
+    size_t e = tc_dense_scratch_elems(B, n->fc[i].In, n->fc[i].Out);
+    if (e > dense_partial) dense_partial = e;
+  }
+  if (256 * 512 > max_partial) max_partial = 256 * 512;  // bias-gradient column sums
+  if (mode == VGG19_MODE_FORWARD) p.partial = take(dense_partial * 4);
+  if (dense_partial > max_partial) max_partial = dense_partial;
   if (mode == VGG19_MODE_BACKWARD) {
     p.dl = take((size_t)B * kClasses * n->elt);
     p.dz2 = take((size_t)B * 4096 * n->elt);
@@ -199,10 +207,11 @@ struct Pass {
                      const T *mask) {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
-    if (n->use_tc && tc_wgrad_supported(s))
-      ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, db, fbuf(p.partial), s,
-                          n->dev_error, st), tc_wgrad_launches(s));
-    else
+    if (n->use_tc && tc_wgrad_supported(s)) {
+      ok(simt_bias_grad<T>(dz, db, fbuf(p.partial), (long)B * c.H * c.W, c.Cout, st), 2);
+      ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, fbuf(p.partial), s, n->dev_error, st),
+         tc_wgrad_launches(s));
+    } else
       ok(simt_conv3x3_wgrad<T>(x, dz, dW, db, fbuf(p.partial), s, st), 4);
     if (dx) {
       ConvShape t{B, c.H, c.W, c.Cout, c.Cin};  // a 3x3 correlation from Cout to Cin channels
@@ -212,6 +221,29 @@ struct Pass {
                       t, false, n->dev_error, st), 1);
       else
         ok(simt_conv3x3<T>(dz, wr, nullptr, mask, dx, t, false, st), 1);
+    }
+  }
+
+  bool tc_dense_ok(int B, const FcLayer &f) const { return n->use_tc && tc_dense_supported(B, f.In, f.Out); }
+
+  void dense_forward(const FcLayer &f, const T *x, int B, T *out_t, float *out_f) {
+    if (tc_dense_ok(B, f))
+      ok(tc_dense_forward((const bf16 *)x, (const bf16 *)wt(f.w_off), n->params + f.b_off, (bf16 *)out_t, out_f,
+                          fbuf(p.partial), B, f.In, f.Out, f.relu, n->dev_error, st), 2);
+    else
+      ok(simt_dense_nt<T>(x, wt(f.w_off), n->params + f.b_off, nullptr, out_t, out_f, B, f.Out, f.In, f.relu, st), 1);
+  }
+
+  // dW, db from (x, dy); dx = (dy W) [* (mask > 0)]
+  void dense_backward(const FcLayer &f, const T *x, const T *dy, int B, float *dW, float *db, T *dx, const T *mask) {
+    if (tc_dense_ok(B, f)) {
+      ok(simt_dense_db<T>(dy, db, B, f.Out, st), 1);
+      ok(tc_dense_dw((const bf16 *)dy, (const bf16 *)x, dW, B, f.In, f.Out, n->dev_error, st), 1);
+      ok(tc_dense_dx((const bf16 *)dy, (const bf16 *)wt(f.w_off), (const bf16 *)mask, (bf16 *)dx, fbuf(p.partial), B,
+                     f.In, f.Out, n->dev_error, st), 2);
+    } else {
+      ok(simt_dense_dw<T>(dy, x, dW, db, B, f.In, f.Out, st), 2);
+      ok(simt_dense_dx<T>(dy, wt(f.w_off), mask, dx, B, f.In, f.Out, st), 1);
     }
   }
 
@@ -227,12 +259,9 @@ struct Pass {
     }
     float *logits = a.logits ? a.logits : fbuf(p.logits);
     const FcLayer *f = n->fc;
-    ok(simt_dense_nt<T>(x, wt(f[0].w_off), n->params + f[0].b_off, nullptr, buf(p.a1), nullptr, B,
-                        f[0].Out, f[0].In, true, st), 1);
-    ok(simt_dense_nt<T>(buf(p.a1), wt(f[1].w_off), n->params + f[1].b_off, nullptr, buf(p.a2),
-                        nullptr, B, f[1].Out, f[1].In, true, st), 1);
-    ok(simt_dense_nt<T>(buf(p.a2), wt(f[2].w_off), n->params + f[2].b_off, nullptr, nullptr, logits,
-                        B, f[2].Out, f[2].In, false, st), 1);
+    dense_forward(f[0], x, B, buf(p.a1), nullptr);
+    dense_forward(f[1], buf(p.a1), B, buf(p.a2), nullptr);
+    dense_forward(f[2], buf(p.a2), B, nullptr, logits);
     if (a.probs && !a.grads)
       ok(softmax_xent<T>(logits, nullptr, a.probs, nullptr, nullptr, nullptr, B, kClasses, st), 1);
   }
@@ -248,12 +277,9 @@ struct Pass {
                        st), 2);
     const T *flat = buf(p.pooled[4]);
     // dense 3, 2, 1: filter gradient, then input gradient masked by the ReLU below
-    ok(simt_dense_dw<T>(buf(p.dl), buf(p.a2), g + f[2].w_off, g + f[2].b_off, B, f[2].In, f[2].Out, st), 2);
-    ok(simt_dense_dx<T>(buf(p.dl), wt(f[2].w_off), buf(p.a2), buf(p.dz2), B, f[2].In, f[2].Out, st), 1);
-    ok(simt_dense_dw<T>(buf(p.dz2), buf(p.a1), g + f[1].w_off, g + f[1].b_off, B, f[1].In, f[1].Out, st), 2);
-    ok(simt_dense_dx<T>(buf(p.dz2), wt(f[1].w_off), buf(p.a1), buf(p.dz1), B, f[1].In, f[1].Out, st), 1);
-    ok(simt_dense_dw<T>(buf(p.dz1), flat, g + f[0].w_off, g + f[0].b_off, B, f[0].In, f[0].Out, st), 2);
-    ok(simt_dense_dx<T>(buf(p.dz1), wt(f[0].w_off), nullptr, buf(p.dflat), B, f[0].In, f[0].Out, st), 1);
+    dense_backward(f[2], buf(p.a2), buf(p.dl), B, g + f[2].w_off, g + f[2].b_off, buf(p.dz2), buf(p.a2));
+    dense_backward(f[1], buf(p.a1), buf(p.dz2), B, g + f[1].w_off, g + f[1].b_off, buf(p.dz1), buf(p.a1));
+    dense_backward(f[0], flat, buf(p.dz1), B, g + f[0].w_off, g + f[0].b_off, buf(p.dflat), nullptr);
     // convolutions 16..1.  `dz` is the gradient at layer l's pre-activation.
     T *dz = buf(p.dza), *other = buf(p.dzb);
     {
@@ -328,6 +354,11 @@ int run_pass(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st) {
   if (rc != VGG19_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
   CUDA_TRY(n, ce);
   GraphEntry e{};
+  size_t n_nodes = 0;
+  if (cudaGraphGetNodes(graph, nullptr, &n_nodes) == cudaSuccess && n_nodes > 0) {
+    launches = (int)n_nodes;  // every node of the captured pass is a kernel launch
+    n->launches[mode] = launches;
+  }
   e.mode = mode; e.batch = a.batch; memcpy(e.p, key, sizeof key); e.n_kernels = launches;
   cudaError_t ie = cudaGraphInstantiate(&e.exec, graph, 0);
   cudaGraphDestroy(graph);
