@@ -48,7 +48,7 @@ template <typename T>
 cudaError_t simt_conv3x3_wgrad(const T* x, const T* dz, float* dW, float* db, float* partial,
                                ConvShape s, cudaStream_t st);
 
-// db[c] = sum_p dz[p][c]; partial: fp32 scratch of at least 256 * C elements.
+// db[c] = sum_p dz[p][c]; partial: fp32 scratch of at least 1024 * C elements.
 template <typename T>
 cudaError_t simt_bias_grad(const T* dz, float* db, float* partial, long P, int C, cudaStream_t st);
 // db[o] = sum_m dY[m][o]

@@ -10,6 +10,8 @@
 // what happens to the finished tile ("epilogue").
 #include "common.cuh"
 
+#include <type_traits>
+
 namespace vgg {
 
 namespace {
@@ -235,8 +237,107 @@ cudaError_t simt_conv3x3_wgrad(const T* x, const T* dz, float* dW, float* db, fl
   return cudaGetLastError();
 }
 
+
+// ---- bf16 fast paths: eight channels (16 bytes) per thread -------------------
+
+union Pack8 {
+  uint4 u;
+  __nv_bfloat162 h2[4];
+  bf16 h[8];
+};
+
+__global__ void maxpool_fwd_bf16x8_kernel(const bf16* __restrict__ x, bf16* __restrict__ y, long total8, int H, int W,
+                                          int C8) {
+  long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total8) return;
+  int Wo = W / 2, Ho = H / 2;
+  int c8 = i % C8; long t = i / C8;
+  int j = t % Wo; t /= Wo;
+  int ii = t % Ho; long n = t / Ho;
+  const uint4* p = reinterpret_cast<const uint4*>(x) + ((n * H + 2 * ii) * W + 2 * j) * C8 + c8;
+  Pack8 a, b, c, d, r;
+  a.u = __ldg(p); b.u = __ldg(p + C8); c.u = __ldg(p + (long)W * C8); d.u = __ldg(p + (long)W * C8 + C8);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) r.h2[e] = __hmax2(__hmax2(a.h2[e], b.h2[e]), __hmax2(c.h2[e], d.h2[e]));
+  reinterpret_cast<uint4*>(y)[i] = r.u;
+}
+
+__global__ void maxpool_bwd_relu_bf16x8_kernel(const bf16* __restrict__ y, const bf16* __restrict__ dp,
+                                               bf16* __restrict__ dy, long total8, int H, int W, int C8) {
+  long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total8) return;
+  int Wo = W / 2, Ho = H / 2;
+  int c8 = i % C8; long t = i / C8;
+  int j = t % Wo; t /= Wo;
+  int ii = t % Ho; long n = t / Ho;
+  const long base = ((n * H + 2 * ii) * W + 2 * j) * C8 + c8;
+  const long off[4] = {0, (long)C8, (long)W * C8, (long)W * C8 + C8};
+  Pack8 v[4], g, o[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) v[q].u = __ldg(reinterpret_cast<const uint4*>(y) + base + off[q]);
+  g.u = __ldg(reinterpret_cast<const uint4*>(dp) + i);
+  const bf16 zero = __float2bfloat16_rn(0.f);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    float m = __bfloat162float(v[0].h[e]);
+    int best = 0;
+#pragma unroll
+    for (int q = 1; q < 4; ++q) {
+      float w = __bfloat162float(v[q].h[e]);
+      if (w > m) { m = w; best = q; }
+    }
+    const bf16 gv = m > 0.f ? g.h[e] : zero;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) o[q].h[e] = q == best ? gv : zero;
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(dy)[base + off[q]] = o[q].u;
+}
+
+// partial[chunk][c] = sum over the chunk's pixels; a block covers 256 / C8 pixels per step
+__global__ void colsum_bf16x8_kernel(const bf16* __restrict__ dz, float* __restrict__ partial, long P, int C8,
+                                     long p_per_chunk) {
+  __shared__ float sm[256][9];
+  const int rows = 256 / C8;             // pixels in flight per step (C8 divides 256)
+  const int c8 = threadIdx.x % C8, r = threadIdx.x / C8;
+  const long p0 = (long)blockIdx.x * p_per_chunk, p1 = min(P, p0 + p_per_chunk);
+  float acc[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+  if (r < rows)
+    for (long p = p0 + r; p < p1; p += rows) {
+      Pack8 v;
+      v.u = __ldg(reinterpret_cast<const uint4*>(dz) + p * C8 + c8);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += __bfloat162float(v.h[e]);
+    }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) sm[threadIdx.x][e] = acc[e];
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < C8 * 8; idx += blockDim.x) {
+    const int cc = idx / 8, e = idx % 8;
+    float tot = 0.f;
+    for (int q = 0; q < rows; ++q) tot += sm[q * C8 + cc][e];
+    partial[(long)blockIdx.x * (C8 * 8) + idx] = tot;
+  }
+}
+
+bool colsum_fast_ok(int C) { return C % 8 == 0 && 256 % (C / 8) == 0 && C <= 256 * 8; }
+int colsum_fast_chunks(long P, int C) {
+  long rows = 256 / (C / 8);
+  long c = (P + rows * 16 - 1) / (rows * 16);
+  return (int)(c > 1024 ? 1024 : (c < 1 ? 1 : c));
+}
+
 template <typename T>
 cudaError_t simt_bias_grad(const T* dz, float* db, float* partial, long P, int C, cudaStream_t st) {
+  if (std::is_same<T, bf16>::value && colsum_fast_ok(C)) {
+    int chunks = colsum_fast_chunks(P, C);
+    long per = (P + chunks - 1) / chunks;
+    colsum_bf16x8_kernel<<<chunks, 256, 0, st>>>((const bf16*)dz, partial, P, C / 8, per);
+    reduce_splits_kernel<<<(C + 255) / 256, 256, 0, st>>>(partial, db, C, chunks);
+    return cudaGetLastError();
+  }
   int chunks = colsum_chunks(P);
   long per = (P + chunks - 1) / chunks;
   dim3 grid((C + 31) / 32, chunks), block(32, 8);
@@ -288,6 +389,11 @@ __global__ void maxpool_bwd_relu_kernel(const T* y, const T* dp, T* dy, long tot
 template <typename T>
 cudaError_t simt_maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st) {
   long total = (long)N * (H / 2) * (W / 2) * C;
+  if (std::is_same<T, bf16>::value && C % 8 == 0) {
+    maxpool_fwd_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>((const bf16*)x, (bf16*)y, total / 8, H,
+                                                                                 W, C / 8);
+    return cudaGetLastError();
+  }
   maxpool_fwd_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(x, y, total, H, W, C);
   return cudaGetLastError();
 }
@@ -296,6 +402,11 @@ template <typename T>
 cudaError_t simt_maxpool_bwd_relu(const T* y, const T* dp, T* dy, int N, int H, int W, int C,
                                   cudaStream_t st) {
   long total = (long)N * (H / 2) * (W / 2) * C;
+  if (std::is_same<T, bf16>::value && C % 8 == 0) {
+    maxpool_bwd_relu_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>(
+        (const bf16*)y, (const bf16*)dp, (bf16*)dy, total / 8, H, W, C / 8);
+    return cudaGetLastError();
+  }
   maxpool_bwd_relu_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(y, dp, dy, total, H, W, C);
   return cudaGetLastError();
 }

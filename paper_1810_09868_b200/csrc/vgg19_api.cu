@@ -136,7 +136,7 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
     size_t e = tc_dense_scratch_elems(B, n->fc[i].In, n->fc[i].Out);
     if (e > dense_partial) dense_partial = e;
   }
-  if (256 * 512 > max_partial) max_partial = 256 * 512;  // bias-gradient column sums
+  if (1024 * 512 > max_partial) max_partial = 1024 * 512;  // bias-gradient column sums
   if (mode == VGG19_MODE_FORWARD) p.partial = take(dense_partial * 4);
   if (dense_partial > max_partial) max_partial = dense_partial;
   if (mode == VGG19_MODE_BACKWARD) {
