@@ -100,6 +100,22 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def slowest_rank_ms(ms, world, device="cpu"):
+    """Max over ranks of a per-rank duration (all-reduce MAX on the default process group)."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_images_per_s(world, batch_per_rank, steps, slowest_ms):
+    """Whole-job throughput: every rank processes its own batch each step (weak scaling)."""
+    return world * batch_per_rank * steps / (slowest_ms * 1e-3)
+
+
 def oracle_forward_rate(n_images, seed_offset=0):
     """images/s of the fp64 CPU checker's forward pass on n_images of the workload."""
     import numpy as np
@@ -210,11 +226,7 @@ def run_native(args):
         torch.cuda.synchronize(dev)
 
     def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return slowest_rank_ms(ms, world, dev)
 
     def timed(fn, steps, warmup):
         with torch.cuda.stream(stream):
@@ -275,7 +287,7 @@ def run_native(args):
 
     n_fwd = pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_FORWARD)
     cpu_rate, cpu_dt = oracle_forward_rate(args.cpu_images)
-    value = world * BATCH * args.steps / (fwd_ms * 1e-3)
+    value = aggregate_images_per_s(world, BATCH, args.steps, fwd_ms)
     fwd_tflops = value * FWD_FLOP_PER_IMAGE / 1e12 / world
     out = {
         "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
@@ -314,7 +326,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
-    ap.add_argument("--cpu-images", type=int, default=8, help="images the CPU checker is timed on")
+    ap.add_argument("--cpu-images", type=int, default=24, help="images the CPU checker is timed on")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     if args.impl == "reference":
