@@ -151,6 +151,21 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_
   return d;
 }
 
+// Descriptor of an operand stored without swizzle as 8 x 16-byte "core
+// matrices" (8 rows of 8 bf16, 128 contiguous bytes).
+//   K-major : lbo = distance between the two 8-element K chunks of one MMA,
+//             sbo = distance between 8-row groups along M/N.
+//   MN-major: lbo = distance between 8-row groups along K,
+//             sbo = distance between 8-element groups along M/N.
+__device__ __forceinline__ uint64_t smem_desc_plain(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+
 // Instruction descriptor of tcgen05.mma kind::f16: bf16 A and B, fp32 D.
 // D format fp32 (bits 4-5 = 1), A/B format bf16 (bits 7-9, 10-12 = 1),
 // A / B major (bit 15 / 16: 0 = K-major, 1 = MN-major), N >> 3 in bits 17-22,
@@ -178,7 +193,11 @@ const TensorMapApi& tensor_map_api();
 
 // [rows][cols] bf16 row-major matrix, box = box_rows x 64 columns, 128 B swizzle.
 bool make_tiled_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// Same with a box of box_rows x 8 columns (16 bytes) and no swizzle.
+bool make_tiled_map_2d_c8(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 // NHWC bf16 tensor read through a 3x3 / pad 1 window: box = `pixels` x 64 channels, 128 B swizzle.
 bool make_im2col_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, uint32_t pixels);
+// Same for a tensor with 8 channels: box = `pixels` x 8 channels (16 bytes), no swizzle.
+bool make_im2col_map_c8(CUtensorMap* map, const void* base, int N, int H, int W, uint32_t pixels);
 
 }  // namespace vgg

@@ -1,0 +1,258 @@
+// First convolution layer (3 input channels) on tensor cores.
+//
+// With 3 channels a pixel is 6 bytes, below TMA's 16-byte granule, so the image
+// is first copied into an 8-channel tensor (channels 3..7 zero).  The layer is
+// then the implicit GEMM  D[pixel][cout] = sum_{tap, c<8} X8[pixel + tap][c] * W8[cout][tap][c]
+// with K = 10 taps x 8 channels = 80 (tap 9 is zero padding so that K is a
+// multiple of the MMA depth 16).  One K step of an MMA is two taps: each tap is
+// its own TMA im2col box of 128 pixels x 8 channels (16-byte rows, no swizzle),
+// i.e. exactly the 8x16-byte core-matrix layout tcgen05 reads without swizzle.
+// The layer is bound by writing its output (128 bytes per pixel), not by math.
+//
+// Roles and pipeline are those of the general convolution kernel: warp 0 TMA
+// producer, warp 1 MMA issuer and TMEM owner, warps 2-5 epilogue; double-buffered
+// accumulator; persistent CTAs; time-limited waits.
+#include "tc_common.cuh"
+#include "tc_kernels.cuh"
+
+namespace vgg {
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 64;
+constexpr int TAP_BYTES = BM * 16;        // 128 pixels x 8 channels
+constexpr int STAGE_BYTES = 10 * TAP_BYTES;
+constexpr int STAGES = 8;
+constexpr int W_TAP_BYTES = BN * 16;      // 64 output channels x 8 channels
+constexpr int W_BYTES = 10 * W_TAP_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + W_BYTES + 1024 + 256;
+constexpr int kThreads = 192;
+
+struct FirstArgs {
+  int pixels, H, W, m_tiles, relu;
+  const float* bias;
+  bf16* out;
+  int* dev_error;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, FirstArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t w_smem = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t bars = w_smem + W_BYTES;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto acc_full_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
+  auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+  const uint32_t w_bar = bars + 8u * (2 * STAGES + 4);
+  const uint32_t drain_bar = bars + 8u * (2 * STAGES + 5);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // the padding tap of every stage is multiplied by zero weights: it must hold finite numbers
+  {
+    uint8_t* base = smem_raw + (smem_base - smem_u32(smem_raw));
+    for (int i = threadIdx.x; i < STAGES * (TAP_BYTES / 16); i += kThreads) {
+      const int s = i / (TAP_BYTES / 16), q = i % (TAP_BYTES / 16);
+      *reinterpret_cast<uint4*>(base + s * STAGE_BYTES + 9 * TAP_BYTES + q * 16) = make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 128); }
+    mbar_init(w_bar, 1);
+    mbar_init(drain_bar, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&map_x);
+    tma_prefetch_desc(&map_w);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t fills[STAGES];
+#pragma unroll
+      for (int s = 0; s < STAGES; ++s) fills[s] = 0;
+      mbar_expect_tx(w_bar, W_BYTES);
+      for (int t = 0; t < 10; ++t) tma_load_2d(w_smem + t * W_TAP_BYTES, &map_w, w_bar, t * 8, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < a.m_tiles; tile += gridDim.x) {
+        const int p0 = tile * BM;
+        const int w0 = p0 % a.W, t = p0 / a.W;
+        const int h0 = t % a.H, n0 = t / a.H;
+        if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
+        const uint32_t sa = smem_base + stage * STAGE_BYTES;
+        mbar_expect_tx(full_bar(stage), 9 * TAP_BYTES);
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap)
+          tma_load_im2col_4d(sa + tap * TAP_BYTES, &map_x, full_bar(stage), 0, w0 - 1, h0 - 1, n0, (uint16_t)(tap % 3),
+                             (uint16_t)(tap / 3));
+        ++fills[stage];
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+      if (!ok) {
+        for (int s = 0; s < STAGES; ++s)
+          if (fills[s]) {
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(full_bar(s), (fills[s] - 1) & 1) && global_timer_ns() - t0 < 100000000ull) {}
+          }
+      }
+      // the filter load is always waited for by the MMA issuer or here
+      {
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(w_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = mbar_wait(w_bar, 0, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
+      for (int tile = blockIdx.x; tile < a.m_tiles && ok; tile += gridDim.x, ++local) {
+        const int buf = local & 1;
+        const uint32_t use = (uint32_t)(local >> 1);
+        if (!mbar_wait(acc_empty_bar(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
+        if (!mbar_wait(full_bar(stage), phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_base + stage * STAGE_BYTES;
+#pragma unroll
+        for (int j = 0; j < 5; ++j) {
+          // K step j = taps 2j and 2j+1: the two 8-element K chunks are one tap buffer apart,
+          // 8-row groups are 128 bytes apart
+          const uint64_t da = smem_desc_plain(sa + 2 * j * TAP_BYTES, TAP_BYTES, 128);
+          const uint64_t db = smem_desc_plain(w_smem + 2 * j * W_TAP_BYTES, W_TAP_BYTES, 128);
+          umma_bf16(tmem_base + (uint32_t)(buf * BN), da, db, idesc, j != 0 ? 1u : 0u);
+        }
+        umma_commit(empty_bar(stage));
+        umma_commit(acc_full_bar(buf));
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+      if (!ok) {
+        umma_commit(drain_bar);
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    int local = 0;
+    for (int tile = blockIdx.x; tile < a.m_tiles; tile += gridDim.x, ++local) {
+      const int buf = local & 1;
+      const uint32_t use = (uint32_t)(local >> 1);
+      if (!mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum)) break;
+      tc_fence_after();
+      const long pixel = (long)tile * BM + row;
+      const bool valid = pixel < a.pixels;
+      bf16* out_row = a.out + pixel * BN;
+#pragma unroll
+      for (int cc = 0; cc < BN; cc += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+        tmem_ld_wait();
+        if (valid) {
+          uint32_t packed[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
+            if (a.bias) { x0 += __ldg(a.bias + cc + j); x1 += __ldg(a.bias + cc + j + 1); }
+            if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
+            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+            packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          uint4* op = reinterpret_cast<uint4*>(out_row + cc);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty_bar(buf));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+// x8[p][0..2] = x[p][0..2], x8[p][3..7] = 0
+__global__ void pad_to8_kernel(const bf16* __restrict__ x, bf16* __restrict__ x8, long P) {
+  long p = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= P) return;
+  const unsigned short* s = reinterpret_cast<const unsigned short*>(x) + p * 3;
+  const uint32_t a = s[0], b = s[1], c = s[2];
+  reinterpret_cast<uint4*>(x8)[p] = make_uint4(a | (b << 16), c, 0u, 0u);
+}
+
+// w8[k][tap][c] = w[k][tap][c] for tap < 9 and c < 3, else 0
+__global__ void first_filter_kernel(const float* __restrict__ w, bf16* __restrict__ w8, int Cout) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= Cout * 80) return;
+  int c = i % 8, tap = (i / 8) % 10, k = i / 80;
+  float v = (tap < 9 && c < 3) ? w[(k * 9 + tap) * 3 + c] : 0.f;
+  w8[i] = __float2bfloat16_rn(v);
+}
+
+}  // namespace
+
+bool tc_first_conv_supported(ConvShape s) {
+  return s.Cin == 3 && s.Cout == 64 && s.H >= 2 && s.W >= 2 && (long)s.N * s.H * s.W < (1L << 31) - 256;
+}
+
+cudaError_t tc_pad_to8(const bf16* x, bf16* x8, long pixels, cudaStream_t st) {
+  pad_to8_kernel<<<(unsigned)((pixels + 255) / 256), 256, 0, st>>>(x, x8, pixels);
+  return cudaGetLastError();
+}
+
+cudaError_t tc_make_first_filter(const float* w, bf16* w8, cudaStream_t st) {
+  first_filter_kernel<<<(64 * 80 + 255) / 256, 256, 0, st>>>(w, w8, 64);
+  return cudaGetLastError();
+}
+
+cudaError_t tc_first_conv(const bf16* x8, const bf16* w8, const float* bias, bf16* out, ConvShape s, bool relu,
+                          int* dev_error, cudaStream_t st) {
+  if (!tc_first_conv_supported(s)) return cudaErrorInvalidValue;
+  CUtensorMap mx, mw;
+  if (!make_im2col_map_c8(&mx, x8, s.N, s.H, s.W, BM)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d_c8(&mw, w8, 64, 80, 64)) return cudaErrorInvalidValue;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_c8_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  FirstArgs a;
+  a.pixels = s.N * s.H * s.W; a.H = s.H; a.W = s.W;
+  a.m_tiles = (a.pixels + BM - 1) / BM;
+  a.relu = relu ? 1 : 0; a.bias = bias; a.out = out; a.dev_error = dev_error;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = a.m_tiles < sms ? a.m_tiles : sms;
+  conv3x3_c8_tc_kernel<<<grid, kThreads, SMEM_BYTES, st>>>(mx, mw, a);
+  return cudaGetLastError();
+}
+
+}  // namespace vgg

@@ -9,6 +9,8 @@
 // does).  A third form of B reads an NHWC activation through a 3x3 window
 // (TMA im2col) with the pixel index as k: that is the filter gradient
 //   dW[cout][tap][c] = sum_pixels dz[pixel][cout] * x[pixel shifted by tap][c].
+// A fourth form does the same for the 8-channel copy of the 3-channel image
+// (16-byte rows, no swizzle; the tile's 80 columns are 10 taps x 8 channels).
 //
 // One CTA computes one 128 x BN tile over its share of K (grid.y splits K):
 //   warp 0 TMA producer, warp 1 TMEM owner + single-thread MMA issuer, warps
@@ -24,7 +26,7 @@ namespace {
 
 using namespace tc;
 
-enum OperandMode { kKMajor = 0, kMnMajor = 1, kMnMajorIm2col = 2 };
+enum OperandMode { kKMajor = 0, kMnMajor = 1, kMnMajorIm2col = 2, kMnMajorIm2colC8 = 3 };
 
 constexpr int BM = 128, BK = 64;
 constexpr int A_BYTES = BM * BK * 2;
@@ -56,7 +58,7 @@ template <int BN, int AMODE, int BMODE>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs g) {
   constexpr int STAGE = stage_bytes<BN>();
-  constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+  constexpr int TMEM_COLS = BN <= 32 ? 32 : (BN <= 64 ? 64 : (BN <= 128 ? 128 : 256));
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = smem_base + g.stages * STAGE;
@@ -109,7 +111,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int kb = kb0; kb < kb1; ++kb) {
         if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, g.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
         const uint32_t sa = smem_base + stage * STAGE, sb = sa + A_BYTES;
-        mbar_expect_tx(full_bar(stage), STAGE);
+        mbar_expect_tx(full_bar(stage), BMODE == kMnMajorIm2colC8 ? A_BYTES + 9 * 1024 : STAGE);
         if (AMODE == kKMajor) {
           tma_load_2d(sa, &map_a, full_bar(stage), kb * BK, m0);
         } else {
@@ -121,7 +123,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         } else if (BMODE == kMnMajor) {
 #pragma unroll
           for (int q = 0; q < BN / 64; ++q) tma_load_2d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), n0 + 64 * q, kb * BK);
-        } else {
+        } else if (BMODE == kMnMajorIm2col) {
           const int p0 = kb * BK;
           const int w0 = p0 % g.W, t = p0 / g.W;
           const int h0 = t % g.H, img = t / g.H;
@@ -129,6 +131,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int q = 0; q < BN / 64; ++q)
             tma_load_im2col_4d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), c0 + 64 * q, w0 - 1, h0 - 1, img,
                                (uint16_t)tap_s, (uint16_t)tap_r);
+        } else {
+          // nine taps of the 8-channel image, 64 pixels x 16 bytes each; the tenth slot (columns
+          // 72..79 of the tile, never stored) is left as it is
+          const int p0 = kb * BK;
+          const int w0 = p0 % g.W, t = p0 / g.W;
+          const int h0 = t % g.H, img = t / g.H;
+#pragma unroll
+          for (int tap = 0; tap < 9; ++tap)
+            tma_load_im2col_4d(sb + tap * 1024, &map_b, full_bar(stage), 0, w0 - 1, h0 - 1, img, (uint16_t)(tap % 3),
+                               (uint16_t)(tap / 3));
         }
         ++fills[stage];
         if (++stage == g.stages) { stage = 0; phase ^= 1; }
@@ -155,7 +167,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int k = 0; k < BK / 16; ++k) {
           // K-major: 16 k = 32 bytes along the swizzled row.  MN-major: 16 k = 16 rows = 2048 bytes.
           const uint64_t da = AMODE == kKMajor ? smem_desc_sw128(sa + k * 32, 16) : smem_desc_sw128(sa + k * 2048, GROUP_BYTES);
-          const uint64_t db = BMODE == kKMajor ? smem_desc_sw128(sb + k * 32, 16) : smem_desc_sw128(sb + k * 2048, GROUP_BYTES);
+          // 8-channel form: 16 k = 16 rows of 16 bytes; 8-row groups 128 bytes apart, taps 1024 bytes apart
+          const uint64_t db = BMODE == kKMajor          ? smem_desc_sw128(sb + k * 32, 16)
+                              : BMODE == kMnMajorIm2colC8 ? smem_desc_plain(sb + k * 256, 128, 1024)
+                                                          : smem_desc_sw128(sb + k * 2048, GROUP_BYTES);
           umma_bf16(tmem_base, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
         }
         umma_commit(empty_bar(stage));
@@ -447,6 +462,48 @@ cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* pa
   }
   if (e != cudaSuccess || splits == 1) return e;
   return finish(g, splits, nullptr, false, nullptr, nullptr, dW, st);
+}
+
+// ---- filter gradient of the first layer (3 channels, read from the 8-channel copy) ----
+
+namespace {
+// dW[k][tap][c] = sum over splits of partial[split][k][tap * 8 + c], c < 3
+__global__ void wgrad_c8_finish_kernel(const float* __restrict__ partial, int splits, int Cout, float* dW) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= Cout * 27) return;
+  int c = i % 3, tap = (i / 3) % 9, k = i / 27;
+  float s = 0.f;
+  for (int z = 0; z < splits; ++z) s += partial[((long)z * Cout + k) * 80 + tap * 8 + c];
+  dW[i] = s;
+}
+void wgrad_c8_plan(ConvShape s, int* k_blocks, int* splits, int* per) {
+  const long P = (long)s.N * s.H * s.W;
+  *k_blocks = (int)((P + BK - 1) / BK);
+  plan_split(1, *k_blocks, splits, per);
+}
+}  // namespace
+
+size_t tc_first_wgrad_scratch_elems(ConvShape s) {
+  int kb, splits, per;
+  wgrad_c8_plan(s, &kb, &splits, &per);
+  return (size_t)splits * s.Cout * 80;
+}
+
+cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* partial, ConvShape s, int* dev_error,
+                           cudaStream_t st) {
+  const long P = (long)s.N * s.H * s.W;
+  CUtensorMap ma, mb;
+  if (!make_tiled_map_2d(&ma, dz, (uint64_t)P, (uint64_t)s.Cout, 64)) return cudaErrorInvalidValue;
+  if (!make_im2col_map_c8(&mb, x8, s.N, s.H, s.W, 64)) return cudaErrorInvalidValue;
+  GemmArgs g{};
+  int splits;
+  wgrad_c8_plan(s, &g.k_blocks, &splits, &g.kb_per_split);
+  g.M = s.Cout; g.N = 80; g.n_tiles = 1; g.H = s.H; g.W = s.W; g.Cin = 8;
+  g.dev_error = dev_error; g.ldc = 80; g.partial = partial;
+  cudaError_t e = launch_gemm_tc<80, kMnMajor, kMnMajorIm2colC8>(ma, mb, g, 1, splits, st);
+  if (e != cudaSuccess) return e;
+  wgrad_c8_finish_kernel<<<(s.Cout * 27 + 255) / 256, 256, 0, st>>>(partial, splits, s.Cout, dW);
+  return cudaGetLastError();
 }
 
 }  // namespace vgg

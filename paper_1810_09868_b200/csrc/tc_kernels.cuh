@@ -36,4 +36,16 @@ cudaError_t tc_dense_dx(const bf16* dY, const bf16* W, const bf16* mask, bf16* d
 cudaError_t tc_dense_dw(const bf16* dY, const bf16* X, float* dW, int M, int In, int Out, int* dev_error,
                         cudaStream_t st);
 
+// First layer (3 input channels, 64 output channels) on tensor cores, through an
+// 8-channel zero-padded copy x8 [N][H][W][8] of the image and a padded filter
+// w8 [64][10 taps][8] (tc_conv_first.cu).  dW fp32 [64][3][3][3].
+bool tc_first_conv_supported(ConvShape s);
+cudaError_t tc_pad_to8(const bf16* x, bf16* x8, long pixels, cudaStream_t st);
+cudaError_t tc_make_first_filter(const float* w, bf16* w8, cudaStream_t st);
+cudaError_t tc_first_conv(const bf16* x8, const bf16* w8, const float* bias, bf16* out, ConvShape s, bool relu,
+                          int* dev_error, cudaStream_t st);
+size_t tc_first_wgrad_scratch_elems(ConvShape s);
+cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* partial, ConvShape s, int* dev_error,
+                           cudaStream_t st);
+
 }  // namespace vgg

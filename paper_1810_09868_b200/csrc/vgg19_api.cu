@@ -62,6 +62,7 @@ struct vgg19 {
   float *params = nullptr;   // fp32 master, device
   void *params_t = nullptr;  // copy in the storage dtype (aliases params in fp32 mode)
   void *dgrad_w = nullptr;   // rotated filters for layers 2..16, storage dtype
+  bf16 *w8 = nullptr;        // first-layer filter padded to [64][10][8] (bf16 tensor-core path)
   int *dev_error = nullptr;
   void *ws = nullptr;
   size_t ws_bytes = 0;
@@ -101,6 +102,8 @@ struct Plan {
   size_t dl, dz2, dz1, dflat;  // backward: dlogits, dense pre-activation grads, d(flatten)
   size_t dza, dzb, dxlow;   // conv backward ping-pong and the pooled-resolution dx
   size_t partial;           // fp32 split-K partials
+  size_t x8;                // image copied to 8 channels (bf16 tensor-core path of layer 1)
+  bool valid = true;
   size_t row_loss, loss;
   size_t total;
   size_t io_images, io_labels, io_logits, io_probs, io_grads, io_loss, io_total;
@@ -126,6 +129,12 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
     size_t te = tc_wgrad_scratch_elems(s);
     if (te > pe) pe = te;
     if (pe > max_partial) max_partial = pe;
+  }
+  p.x8 = take(n->use_tc ? (size_t)B * n->cfg.height * n->cfg.width * 16 : 0);
+  {
+    const ConvLayer &c = n->conv[0];
+    size_t e = n->use_tc ? tc_first_wgrad_scratch_elems(ConvShape{B, c.H, c.W, c.Cin, c.Cout}) : 0;
+    if (e > max_partial) max_partial = e;
   }
   p.a1 = take((size_t)B * 4096 * n->elt);
   p.a2 = take((size_t)B * 4096 * n->elt);
@@ -189,12 +198,19 @@ struct Pass {
   void ok(cudaError_t e, int k) { if (err == cudaSuccess) err = e; launches += k; }
 
   bool tc_conv_ok(const ConvShape &s) const { return n->use_tc && tc_conv3x3_supported(s); }
+  // layer 1 on tensor cores needs the 8-channel image copy, i.e. a planned workspace
+  bool first_tc_ok(int l, const ConvShape &s) const {
+    return l == 0 && n->use_tc && p.valid && tc_first_conv_supported(s);
+  }
 
   // y = relu(conv(x) + b), optionally pooled
   void conv_forward(int l, const T *x, int B, T *y, T *pooled) {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
-    if (tc_conv_ok(s))
+    if (first_tc_ok(l, s)) {
+      ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
+      ok(tc_first_conv((const bf16 *)buf(p.x8), n->w8, n->params + c.b_off, (bf16 *)y, s, true, n->dev_error, st), 1);
+    } else if (tc_conv_ok(s))
       ok(tc_conv3x3((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
                     (bf16 *)y, s, true, n->dev_error, st), 1);
     else
@@ -207,7 +223,11 @@ struct Pass {
                      const T *mask) {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
-    if (n->use_tc && tc_wgrad_supported(s)) {
+    if (first_tc_ok(l, s)) {
+      ok(simt_bias_grad<T>(dz, db, fbuf(p.partial), (long)B * c.H * c.W, c.Cout, st), 2);
+      ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
+      ok(tc_first_wgrad((const bf16 *)buf(p.x8), (const bf16 *)dz, dW, fbuf(p.partial), s, n->dev_error, st), 2);
+    } else if (n->use_tc && tc_wgrad_supported(s)) {
       ok(simt_bias_grad<T>(dz, db, fbuf(p.partial), (long)B * c.H * c.W, c.Cout, st), 2);
       ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, fbuf(p.partial), s, n->dev_error, st),
          tc_wgrad_launches(s));
@@ -385,6 +405,7 @@ int upload_params(vgg19 *n, const float *host) {
     else
       CUDA_TRY(n, make_dgrad_filter<float>(n->params + c.w_off, (float *)n->dgrad_w + c.dgrad_off, c.Cin, c.Cout, 0));
   }
+  if (n->w8) CUDA_TRY(n, tc_make_first_filter(n->params + n->conv[0].w_off, n->w8, 0));
   CUDA_TRY(n, cudaDeviceSynchronize());
   return VGG19_OK;
 }
@@ -438,6 +459,7 @@ int create_common(const vgg19_config *cfg, vgg19 **out) {
     else n->params_t = n->params;
   }
   if (e == cudaSuccess) e = cudaMalloc(&n->dgrad_w, n->n_dgrad * n->elt);
+  if (e == cudaSuccess && n->use_tc) e = cudaMalloc(&n->w8, 64 * 80 * sizeof(bf16));
   if (e == cudaSuccess) e = cudaMalloc(&n->dev_error, 256);
   if (e == cudaSuccess) e = cudaMemset(n->dev_error, 0, 256);
   if (e != cudaSuccess) {
@@ -482,6 +504,7 @@ void vgg19_destroy(vgg19_t *n) {
   if (n->params_t && n->params_t != (void *)n->params) cudaFree(n->params_t);
   if (n->params) cudaFree(n->params);
   if (n->dgrad_w) cudaFree(n->dgrad_w);
+  if (n->w8) cudaFree(n->w8);
   if (n->dev_error) cudaFree(n->dev_error);
   delete n;
 }
@@ -629,12 +652,18 @@ int vgg19_conv_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t b
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
+  Plan plan{};
+  plan.valid = false;  // without a bound workspace the layer runs on kernels that need no scratch
+  if (n->ws && batch <= n->cfg.batch_max) {
+    Plan full = make_plan(n, batch, VGG19_MODE_FORWARD);
+    if (n->ws_bytes >= full.total) plan = full;
+  }
   if (n->cfg.dtype == VGG19_BF16) {
-    Pass<bf16> ps{n, Plan{}, st};
+    Pass<bf16> ps{n, plan, st};
     ps.conv_forward(layer - 1, (const bf16 *)x, batch, (bf16 *)y, (bf16 *)pooled);
     e = ps.err;
   } else {
-    Pass<float> ps{n, Plan{}, st};
+    Pass<float> ps{n, plan, st};
     ps.conv_forward(layer - 1, (const float *)x, batch, (float *)y, (float *)pooled);
     e = ps.err;
   }
@@ -720,9 +749,9 @@ int vgg19_describe(const vgg19_t *n, char *out, size_t cap) {
     ConvShape sd{n->cfg.batch_max, c.H, c.W, c.Cout, c.Cin};
     snprintf(line, sizeof line, "conv%-2d %3dx%-3d %3d->%-3d +bias +relu%s  fwd=%s dgrad=%s wgrad=%s\n",
              l + 1, c.H, c.W, c.Cin, c.Cout, c.pool_after ? " +maxpool2x2" : "",
-             n->use_tc && tc_conv3x3_supported(sh) ? "tcgen05" : "simt",
+             n->use_tc && (tc_conv3x3_supported(sh) || (l == 0 && tc_first_conv_supported(sh))) ? "tcgen05" : "simt",
              l == 0 ? "none" : (n->use_tc && tc_conv3x3_supported(sd) ? "tcgen05" : "simt"),
-             n->use_tc && tc_wgrad_supported(sh) ? "tcgen05" : "simt");
+             n->use_tc && (tc_wgrad_supported(sh) || (l == 0 && tc_first_conv_supported(sh))) ? "tcgen05" : "simt");
     s += line;
   }
   for (int i = 0; i < kFcLayers; ++i) {
