@@ -17,6 +17,11 @@
 //             the fp32 accumulator from tensor memory 32 columns at a time, adds
 //             the bias, applies ReLU and/or the ReLU mask of the layer below,
 //             rounds to bf16 and stores to the NHWC output.
+// Where the image is a whole number of 16 x 8 pixel patches (the 224x224 and
+// 112x112 layers) a tile is such a patch and its input comes from plain tiled
+// TMA boxes shifted by the tap, which the copy engine delivers several times
+// faster than im2col boxes; elsewhere a tile is 128 consecutive pixels (it may
+// span rows and images) fetched in im2col mode.
 // The accumulator is double buffered (2 x BN columns of tensor memory) so the
 // epilogue of one tile overlaps the main loop of the next; CTAs are persistent
 // and walk the tile list with a fixed stride.  Every wait has a time limit.
@@ -65,6 +70,18 @@ bool make_tiled_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64
 
 bool make_tiled_map_2d_c8(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
   return tiled_map(map, base, rows, cols, 8, box_rows, CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+
+bool make_patch_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, uint32_t box_w, uint32_t box_h) {
+  const TensorMapApi& api = tensor_map_api();
+  if (!api.ok) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+  cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+  cuuint32_t box[4] = {64, box_w, box_h, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return api.encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 bool make_im2col_map_c8(CUtensorMap* map, const void* base, int N, int H, int W, uint32_t pixels) {
@@ -122,11 +139,15 @@ struct ConvArgs {
   int Cout;
   int m_tiles, n_tiles;
   int relu;
+  int patch;      // 1: tiles are 16 x 8 pixel patches loaded with tiled boxes
+  int tiles_w, tiles_h;
   const float* bias;
   const bf16* mask;
   bf16* out;
   int* dev_error;
 };
+
+constexpr int PW = 16, PH = 8;  // patch of a tile in patch mode (PW * PH = BM)
 
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -177,16 +198,26 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
-        const int p0 = m_tile * BM;
-        const int w0 = p0 % a.W, t = p0 / a.W;
-        const int h0 = t % a.H, n0 = t / a.H;
+        int w0, h0, n0;
+        if (a.patch) {
+          const int tw = m_tile % a.tiles_w, t = m_tile / a.tiles_w;
+          w0 = tw * PW; h0 = (t % a.tiles_h) * PH; n0 = t / a.tiles_h;
+        } else {
+          const int p0 = m_tile * BM;
+          w0 = p0 % a.W;
+          const int t = p0 / a.W;
+          h0 = t % a.H; n0 = t / a.H;
+        }
         for (int kb = 0; kb < k_blocks; ++kb) {
           const int rs = kb / a.cin_blocks, cb = kb - rs * a.cin_blocks;
           const int r = rs / 3, s = rs - r * 3;
           if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
           mbar_expect_tx(full_bar(stage), T::STAGE_BYTES);
-          tma_load_im2col_4d(sa, &map_x, full_bar(stage), cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
+          if (a.patch)
+            tma_load_4d(sa, &map_x, full_bar(stage), cb * BK, w0 + s - 1, h0 + r - 1, n0);
+          else
+            tma_load_im2col_4d(sa, &map_x, full_bar(stage), cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
           tma_load_2d(sb, &map_w, full_bar(stage), kb * BK, n_tile * BN);
           ++fills[stage];
           if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
@@ -249,7 +280,14 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
       if (!mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum)) { ok = false; break; }
       tc_fence_after();
-      const long pixel = (long)m_tile * BM + row;
+      long pixel;
+      if (a.patch) {
+        const int tw = m_tile % a.tiles_w, t = m_tile / a.tiles_w;
+        const int th = t % a.tiles_h, img = t / a.tiles_h;
+        pixel = ((long)img * a.H + th * PH + row / PW) * a.W + tw * PW + row % PW;
+      } else {
+        pixel = (long)m_tile * BM + row;
+      }
       const bool valid = pixel < a.pixels;
       const int c_base = n_tile * BN;
       bf16* out_row = a.out + pixel * a.Cout + c_base;
@@ -338,9 +376,16 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
   if (!tc_conv3x3_supported(s)) return cudaErrorInvalidValue;
   const int BN = pick_bn(s.Cout);
   CUtensorMap mx, mw;
-  if (!make_im2col_map(&mx, in, s.N, s.H, s.W, s.Cin, BM)) return cudaErrorInvalidValue;
+  const bool patch = s.W % PW == 0 && s.H % PH == 0;
+  if (patch) {
+    if (!make_patch_map(&mx, in, s.N, s.H, s.W, s.Cin, PW, PH)) return cudaErrorInvalidValue;
+  } else if (!make_im2col_map(&mx, in, s.N, s.H, s.W, s.Cin, BM)) {
+    return cudaErrorInvalidValue;
+  }
   if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
   ConvArgs a;
+  a.patch = patch ? 1 : 0;
+  a.tiles_w = s.W / PW; a.tiles_h = s.H / PH;
   a.pixels = s.N * s.H * s.W;
   a.H = s.H; a.W = s.W;
   a.cin_blocks = s.Cin / 64;
