@@ -1,0 +1,303 @@
+// 3x3 convolution on tcgen05 with the input patch held in shared memory once
+// for all nine filter taps.
+//
+// The general kernel (tc_kernels.cu) fetches the input tile again for every
+// tap, so it moves nine times the input through the L2-to-SM path; on the
+// large-image layers with few channels (224x224 and 112x112, 64-128 channels)
+// that path, not the tensor pipe, sets the speed.  Here a tile is a patch of
+// 8 (wide) x 16 (high) output pixels.  For each block of 64 input channels the
+// producer loads the 10 x 18 input patch (one pixel of halo, zero-filled
+// outside the image by TMA) once: 180 rows of 128 bytes, 128-byte swizzled.
+// Output pixel (ph, pw) and tap (r, s) read patch row (ph + r) * 10 + pw + s, so
+// for a fixed tap the 128 rows of the MMA's A operand are 16 groups of 8
+// consecutive rows, 10 rows apart: a K-major operand with a stride of
+// 1280 bytes between 8-row groups, starting (r * 10 + s) rows into the patch.
+// The nine taps are nine MMAs on the same buffer with different start rows.
+// Filter slices (BN x 64 per tap) stream through their own ring.
+//
+// Warps: 0 patch producer, 1 MMA issuer + TMEM owner, 2-5 epilogue, 6 filter
+// producer.  Accumulator double-buffered; persistent CTAs; time-limited waits.
+#include "tc_common.cuh"
+#include "tc_kernels.cuh"
+
+namespace vgg {
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BK = 64;
+constexpr int PW = 8, PH = 16;                  // output patch
+constexpr int IW = PW + 2, IH = PH + 2;         // input patch with halo
+constexpr int A_BYTES = IW * IH * 128;          // 23040
+constexpr int A_SLOT = 23 * 1024;               // 1024-byte aligned slot
+constexpr int NA = 3;
+constexpr int kThreads = 224;
+
+template <int BN>
+struct HaloTile {
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int NB = (227 * 1024 - 2048 - NA * A_SLOT) / B_BYTES > 12 ? 12 : (227 * 1024 - 2048 - NA * A_SLOT) / B_BYTES;
+  static constexpr int SMEM_BYTES = NA * A_SLOT + NB * B_BYTES + 1024 + 512;
+};
+
+struct HaloArgs {
+  int N, H, W;
+  int cin_blocks, Cin, Cout;
+  int tiles_w, tiles_h, m_tiles, n_tiles;
+  int relu;
+  const float* bias;
+  const bf16* mask;
+  bf16* out;
+  int* dev_error;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, HaloArgs a) {
+  using T = HaloTile<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t b_base = smem_base + NA * A_SLOT;
+  const uint32_t bars = b_base + T::NB * T::B_BYTES;
+  auto a_full = [&](int s) { return bars + 8u * s; };
+  auto a_empty = [&](int s) { return bars + 8u * (NA + s); };
+  auto b_full = [&](int s) { return bars + 8u * (2 * NA + s); };
+  auto b_empty = [&](int s) { return bars + 8u * (2 * NA + T::NB + s); };
+  auto acc_full = [&](int b) { return bars + 8u * (2 * NA + 2 * T::NB + b); };
+  auto acc_empty = [&](int b) { return bars + 8u * (2 * NA + 2 * T::NB + 2 + b); };
+  const uint32_t drain_bar = bars + 8u * (2 * NA + 2 * T::NB + 4);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_tiles = a.m_tiles * a.n_tiles;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
+    for (int s = 0; s < T::NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 128); }
+    mbar_init(drain_bar, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&map_x);
+    tma_prefetch_desc(&map_w);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ---------------- input-patch producer ----------------
+    if (lane == 0) {
+      uint32_t fills[NA];
+#pragma unroll
+      for (int s = 0; s < NA; ++s) fills[s] = 0;
+      int slot = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m_tile = tile / a.n_tiles;
+        const int tw = m_tile % a.tiles_w, t = m_tile / a.tiles_w;
+        const int w0 = tw * PW, h0 = (t % a.tiles_h) * PH, img = t / a.tiles_h;
+        for (int cb = 0; cb < a.cin_blocks; ++cb) {
+          if (!mbar_wait(a_empty(slot), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
+          mbar_expect_tx(a_full(slot), A_BYTES);
+          tma_load_4d(smem_base + slot * A_SLOT, &map_x, a_full(slot), cb * BK, w0 - 1, h0 - 1, img);
+          ++fills[slot];
+          if (++slot == NA) { slot = 0; phase ^= 1; }
+        }
+      }
+      if (!ok)
+        for (int s = 0; s < NA; ++s)
+          if (fills[s]) {
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(a_full(s), (fills[s] - 1) & 1) && global_timer_ns() - t0 < 100000000ull) {}
+          }
+    }
+  } else if (warp == 6) {
+    // ---------------- filter producer ----------------
+    if (lane == 0) {
+      uint32_t fills[T::NB];
+#pragma unroll
+      for (int s = 0; s < T::NB; ++s) fills[s] = 0;
+      int slot = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int n_tile = tile % a.n_tiles;
+        for (int cb = 0; cb < a.cin_blocks && ok; ++cb)
+          for (int tap = 0; tap < 9; ++tap) {
+            if (!mbar_wait(b_empty(slot), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
+            mbar_expect_tx(b_full(slot), T::B_BYTES);
+            tma_load_2d(b_base + slot * T::B_BYTES, &map_w, b_full(slot), tap * a.Cin + cb * BK, n_tile * BN);
+            ++fills[slot];
+            if (++slot == T::NB) { slot = 0; phase ^= 1; }
+          }
+      }
+      if (!ok)
+        for (int s = 0; s < T::NB; ++s)
+          if (fills[s]) {
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(b_full(s), (fills[s] - 1) & 1) && global_timer_ns() - t0 < 100000000ull) {}
+          }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, 0, 0);
+      int aslot = 0, bslot = 0;
+      uint32_t aphase = 0, bphase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+        const int buf = local & 1;
+        const uint32_t use = (uint32_t)(local >> 1);
+        if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int cb = 0; cb < a.cin_blocks && ok; ++cb) {
+          if (!mbar_wait(a_full(aslot), aphase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+          const uint32_t sa = smem_base + aslot * A_SLOT;
+          for (int tap = 0; tap < 9; ++tap) {
+            if (!mbar_wait(b_full(bslot), bphase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sb = b_base + bslot * T::B_BYTES;
+            const int r = tap / 3, s = tap - r * 3;
+            const uint32_t a_tap = sa + (uint32_t)(r * IW + s) * 128u;
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k) {
+              const uint64_t da = smem_desc_sw128_sbo(a_tap + k * 32, IW * 128);
+              const uint64_t db = smem_desc_sw128(sb + k * 32, 16);
+              umma_bf16(d_tmem, da, db, idesc, (cb | tap | k) != 0 ? 1u : 0u);
+            }
+            umma_commit(b_empty(bslot));
+            if (++bslot == T::NB) { bslot = 0; bphase ^= 1; }
+          }
+          if (!ok) break;
+          umma_commit(a_empty(aslot));
+          if (++aslot == NA) { aslot = 0; aphase ^= 1; }
+        }
+        if (ok) umma_commit(acc_full(buf));
+      }
+      if (!ok) {
+        umma_commit(drain_bar);
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else {
+    // ---------------- epilogue ----------------
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    int local = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+      const int buf = local & 1;
+      const uint32_t use = (uint32_t)(local >> 1);
+      const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
+      if (!mbar_wait(acc_full(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum)) break;
+      tc_fence_after();
+      const int tw = m_tile % a.tiles_w, t = m_tile / a.tiles_w;
+      const int h = (t % a.tiles_h) * PH + row / PW, img = t / a.tiles_h;
+      const bool valid = h < a.H;
+      const long pixel = ((long)img * a.H + h) * a.W + tw * PW + row % PW;
+      const int c_base = n_tile * BN;
+      bf16* out_row = a.out + pixel * a.Cout + c_base;
+      const bf16* mask_row = a.mask ? a.mask + pixel * a.Cout + c_base : nullptr;
+#pragma unroll 1
+      for (int cc = 0; cc < BN; cc += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+        tmem_ld_wait();
+        if (valid) {
+          uint32_t packed[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
+            if (a.bias) { x0 += __ldg(a.bias + c_base + cc + j); x1 += __ldg(a.bias + c_base + cc + j + 1); }
+            if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
+            __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+            packed[j >> 1] = *reinterpret_cast<uint32_t*>(&hh);
+          }
+          if (mask_row) {
+            const uint4* mp = reinterpret_cast<const uint4*>(mask_row + cc);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 m = __ldg(mp + q);
+              const uint32_t mw[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t lo = mw[e] & 0xFFFFu, hi = mw[e] >> 16;
+                uint32_t keep = 0;
+                if (lo != 0 && !(lo & 0x8000u)) keep |= 0x0000FFFFu;
+                if (hi != 0 && !(hi & 0x8000u)) keep |= 0xFFFF0000u;
+                packed[q * 4 + e] &= keep;
+              }
+            }
+          }
+          uint4* op = reinterpret_cast<uint4*>(out_row + cc);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty(buf));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+template <int BN>
+cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, HaloArgs a, cudaStream_t st) {
+  using T = HaloTile<BN>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_halo_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int tiles = a.m_tiles * a.n_tiles;
+  conv3x3_halo_tc_kernel<BN><<<tiles < sms ? tiles : sms, kThreads, T::SMEM_BYTES, st>>>(mx, mw, a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_conv3x3_halo_supported(ConvShape s) {
+  return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.Cout <= 128 && s.W % PW == 0 && s.H % PH == 0 && s.W >= 64 &&
+         (long)s.N * s.H * s.W < (1L << 31) - 256;
+}
+
+cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out, ConvShape s,
+                            bool relu, int* dev_error, cudaStream_t st) {
+  if (!tc_conv3x3_halo_supported(s)) return cudaErrorInvalidValue;
+  const int BN = s.Cout % 128 == 0 ? 128 : 64;
+  CUtensorMap mx, mw;
+  if (!make_patch_map(&mx, in, s.N, s.H, s.W, s.Cin, IW, IH)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
+  HaloArgs a;
+  a.N = s.N; a.H = s.H; a.W = s.W;
+  a.cin_blocks = s.Cin / 64; a.Cin = s.Cin; a.Cout = s.Cout;
+  a.tiles_w = s.W / PW; a.tiles_h = s.H / PH;
+  a.m_tiles = s.N * a.tiles_w * a.tiles_h;
+  a.n_tiles = s.Cout / BN;
+  a.relu = relu ? 1 : 0; a.bias = bias; a.mask = mask; a.out = out; a.dev_error = dev_error;
+  return BN == 128 ? launch_halo<128>(mx, mw, a, st) : launch_halo<64>(mx, mw, a, st);
+}
+
+}  // namespace vgg

@@ -17,6 +17,12 @@ bool tc_conv3x3_supported(ConvShape s);
 cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const bf16* mask,
                        bf16* out, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
 
+// The same convolution with the input patch (plus halo) kept in shared memory
+// for all nine taps (tc_conv_halo.cu): the large-image, few-channel layers.
+bool tc_conv3x3_halo_supported(ConvShape s);
+cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out,
+                            ConvShape s, bool relu, int* dev_error, cudaStream_t st);
+
 // Filter gradient of the same convolution as a GEMM with M = Cout, N = 9*Cin,
 // K = pixels (both operands read transposed, x through the im2col window):
 // dW fp32 [Cout][3][3][Cin].  partial: fp32 scratch of tc_wgrad_scratch_elems().

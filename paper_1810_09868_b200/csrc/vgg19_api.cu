@@ -210,7 +210,10 @@ struct Pass {
     if (first_tc_ok(l, s)) {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       ok(tc_first_conv((const bf16 *)buf(p.x8), n->w8, n->params + c.b_off, (bf16 *)y, s, true, n->dev_error, st), 1);
-    } else if (tc_conv_ok(s))
+    } else if (n->use_tc && tc_conv3x3_halo_supported(s))
+      ok(tc_conv3x3_halo((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr, (bf16 *)y, s, true,
+                         n->dev_error, st), 1);
+    else if (tc_conv_ok(s))
       ok(tc_conv3x3((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
                     (bf16 *)y, s, true, n->dev_error, st), 1);
     else
@@ -236,7 +239,10 @@ struct Pass {
     if (dx) {
       ConvShape t{B, c.H, c.W, c.Cout, c.Cin};  // a 3x3 correlation from Cout to Cin channels
       const T *wr = static_cast<const T *>(n->dgrad_w) + c.dgrad_off;
-      if (tc_conv_ok(t))
+      if (n->use_tc && tc_conv3x3_halo_supported(t))
+        ok(tc_conv3x3_halo((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx, t, false,
+                           n->dev_error, st), 1);
+      else if (tc_conv_ok(t))
         ok(tc_conv3x3((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
                       t, false, n->dev_error, st), 1);
       else
