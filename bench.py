@@ -320,6 +320,35 @@ def run_native(args):
         dist.destroy_process_group()
 
 
+def run_profile_layer(args):
+    """A few launches of one convolution layer on a small batch, for `ncu -k ...` captures
+    (prints nothing the driver parses)."""
+    import torch
+    import seeded_inputs as si
+    import paper_1810_09868_b200 as pkg
+    L, B = args.profile_layer, args.profile_batch
+    s, ci, co = CONV[L - 1]
+    params = si.vgg19_params(H, W, seed=0, bf16_exact=True)
+    net = pkg.Net(H, W, B, pkg.VGG19_BF16, params=params)
+    x = torch.from_numpy(si.normal(B * s * s * ci, seed=100 + L, take_abs=True, bf16_exact=True)
+                         .reshape(B, s, s, ci)).cuda().to(torch.bfloat16)
+    y = torch.empty(B, s, s, co, dtype=torch.bfloat16, device="cuda")
+    stream = torch.cuda.Stream()
+    if args.profile_kind == "fwd":
+        for _ in range(3):
+            pkg.vgg19_conv_layer_forward(net.handle, L, x, B, y, None, stream)
+    else:
+        dz = torch.from_numpy(si.normal(B * s * s * co, seed=200 + L, stddev=1e-3, bf16_exact=True)
+                              .reshape(B, s, s, co)).cuda().to(torch.bfloat16)
+        dw = torch.empty(co, 3, 3, ci, dtype=torch.float32, device="cuda")
+        db = torch.empty(co, dtype=torch.float32, device="cuda")
+        dx = None if L == 1 else torch.empty(B, s, s, ci, dtype=torch.bfloat16, device="cuda")
+        for _ in range(3):
+            pkg.vgg19_conv_layer_backward(net.handle, L, x, dz, B, dw, db, dx, stream)
+    net.sync_status(stream)
+    print(f"profiled conv layer {L} ({args.profile_kind}), batch {B}: {s}x{s}, {ci}->{co}")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -327,7 +356,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--cpu-images", type=int, default=24, help="images the CPU checker is timed on")
+    ap.add_argument("--profile-layer", type=int, default=0, help="run only this conv layer (1..16) a few times and exit")
+    ap.add_argument("--profile-batch", type=int, default=16)
+    ap.add_argument("--profile-kind", default="fwd", choices=["fwd", "bwd"])
     args = ap.parse_args()
+    if args.profile_layer:
+        run_profile_layer(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     if args.impl == "reference":
         run_reference(args)

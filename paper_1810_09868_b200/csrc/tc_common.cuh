@@ -15,7 +15,7 @@ namespace tc {
 
 // A wait gives up after this long (far above any tile's duration, profiler
 // replays included), records a DeviceError code and lets the CTA drain.
-constexpr unsigned long long kWaitLimitNs = 2000ull * 1000ull * 1000ull;
+constexpr long long kWaitLimitCycles = 4000ll * 1000ll * 1000ll;  // about two seconds of SM clock
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -53,15 +53,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Wait for the phase with the given parity.  Returns false if another role has
 // already given up (abort flag in shared memory) or if this wait ran out, in
-// which case `code` is recorded in the device error word.
+// which case `code` is recorded in the device error word.  The limit is counted
+// on the SM's own cycle counter, which is cheap to read; the global nanosecond
+// timer costs on the order of a microsecond per read and would sit on the
+// critical path of every hand-off.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int* dev_error, int code) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (;;) {
-    if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) {
+    if (clock64() - t0 > kWaitLimitCycles) {
       *abort_flag = 1;
       atomicCAS(dev_error, 0, code);
       return false;

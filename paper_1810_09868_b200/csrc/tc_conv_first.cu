@@ -50,6 +50,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   const uint32_t drain_bar = bars + 8u * (2 * STAGES + 5);
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  __shared__ __align__(16) float bias_s[512];  // the layer's bias (zeros when it has none)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -62,6 +63,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  for (int i = threadIdx.x; i < BN; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -172,7 +174,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
-            if (a.bias) { x0 += __ldg(a.bias + cc + j); x1 += __ldg(a.bias + cc + j + 1); }
+            x0 += bias_s[cc + j]; x1 += bias_s[cc + j + 1];
             if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
             __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
             packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);

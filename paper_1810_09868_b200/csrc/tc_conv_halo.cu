@@ -36,7 +36,7 @@ constexpr int kThreads = 224;
 template <int BN>
 struct HaloTile {
   static constexpr int B_BYTES = BN * BK * 2;
-  static constexpr int NB = (227 * 1024 - 2048 - NA * A_SLOT) / B_BYTES > 12 ? 12 : (227 * 1024 - 2048 - NA * A_SLOT) / B_BYTES;
+  static constexpr int NB = (227 * 1024 - 4608 - NA * A_SLOT) / B_BYTES > 12 ? 12 : (227 * 1024 - 4608 - NA * A_SLOT) / B_BYTES;
   static constexpr int SMEM_BYTES = NA * A_SLOT + NB * B_BYTES + 1024 + 512;
 };
 
@@ -68,10 +68,12 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const uint32_t drain_bar = bars + 8u * (2 * NA + 2 * T::NB + 4);
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  __shared__ __align__(16) float bias_s[512];  // the layer's bias (zeros when it has none)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_tiles = a.m_tiles * a.n_tiles;
 
+  for (int i = threadIdx.x; i < a.Cout; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
@@ -218,7 +220,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
-            if (a.bias) { x0 += __ldg(a.bias + c_base + cc + j); x1 += __ldg(a.bias + c_base + cc + j + 1); }
+            x0 += bias_s[c_base + cc + j]; x1 += bias_s[c_base + cc + j + 1];
             if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
             __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
             packed[j >> 1] = *reinterpret_cast<uint32_t*>(&hh);

@@ -127,7 +127,7 @@ template <int BN>
 struct ConvTile {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (kSmemLimit - 2048) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 2048) / STAGE_BYTES;
+  static constexpr int STAGES = (kSmemLimit - 4608) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608) / STAGE_BYTES;  // leaves room for barriers, bias and alignment
   static constexpr int TMEM_COLS = 2 * BN;  // 128, 256 or 512: powers of two
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
@@ -164,11 +164,13 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   const uint32_t drain_bar = bars + 8u * (2 * T::STAGES + 4);
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  __shared__ __align__(16) float bias_s[512];  // the layer's bias (zeros when it has none)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k_blocks = 9 * a.cin_blocks;
   const int total_tiles = a.m_tiles * a.n_tiles;
 
+  for (int i = threadIdx.x; i < a.Cout; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < T::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -302,7 +304,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
-            if (a.bias) { x0 += __ldg(a.bias + c_base + cc + j); x1 += __ldg(a.bias + c_base + cc + j + 1); }
+            x0 += bias_s[c_base + cc + j]; x1 += bias_s[c_base + cc + j + 1];
             if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
             __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
             packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
@@ -367,7 +369,7 @@ int pick_bn(int Cout) { return Cout % 256 == 0 ? 256 : (Cout % 128 == 0 ? 128 : 
 }  // namespace
 
 bool tc_conv3x3_supported(ConvShape s) {
-  return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.H >= 2 && s.W >= 2 && s.N >= 1 &&
+  return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.Cout <= 512 && s.H >= 2 && s.W >= 2 && s.N >= 1 &&
          (long)s.N * s.H * s.W < (1L << 31) - 256;
 }
 
