@@ -160,6 +160,24 @@ __global__ void reduce_splits_kernel(const float* partial, float* out, long n, i
   out[i] = s;
 }
 
+// out[c] = sum over chunks of partial[chunk][c]: eight threads per column add interleaved
+// chunks, then the eight sums are added in a fixed order
+__global__ void reduce_columns_kernel(const float* __restrict__ partial, float* __restrict__ out, int C, int chunks) {
+  __shared__ float sm[8][33];
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  float s = 0.f;
+  if (c < C)
+    for (int z = threadIdx.y; z < chunks; z += 8) s += partial[(long)z * C + c];
+  sm[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && c < C) {
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tot += sm[i][threadIdx.x];
+    out[c] = tot;
+  }
+}
+
 // partial[chunk][c] = sum of dz[p][c] over the chunk's pixels
 template <typename T>
 __global__ void colsum_partial_kernel(const T* dz, float* partial, long P, int C, long p_per_chunk) {
@@ -326,7 +344,7 @@ bool colsum_fast_ok(int C) { return C % 8 == 0 && 256 % (C / 8) == 0 && C <= 256
 int colsum_fast_chunks(long P, int C) {
   long rows = 256 / (C / 8);
   long c = (P + rows * 16 - 1) / (rows * 16);
-  return (int)(c > 1024 ? 1024 : (c < 1 ? 1 : c));
+  return (int)(c > 592 ? 592 : (c < 1 ? 1 : c));
 }
 
 template <typename T>
@@ -335,7 +353,7 @@ cudaError_t simt_bias_grad(const T* dz, float* db, float* partial, long P, int C
     int chunks = colsum_fast_chunks(P, C);
     long per = (P + chunks - 1) / chunks;
     colsum_bf16x8_kernel<<<chunks, 256, 0, st>>>((const bf16*)dz, partial, P, C / 8, per);
-    reduce_splits_kernel<<<(C + 255) / 256, 256, 0, st>>>(partial, db, C, chunks);
+    reduce_columns_kernel<<<(C + 31) / 32, dim3(32, 8), 0, st>>>(partial, db, C, chunks);
     return cudaGetLastError();
   }
   int chunks = colsum_chunks(P);

@@ -101,13 +101,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      int tap_s = 0, tap_r = 0, c0 = 0;
-      if (BMODE == kMnMajorIm2col) {
-        const int tap = n0 / g.Cin;
-        c0 = n0 - tap * g.Cin;
-        tap_r = tap / 3;
-        tap_s = tap - tap_r * 3;
-      }
       for (int kb = kb0; kb < kb1; ++kb) {
         if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, g.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
         const uint32_t sa = smem_base + stage * STAGE, sb = sa + A_BYTES;
@@ -128,9 +121,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int w0 = p0 % g.W, t = p0 / g.W;
           const int h0 = t % g.H, img = t / g.H;
 #pragma unroll
-          for (int q = 0; q < BN / 64; ++q)
-            tma_load_im2col_4d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), c0 + 64 * q, w0 - 1, h0 - 1, img,
-                               (uint16_t)tap_s, (uint16_t)tap_r);
+          for (int q = 0; q < BN / 64; ++q) {
+            // each 64-column group of the tile is (tap, 64 channels); groups of one tile may be different taps
+            const int j = n0 + 64 * q, tap = j / g.Cin, c0 = j - tap * g.Cin;
+            tma_load_im2col_4d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), c0, w0 - 1, h0 - 1, img,
+                               (uint16_t)(tap % 3), (uint16_t)(tap / 3));
+          }
         } else {
           // nine taps of the 8-channel image, 64 pixels x 16 bytes each; the tenth slot (columns
           // 72..79 of the tile, never stored) is left as it is
@@ -412,7 +408,8 @@ cudaError_t tc_dense_dw(const bf16* dY, const bf16* X, float* dW, int M, int In,
 // ---- convolution filter gradient ----------------------------------------------
 
 namespace {
-int wgrad_bn(int Cin) { return Cin % 256 == 0 ? 256 : (Cin % 128 == 0 ? 128 : 64); }
+// 9*Cin columns in tiles of whole 64-channel groups: 256 or 128 wide, and 192 (three taps) for 64 channels
+int wgrad_bn(int Cin) { return Cin % 256 == 0 ? 256 : (Cin % 128 == 0 ? 128 : 192); }
 void wgrad_plan(ConvShape s, int* m_tiles, int* n_tiles, int* k_blocks, int* splits, int* per) {
   const long P = (long)s.N * s.H * s.W;
   *m_tiles = (s.Cout + BM - 1) / BM;
@@ -458,7 +455,7 @@ cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* pa
   switch (BN) {
     case 256: e = launch_gemm_tc<256, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
     case 128: e = launch_gemm_tc<128, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
-    default: e = launch_gemm_tc<64, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
+    default: e = launch_gemm_tc<192, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
   }
   if (e != cudaSuccess || splits == 1) return e;
   return finish(g, splits, nullptr, false, nullptr, nullptr, dW, st);
