@@ -278,12 +278,19 @@ def run_native(args):
         bwd()  # leaves the batch-100 activations of every layer in the workspace
     stream.synchronize()
     layers = time_conv_layers(pkg, net, torch, stream)
-    conv_ms = sum(ms for _, ms, _, _ in layers)
-    conv_flop = sum(f for _, _, f, _ in layers)
+    # dominant kernel: conv3x3_tc_kernel<256>, the 12 launches of layers 5..16 (about half the pass)
+    dom = [t for t in layers if t[0] >= 5]
+    conv_ms = sum(ms for _, ms, _, _ in dom)
+    conv_flop = sum(f for _, _, f, _ in dom)
     achieved = conv_flop / (conv_ms * 1e-3) / 1e12
+    all_ms = sum(ms for _, ms, _, _ in layers)
+    all_flop = sum(f for _, _, f, _ in layers)
     peak = pk["bf16_tflops"]
     per_layer = {f"conv{l}": {"ms": round(ms, 4), "tflops": round(f / (ms * 1e-3) / 1e12, 1), "path": path}
                  for l, ms, f, path in layers}
+    # dram__bytes_read+write of one launch of this kernel on layer 6 (56x56, 256->256), captured with
+    # ncu at batch 48 (107.3 MB) and scaled by the pixel count to the batch-100 launch timed here
+    traffic = 107.35e6 * BATCH / 48
 
     n_fwd = pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_FORWARD)
     cpu_rate, cpu_dt = oracle_forward_rate(args.cpu_images)
@@ -307,9 +314,14 @@ def run_native(args):
                     "ms_per_step": bwd_ms / bwd_steps,
                     "launches_per_step": pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_BACKWARD)},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "traffic": None,
-                     "kernel": "3x3 convolution forward (implicit GEMM), layers 2..16, flop-weighted",
+                     "frac": achieved / peak, "traffic": traffic,
+                     "kernel": "conv3x3_tc_kernel<256>: 3x3 convolution forward as a tcgen05 implicit GEMM, "
+                               "layers 5..16 (12 launches per pass), algorithmic flops / summed launch time",
+                     "traffic_note": "DRAM bytes of the layer-6 launch (algorithmic: 160.6 MB in + 160.6 MB out "
+                                     "+ 1.2 MB filter at batch 100); the output is still in L2 when the launch ends",
                      "peak_source": f"{pk['source']} burst bf16 GEMM (kernel timed alone per layer)",
+                     "all_conv_layers_2_16": {"tflops": all_flop / (all_ms * 1e-3) / 1e12,
+                                              "frac": all_flop / (all_ms * 1e-3) / 1e12 / peak},
                      "per_layer": per_layer},
         "cpu_baseline": {"value": cpu_rate, "unit": "images/s", "cores": os.cpu_count(), "kind": "oracle",
                          "sample": f"forward of {args.cpu_images} of the 100 images, {cpu_dt:.1f} s"},
