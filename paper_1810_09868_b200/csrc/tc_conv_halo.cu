@@ -171,12 +171,11 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             const uint32_t sb = b_base + bslot * T::B_BYTES;
             const int r = tap / 3, s = tap - r * 3;
             const uint32_t a_tap = sa + (uint32_t)(r * IW + s) * 128u;
+            const uint64_t da = smem_desc_sw128_sbo(a_tap, IW * 128), db = smem_desc_sw128(sb, 16);
+            umma_bf16(d_tmem, da, db, idesc, (cb | tap) != 0 ? 1u : 0u);
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k) {
-              const uint64_t da = smem_desc_sw128_sbo(a_tap + k * 32, IW * 128);
-              const uint64_t db = smem_desc_sw128(sb + k * 32, 16);
-              umma_bf16(d_tmem, da, db, idesc, (cb | tap | k) != 0 ? 1u : 0u);
-            }
+            for (int k = 1; k < BK / 16; ++k)
+              umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
             umma_commit(b_empty(bslot));
             if (++bslot == T::NB) { bslot = 0; bphase ^= 1; }
           }

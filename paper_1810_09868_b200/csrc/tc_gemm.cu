@@ -159,16 +159,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!mbar_wait(full_bar(stage), phase, &abort_flag, g.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
         tc_fence_after();
         const uint32_t sa = smem_base + stage * STAGE, sb = sa + A_BYTES;
+        // K-major: 16 k = 32 bytes along the swizzled row.  MN-major: 16 k = 16 rows = 2048 bytes.
+        // 8-channel form: 16 k = 16 rows of 16 bytes; 8-row groups 128 bytes apart, taps 1024 bytes apart.
+        constexpr uint32_t a_step = AMODE == kKMajor ? 32 : 2048;
+        constexpr uint32_t b_step = BMODE == kKMajor ? 32 : (BMODE == kMnMajorIm2colC8 ? 256 : 2048);
+        const uint64_t da = AMODE == kKMajor ? smem_desc_sw128(sa, 16) : smem_desc_sw128(sa, GROUP_BYTES);
+        const uint64_t db = BMODE == kKMajor          ? smem_desc_sw128(sb, 16)
+                            : BMODE == kMnMajorIm2colC8 ? smem_desc_plain(sb, 128, 1024)
+                                                        : smem_desc_sw128(sb, GROUP_BYTES);
+        umma_bf16(tmem_base, da, db, idesc, kb > kb0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 0; k < BK / 16; ++k) {
-          // K-major: 16 k = 32 bytes along the swizzled row.  MN-major: 16 k = 16 rows = 2048 bytes.
-          const uint64_t da = AMODE == kKMajor ? smem_desc_sw128(sa + k * 32, 16) : smem_desc_sw128(sa + k * 2048, GROUP_BYTES);
-          // 8-channel form: 16 k = 16 rows of 16 bytes; 8-row groups 128 bytes apart, taps 1024 bytes apart
-          const uint64_t db = BMODE == kKMajor          ? smem_desc_sw128(sb + k * 32, 16)
-                              : BMODE == kMnMajorIm2colC8 ? smem_desc_plain(sb + k * 256, 128, 1024)
-                                                          : smem_desc_sw128(sb + k * 2048, GROUP_BYTES);
-          umma_bf16(tmem_base, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-        }
+        for (int k = 1; k < BK / 16; ++k)
+          umma_bf16_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), idesc);
         umma_commit(empty_bar(stage));
         if (++stage == g.stages) { stage = 0; phase ^= 1; }
       }

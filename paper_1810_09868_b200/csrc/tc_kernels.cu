@@ -252,12 +252,13 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           if (!mbar_wait(full_bar(stage), phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
+          // the issue loop is the critical path of the tensor pipe: one descriptor pair per stage,
+          // advanced by 32 bytes (16 K elements) with a single add per MMA
+          const uint64_t da = smem_desc_sw128(sa, 16), db = smem_desc_sw128(sb, 16);
+          umma_bf16(d_tmem, da, db, idesc, kb != 0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            const uint64_t da = smem_desc_sw128(sa + k * 32, 16);
-            const uint64_t db = smem_desc_sw128(sb + k * 32, 16);
-            umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
-          }
+          for (int k = 1; k < BK / 16; ++k)
+            umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
           umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
           if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
         }
