@@ -101,6 +101,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      // im2col forms: each 64-column group of the tile is (tap, 64 channels), fixed for the CTA; the
+      // pixel a K block starts at advances by 64 per block (no divisions in the loop)
+      int grp_c[BN / 64 > 0 ? BN / 64 : 1], grp_s[BN / 64 > 0 ? BN / 64 : 1], grp_r[BN / 64 > 0 ? BN / 64 : 1];
+      int w0 = 0, h0 = 0, img = 0;
+      if (BMODE == kMnMajorIm2col || BMODE == kMnMajorIm2colC8) {
+        if (BMODE == kMnMajorIm2col) {
+#pragma unroll
+          for (int q = 0; q < BN / 64; ++q) {
+            const int j = n0 + 64 * q, tap = j / g.Cin;
+            grp_c[q] = j - tap * g.Cin; grp_r[q] = tap / 3; grp_s[q] = tap - 3 * (tap / 3);
+          }
+        }
+        const long p0 = (long)kb0 * BK;
+        w0 = (int)(p0 % g.W);
+        const long t = p0 / g.W;
+        h0 = (int)(t % g.H); img = (int)(t / g.H);
+      }
       for (int kb = kb0; kb < kb1; ++kb) {
         if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, g.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
         const uint32_t sa = smem_base + stage * STAGE, sb = sa + A_BYTES;
@@ -117,26 +134,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
           for (int q = 0; q < BN / 64; ++q) tma_load_2d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), n0 + 64 * q, kb * BK);
         } else if (BMODE == kMnMajorIm2col) {
-          const int p0 = kb * BK;
-          const int w0 = p0 % g.W, t = p0 / g.W;
-          const int h0 = t % g.H, img = t / g.H;
 #pragma unroll
-          for (int q = 0; q < BN / 64; ++q) {
-            // each 64-column group of the tile is (tap, 64 channels); groups of one tile may be different taps
-            const int j = n0 + 64 * q, tap = j / g.Cin, c0 = j - tap * g.Cin;
-            tma_load_im2col_4d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), c0, w0 - 1, h0 - 1, img,
-                               (uint16_t)(tap % 3), (uint16_t)(tap / 3));
-          }
+          for (int q = 0; q < BN / 64; ++q)
+            tma_load_im2col_4d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), grp_c[q], w0 - 1, h0 - 1, img,
+                               (uint16_t)grp_s[q], (uint16_t)grp_r[q]);
         } else {
           // nine taps of the 8-channel image, 64 pixels x 16 bytes each; the tenth slot (columns
           // 72..79 of the tile, never stored) is left as it is
-          const int p0 = kb * BK;
-          const int w0 = p0 % g.W, t = p0 / g.W;
-          const int h0 = t % g.H, img = t / g.H;
 #pragma unroll
           for (int tap = 0; tap < 9; ++tap)
             tma_load_im2col_4d(sb + tap * 1024, &map_b, full_bar(stage), 0, w0 - 1, h0 - 1, img, (uint16_t)(tap % 3),
                                (uint16_t)(tap / 3));
+        }
+        if (BMODE == kMnMajorIm2col || BMODE == kMnMajorIm2colC8) {
+          w0 += BK;
+          while (w0 >= g.W) { w0 -= g.W; if (++h0 == g.H) { h0 = 0; ++img; } }
         }
         ++fills[stage];
         if (++stage == g.stages) { stage = 0; phase ^= 1; }

@@ -210,20 +210,21 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           const int t = p0 / a.W;
           h0 = t % a.H; n0 = t / a.H;
         }
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          const int rs = kb / a.cin_blocks, cb = kb - rs * a.cin_blocks;
-          const int r = rs / 3, s = rs - r * 3;
-          if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
-          const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
-          mbar_expect_tx(full_bar(stage), T::STAGE_BYTES);
-          if (a.patch)
-            tma_load_4d(sa, &map_x, full_bar(stage), cb * BK, w0 + s - 1, h0 + r - 1, n0);
-          else
-            tma_load_im2col_4d(sa, &map_x, full_bar(stage), cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
-          tma_load_2d(sb, &map_w, full_bar(stage), kb * BK, n_tile * BN);
-          ++fills[stage];
-          if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
-        }
+        int kb = 0;
+        for (int r = 0; r < 3 && ok; ++r)
+          for (int s = 0; s < 3 && ok; ++s)
+            for (int cb = 0; cb < a.cin_blocks; ++cb, ++kb) {
+              if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
+              const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
+              mbar_expect_tx(full_bar(stage), T::STAGE_BYTES);
+              if (a.patch)
+                tma_load_4d(sa, &map_x, full_bar(stage), cb * BK, w0 + s - 1, h0 + r - 1, n0);
+              else
+                tma_load_im2col_4d(sa, &map_x, full_bar(stage), cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
+              tma_load_2d(sb, &map_w, full_bar(stage), kb * BK, n_tile * BN);
+              ++fills[stage];
+              if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
+            }
       }
       if (!ok) {
         // let every copy already in flight land before the CTA may exit
