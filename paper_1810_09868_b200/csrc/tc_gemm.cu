@@ -299,9 +299,10 @@ int sm_count() {
   return sms;
 }
 
-// K split: aim at about two CTAs per SM in total, never an empty split.
+// K split: as many CTAs as fit in one wave (one CTA per SM: a second, partial wave would leave most
+// SMs idle for its whole duration), never an empty split.
 void plan_split(int mn_tiles, int k_blocks, int* splits, int* kb_per_split) {
-  int want = (2 * sm_count() + mn_tiles - 1) / mn_tiles;
+  int want = sm_count() / mn_tiles;
   if (want < 1) want = 1;
   if (want > k_blocks) want = k_blocks;
   int per = (k_blocks + want - 1) / want;
