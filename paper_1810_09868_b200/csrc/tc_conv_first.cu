@@ -10,8 +10,10 @@
 // The layer is bound by writing its output (128 bytes per pixel), not by math.
 //
 // Roles and pipeline are those of the general convolution kernel: warp 0 TMA
-// producer, warp 1 MMA issuer and TMEM owner, warps 2-5 epilogue; double-buffered
-// accumulator; persistent CTAs; time-limited waits.
+// producer, warp 1 MMA issuer and TMEM owner, then epilogue warps; double-buffered
+// accumulator; persistent CTAs; time-limited waits.  The main loop is five MMAs
+// per tile, so the epilogue sets the pace: eight epilogue warps, two per TMEM lane
+// quarter, each converting and storing 32 of the 64 output channels of its rows.
 #include "tc_common.cuh"
 #include "tc_kernels.cuh"
 
@@ -27,7 +29,7 @@ constexpr int STAGES = 8;
 constexpr int W_TAP_BYTES = BN * 16;      // 64 output channels x 8 channels
 constexpr int W_BYTES = 10 * W_TAP_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + W_BYTES + 1024 + 256;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;  // producer, MMA issuer, eight epilogue warps (two per TMEM lane quarter)
 
 struct FirstArgs {
   int pixels, H, W, m_tiles, relu;
@@ -67,7 +69,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 128); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 256); }
     mbar_init(w_bar, 1);
     mbar_init(drain_bar, 1);
     mbar_fence_init();
@@ -164,8 +166,8 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       const long pixel = (long)tile * BM + row;
       const bool valid = pixel < a.pixels;
       bf16* out_row = a.out + pixel * BN;
-#pragma unroll
-      for (int cc = 0; cc < BN; cc += 32) {
+      {
+        const int cc = ((warp - 2) >> 2) * 32;  // warps 2-5 take channels 0..31, warps 6-9 channels 32..63
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
         tmem_ld_wait();
