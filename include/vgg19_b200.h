@@ -151,7 +151,9 @@ int vgg19_conv_layer_backward(vgg19_t *net, int32_t layer, const void *x, const 
  * index 0..15: output of conv layer index+1 after bias and ReLU,
  * [batch][h][w][Cout]; 16..20: outputs of the five max-pools; 21, 22: outputs
  * of dense layers 1 and 2 after ReLU, [batch][4096] (dims[2] = dims[3] = 1).
- * Element type is the config's dtype. */
+ * Element type is the config's dtype.  A forward-only pass does not write the
+ * pre-pool output of a layer whose max-pool is fused into the convolution
+ * (layers 2 and 4 at 224x224); a backward pass stores everything. */
 int vgg19_saved_tensor(const vgg19_t *net, int32_t batch, int32_t mode, int32_t index,
                        size_t *offset_bytes, int64_t dims[4]);
 

@@ -47,7 +47,8 @@ struct HaloArgs {
   int relu;
   const float* bias;
   const bf16* mask;
-  bf16* out;
+  bf16* out;     // full-resolution output, or null when only the pooled output is wanted
+  bf16* pooled;  // 2x2 max-pooled output [N][H/2][W/2][Cout], or null
   int* dev_error;
 };
 
@@ -204,17 +205,22 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       tc_fence_after();
       const int tw = m_tile % a.tiles_w, t = m_tile / a.tiles_w;
       const int h = (t % a.tiles_h) * PH + row / PW, img = t / a.tiles_h;
-      const bool valid = h < a.H;
-      const long pixel = ((long)img * a.H + h) * a.W + tw * PW + row % PW;
+      const int w = tw * PW + row % PW;
+      const long pixel = ((long)img * a.H + h) * a.W + w;  // always inside the image: H % 16 == 0, W % 8 == 0
       const int c_base = n_tile * BN;
-      bf16* out_row = a.out + pixel * a.Cout + c_base;
+      bf16* out_row = a.out ? a.out + pixel * a.Cout + c_base : nullptr;
+      // 2x2 pooling: a warp holds four patch rows of eight pixels (lane = 8 * row + column), so every
+      // window lies inside one warp; the lane of the window's top-left pixel stores the maximum
+      const bool pool_lane = (lane & 1) == 0 && (lane & 8) == 0;
+      bf16* pool_row = a.pooled ? a.pooled + (((long)img * (a.H / 2) + h / 2) * (a.W / 2) + w / 2) * a.Cout + c_base
+                                : nullptr;
       const bf16* mask_row = a.mask ? a.mask + pixel * a.Cout + c_base : nullptr;
 #pragma unroll 1
       for (int cc = 0; cc < BN; cc += 32) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
         tmem_ld_wait();
-        if (valid) {
+        {
           uint32_t packed[16];
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
@@ -240,10 +246,30 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
               }
             }
           }
-          uint4* op = reinterpret_cast<uint4*>(out_row + cc);
+          if (out_row) {
+            uint4* op = reinterpret_cast<uint4*>(out_row + cc);
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+            for (int q = 0; q < 4; ++q)
+              op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+          }
+          if (a.pooled) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              __nv_bfloat162 m = *reinterpret_cast<__nv_bfloat162*>(&packed[i]);
+              uint32_t o = __shfl_down_sync(0xffffffffu, packed[i], 1);
+              m = __hmax2(m, *reinterpret_cast<__nv_bfloat162*>(&o));
+              uint32_t mb = *reinterpret_cast<uint32_t*>(&m);
+              o = __shfl_down_sync(0xffffffffu, mb, 8);
+              m = __hmax2(m, *reinterpret_cast<__nv_bfloat162*>(&o));
+              packed[i] = *reinterpret_cast<uint32_t*>(&m);
+            }
+            if (pool_lane) {
+              uint4* pp = reinterpret_cast<uint4*>(pool_row + cc);
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                pp[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+            }
+          }
         }
       }
       tc_fence_before();
@@ -284,8 +310,9 @@ bool tc_conv3x3_halo_supported(ConvShape s) {
          (long)s.N * s.H * s.W < (1L << 31) - 256;
 }
 
-cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out, ConvShape s,
-                            bool relu, int* dev_error, cudaStream_t st) {
+cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out,
+                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st) {
+  if (!out && !pooled) return cudaErrorInvalidValue;
   if (!tc_conv3x3_halo_supported(s)) return cudaErrorInvalidValue;
   const int BN = s.Cout % 128 == 0 ? 128 : 64;
   CUtensorMap mx, mw;
@@ -297,7 +324,7 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, c
   a.tiles_w = s.W / PW; a.tiles_h = s.H / PH;
   a.m_tiles = s.N * a.tiles_w * a.tiles_h;
   a.n_tiles = s.Cout / BN;
-  a.relu = relu ? 1 : 0; a.bias = bias; a.mask = mask; a.out = out; a.dev_error = dev_error;
+  a.relu = relu ? 1 : 0; a.bias = bias; a.mask = mask; a.out = out; a.pooled = pooled; a.dev_error = dev_error;
   return BN == 128 ? launch_halo<128>(mx, mw, a, st) : launch_halo<64>(mx, mw, a, st);
 }
 

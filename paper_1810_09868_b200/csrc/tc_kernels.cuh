@@ -20,8 +20,9 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
 // The same convolution with the input patch (plus halo) kept in shared memory
 // for all nine taps (tc_conv_halo.cu): the large-image, few-channel layers.
 bool tc_conv3x3_halo_supported(ConvShape s);
+// `pooled` (or null) also receives the 2x2 max-pool of the result; `out` may then be null.
 cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out,
-                            ConvShape s, bool relu, int* dev_error, cudaStream_t st);
+                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
 
 // Filter gradient of the same convolution as a GEMM with M = Cout, N = 9*Cin,
 // K = pixels (both operands read transposed, x through the im2col window):

@@ -191,6 +191,7 @@ struct Pass {
   cudaStream_t st;
   int launches = 0;
   cudaError_t err = cudaSuccess;
+  bool keep_activations = true;  // false in a forward-only pass: nothing will read a pre-pool output again
 
   T *buf(size_t off) const { return reinterpret_cast<T *>(static_cast<char *>(n->ws) + off); }
   float *fbuf(size_t off) const { return reinterpret_cast<float *>(static_cast<char *>(n->ws) + off); }
@@ -203,17 +204,19 @@ struct Pass {
     return l == 0 && n->use_tc && p.valid && tc_first_conv_supported(s);
   }
 
-  // y = relu(conv(x) + b), optionally pooled
-  void conv_forward(int l, const T *x, int B, T *y, T *pooled) {
+  // y = relu(conv(x) + b), optionally pooled.  With need_y false the full-resolution output may be
+  // left unwritten when the pool is fused into the convolution's epilogue.
+  void conv_forward(int l, const T *x, int B, T *y, T *pooled, bool need_y = true) {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
     if (first_tc_ok(l, s)) {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       ok(tc_first_conv((const bf16 *)buf(p.x8), n->w8, n->params + c.b_off, (bf16 *)y, s, true, n->dev_error, st), 1);
-    } else if (n->use_tc && tc_conv3x3_halo_supported(s))
-      ok(tc_conv3x3_halo((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr, (bf16 *)y, s, true,
-                         n->dev_error, st), 1);
-    else if (tc_conv_ok(s))
+    } else if (n->use_tc && tc_conv3x3_halo_supported(s)) {
+      ok(tc_conv3x3_halo((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
+                         (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st), 1);
+      return;
+    } else if (tc_conv_ok(s))
       ok(tc_conv3x3((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
                     (bf16 *)y, s, true, n->dev_error, st), 1);
     else
@@ -240,8 +243,8 @@ struct Pass {
       ConvShape t{B, c.H, c.W, c.Cout, c.Cin};  // a 3x3 correlation from Cout to Cin channels
       const T *wr = static_cast<const T *>(n->dgrad_w) + c.dgrad_off;
       if (n->use_tc && tc_conv3x3_halo_supported(t))
-        ok(tc_conv3x3_halo((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx, t, false,
-                           n->dev_error, st), 1);
+        ok(tc_conv3x3_halo((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr, t,
+                           false, n->dev_error, st), 1);
       else if (tc_conv_ok(t))
         ok(tc_conv3x3((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
                       t, false, n->dev_error, st), 1);
@@ -280,7 +283,7 @@ struct Pass {
     for (int l = 0; l < kConvLayers; ++l) {
       T *y = buf(p.act[l]);
       T *pooled = n->conv[l].pool_after ? buf(p.pooled[pi++]) : nullptr;
-      conv_forward(l, x, B, y, pooled);
+      conv_forward(l, x, B, y, pooled, keep_activations);
       x = pooled ? pooled : y;
     }
     float *logits = a.logits ? a.logits : fbuf(p.logits);
@@ -347,7 +350,7 @@ int check_batch(vgg19 *n, int batch, int mode, size_t extra) {
 template <typename T>
 int enqueue(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st, int *launches) {
   Pass<T> pass{n, make_plan(n, a.batch, mode), st};
-  if (mode == VGG19_MODE_FORWARD) pass.forward(a); else pass.backward(a);
+  if (mode == VGG19_MODE_FORWARD) { pass.keep_activations = false; pass.forward(a); } else pass.backward(a);
   if (launches) *launches = pass.launches;
   n->launches[mode] = pass.launches;
   if (pass.err != cudaSuccess)
