@@ -239,6 +239,8 @@ bool make_tiled_map_2d_c8(CUtensorMap* map, const void* base, uint64_t rows, uin
 bool make_patch_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, uint32_t box_w, uint32_t box_h);
 // NHWC bf16 tensor read through a 3x3 / pad 1 window: box = `pixels` x 64 channels, 128 B swizzle.
 bool make_im2col_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, uint32_t pixels);
+// NHWC bf16 tensor with 8 channels, tiled box of box_h x box_w pixels x 8 channels, no swizzle.
+bool make_patch_map_c8(CUtensorMap* map, const void* base, int N, int H, int W, uint32_t box_w, uint32_t box_h);
 // Same for a tensor with 8 channels: box = `pixels` x 8 channels (16 bytes), no swizzle.
 bool make_im2col_map_c8(CUtensorMap* map, const void* base, int N, int H, int W, uint32_t pixels);
 

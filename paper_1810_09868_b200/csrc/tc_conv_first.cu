@@ -7,6 +7,11 @@
 // multiple of the MMA depth 16).  One K step of an MMA is two taps: each tap is
 // its own TMA im2col box of 128 pixels x 8 channels (16-byte rows, no swizzle),
 // i.e. exactly the 8x16-byte core-matrix layout tcgen05 reads without swizzle.
+// Where the image is a whole number of 8 x 16 pixel patches, a tile is such a
+// patch and its 10 x 18 input patch (with halo) arrives as ONE tiled box of 180
+// 16-byte rows instead of nine boxes of 128; tap (r, s) then starts r*10 + s
+// rows into that buffer, 8-row groups are 10 rows apart, and the two taps of a
+// K step are 1 row (or, across a row change, 8 rows) apart.
 // The layer is bound by writing its output (128 bytes per pixel), not by math.
 //
 // Roles and pipeline are those of the general convolution kernel: warp 0 TMA
@@ -31,8 +36,13 @@ constexpr int W_BYTES = 10 * W_TAP_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + W_BYTES + 1024 + 256;
 constexpr int kThreads = 320;  // producer, MMA issuer, eight epilogue warps (two per TMEM lane quarter)
 
+constexpr int PW = 8, PH = 16, IW = PW + 2, IH = PH + 2;  // patch mode: output patch and input patch with halo
+constexpr int PATCH_BYTES = IW * IH * 16;                 // 2880
+constexpr int PATCH_ROWS_READ = 184;                      // the padding tap reads up to row 181
+
 struct FirstArgs {
   int pixels, H, W, m_tiles, relu;
+  int patch, tiles_w, tiles_h;
   const float* bias;
   bf16* out;
   int* dev_error;
@@ -62,6 +72,11 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     for (int i = threadIdx.x; i < STAGES * (TAP_BYTES / 16); i += kThreads) {
       const int s = i / (TAP_BYTES / 16), q = i % (TAP_BYTES / 16);
       *reinterpret_cast<uint4*>(base + s * STAGE_BYTES + 9 * TAP_BYTES + q * 16) = make_uint4(0, 0, 0, 0);
+    }
+    // patch mode: rows 180..183 of every stage lie behind the copied patch and are read (times zero)
+    for (int i = threadIdx.x; i < STAGES * (PATCH_ROWS_READ - IW * IH); i += kThreads) {
+      const int s = i / (PATCH_ROWS_READ - IW * IH), q = i % (PATCH_ROWS_READ - IW * IH);
+      *reinterpret_cast<uint4*>(base + s * STAGE_BYTES + PATCH_BYTES + q * 16) = make_uint4(0, 0, 0, 0);
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -96,16 +111,22 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < a.m_tiles; tile += gridDim.x) {
-        const int p0 = tile * BM;
-        const int w0 = p0 % a.W, t = p0 / a.W;
-        const int h0 = t % a.H, n0 = t / a.H;
         if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
         const uint32_t sa = smem_base + stage * STAGE_BYTES;
-        mbar_expect_tx(full_bar(stage), 9 * TAP_BYTES);
+        if (a.patch) {
+          const int tw = tile % a.tiles_w, t = tile / a.tiles_w;
+          mbar_expect_tx(full_bar(stage), PATCH_BYTES);
+          tma_load_4d(sa, &map_x, full_bar(stage), 0, tw * PW - 1, (t % a.tiles_h) * PH - 1, t / a.tiles_h);
+        } else {
+          const int p0 = tile * BM;
+          const int w0 = p0 % a.W, t = p0 / a.W;
+          const int h0 = t % a.H, n0 = t / a.H;
+          mbar_expect_tx(full_bar(stage), 9 * TAP_BYTES);
 #pragma unroll
-        for (int tap = 0; tap < 9; ++tap)
-          tma_load_im2col_4d(sa + tap * TAP_BYTES, &map_x, full_bar(stage), 0, w0 - 1, h0 - 1, n0, (uint16_t)(tap % 3),
-                             (uint16_t)(tap / 3));
+          for (int tap = 0; tap < 9; ++tap)
+            tma_load_im2col_4d(sa + tap * TAP_BYTES, &map_x, full_bar(stage), 0, w0 - 1, h0 - 1, n0, (uint16_t)(tap % 3),
+                               (uint16_t)(tap / 3));
+        }
         ++fills[stage];
         if (++stage == STAGES) { stage = 0; phase ^= 1; }
       }
@@ -140,7 +161,11 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         for (int j = 0; j < 5; ++j) {
           // K step j = taps 2j and 2j+1: the two 8-element K chunks are one tap buffer apart,
           // 8-row groups are 128 bytes apart
-          const uint64_t da = smem_desc_plain(sa + 2 * j * TAP_BYTES, TAP_BYTES, 128);
+          // (patch mode: tap 2j starts (r*10 + s) rows in; the next tap is one row on, or eight when the
+          // pair straddles a filter row (j == 1: taps (0,2) and (1,0)); patch rows are 10 rows apart)
+          const int t0 = 2 * j, r0 = t0 / 3, s0 = t0 - 3 * r0;
+          const uint64_t da = a.patch ? smem_desc_plain(sa + (r0 * IW + s0) * 16, j == 1 ? (IW - 2) * 16 : 16, IW * 16)
+                                      : smem_desc_plain(sa + 2 * j * TAP_BYTES, TAP_BYTES, 128);
           const uint64_t db = smem_desc_plain(w_smem + 2 * j * W_TAP_BYTES, W_TAP_BYTES, 128);
           umma_bf16(tmem_base + (uint32_t)(buf * BN), da, db, idesc, j != 0 ? 1u : 0u);
         }
@@ -163,7 +188,13 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       const uint32_t use = (uint32_t)(local >> 1);
       if (!mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum)) break;
       tc_fence_after();
-      const long pixel = (long)tile * BM + row;
+      long pixel;
+      if (a.patch) {
+        const int tw = tile % a.tiles_w, t = tile / a.tiles_w;
+        pixel = ((long)(t / a.tiles_h) * a.H + (t % a.tiles_h) * PH + row / PW) * a.W + tw * PW + row % PW;
+      } else {
+        pixel = (long)tile * BM + row;
+      }
       const bool valid = pixel < a.pixels;
       bf16* out_row = a.out + pixel * BN;
       {
@@ -239,7 +270,12 @@ cudaError_t tc_first_conv(const bf16* x8, const bf16* w8, const float* bias, bf1
                           int* dev_error, cudaStream_t st) {
   if (!tc_first_conv_supported(s)) return cudaErrorInvalidValue;
   CUtensorMap mx, mw;
-  if (!make_im2col_map_c8(&mx, x8, s.N, s.H, s.W, BM)) return cudaErrorInvalidValue;
+  const bool patch = s.W % PW == 0 && s.H % PH == 0;
+  if (patch) {
+    if (!make_patch_map_c8(&mx, x8, s.N, s.H, s.W, IW, IH)) return cudaErrorInvalidValue;
+  } else if (!make_im2col_map_c8(&mx, x8, s.N, s.H, s.W, BM)) {
+    return cudaErrorInvalidValue;
+  }
   if (!make_tiled_map_2d_c8(&mw, w8, 64, 80, 64)) return cudaErrorInvalidValue;
   static bool configured = false;
   if (!configured) {
@@ -249,7 +285,9 @@ cudaError_t tc_first_conv(const bf16* x8, const bf16* w8, const float* bias, bf1
   }
   FirstArgs a;
   a.pixels = s.N * s.H * s.W; a.H = s.H; a.W = s.W;
-  a.m_tiles = (a.pixels + BM - 1) / BM;
+  a.patch = patch ? 1 : 0;
+  a.tiles_w = s.W / PW; a.tiles_h = s.H / PH;
+  a.m_tiles = patch ? s.N * a.tiles_w * a.tiles_h : (a.pixels + BM - 1) / BM;
   a.relu = relu ? 1 : 0; a.bias = bias; a.out = out; a.dev_error = dev_error;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);

@@ -84,6 +84,18 @@ bool make_patch_map(CUtensorMap* map, const void* base, int N, int H, int W, int
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_patch_map_c8(CUtensorMap* map, const void* base, int N, int H, int W, uint32_t box_w, uint32_t box_h) {
+  const TensorMapApi& api = tensor_map_api();
+  if (!api.ok) return false;
+  cuuint64_t dims[4] = {8, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+  cuuint64_t strides[3] = {16, (cuuint64_t)W * 16, (cuuint64_t)H * W * 16};
+  cuuint32_t box[4] = {8, box_w, box_h, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return api.encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_im2col_map_c8(CUtensorMap* map, const void* base, int N, int H, int W, uint32_t pixels) {
   const TensorMapApi& api = tensor_map_api();
   if (!api.ok) return false;
