@@ -33,7 +33,8 @@ constexpr int STAGE_BYTES = 10 * TAP_BYTES;
 constexpr int STAGES = 8;
 constexpr int W_TAP_BYTES = BN * 16;      // 64 output channels x 8 channels
 constexpr int W_BYTES = 10 * W_TAP_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + W_BYTES + 1024 + 256;
+constexpr int OUT_TILE_BYTES = BM * BN * 2;  // 16 KB staging tile for the TMA store, two of them
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_TILE_BYTES + W_BYTES + 1024 + 256;
 constexpr int kThreads = 320;  // producer, MMA issuer, eight epilogue warps (two per TMEM lane quarter)
 
 constexpr int PW = 8, PH = 16, IW = PW + 2, IH = PH + 2;  // patch mode: output patch and input patch with halo
@@ -49,10 +50,12 @@ struct FirstArgs {
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
-conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, FirstArgs a) {
+conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                     const __grid_constant__ CUtensorMap map_y, FirstArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t w_smem = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t out_smem = smem_base + STAGES * STAGE_BYTES;  // 1024-byte aligned (20 KB stages)
+  const uint32_t w_smem = out_smem + 2 * OUT_TILE_BYTES;
   const uint32_t bars = w_smem + W_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
@@ -186,33 +189,48 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     for (int tile = blockIdx.x; tile < a.m_tiles; tile += gridDim.x, ++local) {
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
-      if (!mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum)) break;
+      const bool got = mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
+      // the store that last used this tile's staging buffer must have read it before anyone refills it;
+      // the barrier doubles as the vote that lets all eight warps leave together if any wait failed
+      if (threadIdx.x == 64) tma_store_wait_read<1>();
+      if (named_bar_or(1, 256, !got)) break;
       tc_fence_after();
-      long pixel;
-      if (a.patch) {
-        const int tw = tile % a.tiles_w, t = tile / a.tiles_w;
-        pixel = ((long)(t / a.tiles_h) * a.H + (t % a.tiles_h) * PH + row / PW) * a.W + tw * PW + row % PW;
-      } else {
-        pixel = (long)tile * BM + row;
-      }
-      const bool valid = pixel < a.pixels;
-      bf16* out_row = a.out + pixel * BN;
-      {
-        const int cc = ((warp - 2) >> 2) * 32;  // warps 2-5 take channels 0..31, warps 6-9 channels 32..63
-        uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
-        tmem_ld_wait();
-        if (valid) {
-          uint32_t packed[16];
+      const int cc = ((warp - 2) >> 2) * 32;  // warps 2-5 take channels 0..31, warps 6-9 channels 32..63
+      uint32_t v[32];
+      tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+      tmem_ld_wait();
+      uint32_t packed[16];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
-            x0 += bias_s[cc + j]; x1 += bias_s[cc + j + 1];
-            if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
-            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
-            packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
-          }
-          uint4* op = reinterpret_cast<uint4*>(out_row + cc);
+      for (int j = 0; j < 32; j += 2) {
+        float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
+        x0 += bias_s[cc + j]; x1 += bias_s[cc + j + 1];
+        if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
+        __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+        packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      if (a.patch) {
+        // the tile leaves through shared memory and one TMA store (whole 128-byte lines) instead of
+        // 256 threads writing 64-byte pieces of their own rows; two staging tiles alternate
+        const uint32_t stage_out = out_smem + (uint32_t)(local & 1) * OUT_TILE_BYTES;
+        const bool issuer = threadIdx.x == 64;  // first epilogue thread owns the store groups
+        uint8_t* dst = smem_raw + (stage_out - smem_u32(smem_raw)) + row * 128;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int chunk = (cc >> 3) + q;  // 16-byte chunk of the 128-byte row, 128-byte swizzled
+          *reinterpret_cast<uint4*>(dst + ((chunk ^ (row & 7)) << 4)) =
+              make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+        }
+        fence_async_smem();
+        named_bar_sync(1, 256);
+        if (issuer) {
+          const int tw = tile % a.tiles_w, t = tile / a.tiles_w;
+          tma_store_4d(&map_y, stage_out, 0, tw * PW, (t % a.tiles_h) * PH, t / a.tiles_h);
+          tma_store_commit();
+        }
+      } else {
+        const long pixel = (long)tile * BM + row;
+        if (pixel < a.pixels) {
+          uint4* op = reinterpret_cast<uint4*>(a.out + pixel * BN + cc);
 #pragma unroll
           for (int q = 0; q < 4; ++q)
             op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
@@ -221,6 +239,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       tc_fence_before();
       mbar_arrive(acc_empty_bar(buf));
     }
+    if (threadIdx.x == 64) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }
 
   tc_fence_before();
@@ -277,6 +296,8 @@ cudaError_t tc_first_conv(const bf16* x8, const bf16* w8, const float* bias, bf1
     return cudaErrorInvalidValue;
   }
   if (!make_tiled_map_2d_c8(&mw, w8, 64, 80, 64)) return cudaErrorInvalidValue;
+  CUtensorMap my = mw;  // only read in patch mode
+  if (patch && !make_patch_map(&my, out, s.N, s.H, s.W, 64, PW, PH)) return cudaErrorInvalidValue;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(conv3x3_c8_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
@@ -293,7 +314,7 @@ cudaError_t tc_first_conv(const bf16* x8, const bf16* w8, const float* bias, bf1
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int grid = a.m_tiles < sms ? a.m_tiles : sms;
-  conv3x3_c8_tc_kernel<<<grid, kThreads, SMEM_BYTES, st>>>(mx, mw, a);
+  conv3x3_c8_tc_kernel<<<grid, kThreads, SMEM_BYTES, st>>>(mx, mw, my, a);
   return cudaGetLastError();
 }
 
