@@ -139,9 +139,11 @@ template <int BN>
 struct ConvTile {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (kSmemLimit - 4608) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608) / STAGE_BYTES;  // leaves room for barriers, bias and alignment
+  static constexpr int OUT_BYTES = BM * 64 * 2;  // staging tile of the TMA store: 128 rows x 64 channels
+  // leaves room for the staging tile, barriers, bias and alignment
+  static constexpr int STAGES = (kSmemLimit - 4608 - OUT_BYTES) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608 - OUT_BYTES) / STAGE_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;  // 128, 256 or 512: powers of two
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 struct ConvArgs {
@@ -163,12 +165,14 @@ constexpr int PW = 16, PH = 8;  // patch of a tile in patch mode (PW * PH = BM)
 
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
-conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, ConvArgs a) {
+conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                  const __grid_constant__ CUtensorMap map_y, ConvArgs a) {
   using T = ConvTile<BN>;
   extern __shared__ uint8_t smem_raw[];
   // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bars = smem_base + T::STAGES * T::STAGE_BYTES;
+  const uint32_t out_smem = smem_base + T::STAGES * T::STAGE_BYTES;  // 1024-byte aligned
+  const uint32_t bars = out_smem + T::OUT_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (T::STAGES + s); };
   auto acc_full_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + b); };
@@ -289,31 +293,40 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     const int quarter = warp & 3;  // the TMEM lane quarter this warp may read
     const int row = quarter * 32 + lane;
     int local = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+    // The tile leaves 64 channels at a time through a 128-byte-swizzled staging tile and one TMA
+    // store (whole 128-byte lines), not as per-thread pieces of rows.  Thread 64 owns the store groups.
+    const bool issuer = threadIdx.x == 64;
+    uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
       const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
-      if (!mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum)) { ok = false; break; }
+      const bool got = mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
+      if (named_bar_or(1, 128, !got)) break;  // all four warps leave together
       tc_fence_after();
       long pixel;
+      int tw = 0, th = 0, img = 0;
       if (a.patch) {
-        const int tw = m_tile % a.tiles_w, t = m_tile / a.tiles_w;
-        const int th = t % a.tiles_h, img = t / a.tiles_h;
+        tw = m_tile % a.tiles_w;
+        const int t = m_tile / a.tiles_w;
+        th = t % a.tiles_h; img = t / a.tiles_h;
         pixel = ((long)img * a.H + th * PH + row / PW) * a.W + tw * PW + row % PW;
       } else {
         pixel = (long)m_tile * BM + row;
       }
       const bool valid = pixel < a.pixels;
       const int c_base = n_tile * BN;
-      bf16* out_row = a.out + pixel * a.Cout + c_base;
-      const bf16* mask_row = a.mask ? a.mask + pixel * a.Cout + c_base : nullptr;
+      const bf16* mask_row = (a.mask && valid) ? a.mask + pixel * a.Cout + c_base : nullptr;
 #pragma unroll 1
-      for (int cc = 0; cc < BN; cc += 32) {
-        uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
-        tmem_ld_wait();
-        if (valid) {
+      for (int c64 = 0; c64 < BN; c64 += 64) {
+        if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
+        named_bar_sync(1, 128);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int cc = c64 + half * 32;
+          uint32_t v[32];
+          tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+          tmem_ld_wait();
           uint32_t packed[16];
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
@@ -340,15 +353,26 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
               }
             }
           }
-          uint4* op = reinterpret_cast<uint4*>(out_row + cc);
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+          for (int q = 0; q < 4; ++q) {
+            const int chunk = half * 4 + q;  // 16-byte chunk of the 128-byte staging row
+            *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) =
+                make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+          }
+        }
+        fence_async_smem();
+        named_bar_sync(1, 128);
+        if (issuer) {
+          // rows past the end of the tensor (last tile) are clipped by the copy engine
+          if (a.patch) tma_store_4d(&map_y, out_smem, c_base + c64, tw * PW, th * PH, img);
+          else tma_store_2d(&map_y, out_smem, c_base + c64, m_tile * BM);
+          tma_store_commit();
         }
       }
       tc_fence_before();
       mbar_arrive(acc_empty_bar(buf));
     }
+    if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }
 
   tc_fence_before();
@@ -361,7 +385,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 }
 
 template <int BN>
-cudaError_t launch_conv(const CUtensorMap& mx, const CUtensorMap& mw, ConvArgs a, cudaStream_t st) {
+cudaError_t launch_conv(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, ConvArgs a,
+                        cudaStream_t st) {
   using T = ConvTile<BN>;
   static bool configured = false;
   if (!configured) {
@@ -374,7 +399,7 @@ cudaError_t launch_conv(const CUtensorMap& mx, const CUtensorMap& mw, ConvArgs a
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int tiles = a.m_tiles * a.n_tiles;
   const int grid = tiles < sms ? tiles : sms;
-  conv3x3_tc_kernel<BN><<<grid, kThreads, T::SMEM_BYTES, st>>>(mx, mw, a);
+  conv3x3_tc_kernel<BN><<<grid, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
   return cudaGetLastError();
 }
 
@@ -399,6 +424,12 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
     return cudaErrorInvalidValue;
   }
   if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
+  CUtensorMap my;
+  if (patch) {
+    if (!make_patch_map(&my, out, s.N, s.H, s.W, s.Cout, PW, PH)) return cudaErrorInvalidValue;
+  } else if (!make_tiled_map_2d(&my, out, (uint64_t)s.N * s.H * s.W, (uint64_t)s.Cout, BM)) {
+    return cudaErrorInvalidValue;
+  }
   ConvArgs a;
   a.patch = patch ? 1 : 0;
   a.tiles_w = s.W / PW; a.tiles_h = s.H / PH;
@@ -411,9 +442,9 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
   a.relu = relu ? 1 : 0;
   a.bias = bias; a.mask = mask; a.out = out; a.dev_error = dev_error;
   switch (BN) {
-    case 256: return launch_conv<256>(mx, mw, a, st);
-    case 128: return launch_conv<128>(mx, mw, a, st);
-    default: return launch_conv<64>(mx, mw, a, st);
+    case 256: return launch_conv<256>(mx, mw, my, a, st);
+    case 128: return launch_conv<128>(mx, mw, my, a, st);
+    default: return launch_conv<64>(mx, mw, my, a, st);
   }
 }
 
