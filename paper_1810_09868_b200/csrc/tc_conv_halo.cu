@@ -36,8 +36,10 @@ constexpr int kThreads = 224;
 template <int BN>
 struct HaloTile {
   static constexpr int B_BYTES = BN * BK * 2;
-  static constexpr int NB = (227 * 1024 - 4608 - NA * A_SLOT) / B_BYTES > 12 ? 12 : (227 * 1024 - 4608 - NA * A_SLOT) / B_BYTES;
-  static constexpr int SMEM_BYTES = NA * A_SLOT + NB * B_BYTES + 1024 + 512;
+  static constexpr int OUT_BYTES = BM * 64 * 2;  // staging tile of the TMA store
+  static constexpr int kBudget = 227 * 1024 - 4608 - NA * A_SLOT - OUT_BYTES;
+  static constexpr int NB = kBudget / B_BYTES > 12 ? 12 : kBudget / B_BYTES;
+  static constexpr int SMEM_BYTES = NA * A_SLOT + NB * B_BYTES + OUT_BYTES + 1024 + 512;
 };
 
 struct HaloArgs {
@@ -54,12 +56,14 @@ struct HaloArgs {
 
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
-conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, HaloArgs a) {
+conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                       const __grid_constant__ CUtensorMap map_y, HaloArgs a) {
   using T = HaloTile<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_base = smem_base + NA * A_SLOT;
-  const uint32_t bars = b_base + T::NB * T::B_BYTES;
+  const uint32_t out_smem = b_base + T::NB * T::B_BYTES;  // 1024-byte aligned
+  const uint32_t bars = out_smem + T::OUT_BYTES;
   auto a_full = [&](int s) { return bars + 8u * s; };
   auto a_empty = [&](int s) { return bars + 8u * (NA + s); };
   auto b_full = [&](int s) { return bars + 8u * (2 * NA + s); };
@@ -197,18 +201,24 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     int local = 0;
+    // The full-resolution tile leaves 64 channels at a time through a 128-byte-swizzled staging tile
+    // and one TMA store; the pooled output (a quarter of it) is stored directly.  Thread 64 owns the
+    // store groups.
+    const bool issuer = threadIdx.x == 64;
+    uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
       const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
-      if (!mbar_wait(acc_full(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum)) break;
+      const bool got = mbar_wait(acc_full(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
+      if (named_bar_or(1, 128, !got)) break;  // all four warps leave together
       tc_fence_after();
       const int tw = m_tile % a.tiles_w, t = m_tile / a.tiles_w;
-      const int h = (t % a.tiles_h) * PH + row / PW, img = t / a.tiles_h;
+      const int th = t % a.tiles_h, img = t / a.tiles_h;
+      const int h = th * PH + row / PW;
       const int w = tw * PW + row % PW;
       const long pixel = ((long)img * a.H + h) * a.W + w;  // always inside the image: H % 16 == 0, W % 8 == 0
       const int c_base = n_tile * BN;
-      bf16* out_row = a.out ? a.out + pixel * a.Cout + c_base : nullptr;
       // 2x2 pooling: a warp holds four patch rows of eight pixels (lane = 8 * row + column), so every
       // window lies inside one warp; the lane of the window's top-left pixel stores the maximum
       const bool pool_lane = (lane & 1) == 0 && (lane & 8) == 0;
@@ -216,11 +226,17 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                                 : nullptr;
       const bf16* mask_row = a.mask ? a.mask + pixel * a.Cout + c_base : nullptr;
 #pragma unroll 1
-      for (int cc = 0; cc < BN; cc += 32) {
-        uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
-        tmem_ld_wait();
-        {
+      for (int c64 = 0; c64 < BN; c64 += 64) {
+        if (a.out) {
+          if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
+          named_bar_sync(1, 128);
+        }
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int cc = c64 + half * 32;
+          uint32_t v[32];
+          tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+          tmem_ld_wait();
           uint32_t packed[16];
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
@@ -246,11 +262,13 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
               }
             }
           }
-          if (out_row) {
-            uint4* op = reinterpret_cast<uint4*>(out_row + cc);
+          if (a.out) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-              op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+            for (int q = 0; q < 4; ++q) {
+              const int chunk = half * 4 + q;  // 16-byte chunk of the 128-byte staging row
+              *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) =
+                  make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+            }
           }
           if (a.pooled) {
 #pragma unroll
@@ -271,10 +289,19 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             }
           }
         }
+        if (a.out) {
+          fence_async_smem();
+          named_bar_sync(1, 128);
+          if (issuer) {
+            tma_store_4d(&map_y, out_smem, c_base + c64, tw * PW, th * PH, img);
+            tma_store_commit();
+          }
+        }
       }
       tc_fence_before();
       mbar_arrive(acc_empty(buf));
     }
+    if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }
 
   tc_fence_before();
@@ -287,7 +314,8 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 }
 
 template <int BN>
-cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, HaloArgs a, cudaStream_t st) {
+cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, HaloArgs a,
+                        cudaStream_t st) {
   using T = HaloTile<BN>;
   static bool configured = false;
   if (!configured) {
@@ -299,7 +327,7 @@ cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, HaloArgs a
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int tiles = a.m_tiles * a.n_tiles;
-  conv3x3_halo_tc_kernel<BN><<<tiles < sms ? tiles : sms, kThreads, T::SMEM_BYTES, st>>>(mx, mw, a);
+  conv3x3_halo_tc_kernel<BN><<<tiles < sms ? tiles : sms, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
   return cudaGetLastError();
 }
 
@@ -318,6 +346,8 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, c
   CUtensorMap mx, mw;
   if (!make_patch_map(&mx, in, s.N, s.H, s.W, s.Cin, IW, IH)) return cudaErrorInvalidValue;
   if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
+  CUtensorMap my = mw;  // only read when there is a full-resolution output
+  if (out && !make_patch_map(&my, out, s.N, s.H, s.W, s.Cout, PW, PH)) return cudaErrorInvalidValue;
   HaloArgs a;
   a.N = s.N; a.H = s.H; a.W = s.W;
   a.cin_blocks = s.Cin / 64; a.Cin = s.Cin; a.Cout = s.Cout;
@@ -325,7 +355,7 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, c
   a.m_tiles = s.N * a.tiles_w * a.tiles_h;
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0; a.bias = bias; a.mask = mask; a.out = out; a.pooled = pooled; a.dev_error = dev_error;
-  return BN == 128 ? launch_halo<128>(mx, mw, a, st) : launch_halo<64>(mx, mw, a, st);
+  return BN == 128 ? launch_halo<128>(mx, mw, my, a, st) : launch_halo<64>(mx, mw, my, a, st);
 }
 
 }  // namespace vgg
