@@ -81,6 +81,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
 // Tiled load of a [1][box_h][box_w][channels] box of an NHWC tensor; coordinates
 // outside the tensor (a halo of the padding) read as zero.
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w, int h,
@@ -271,6 +277,8 @@ const TensorMapApi& tensor_map_api();
 bool make_tiled_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 // Same with a box of box_rows x 8 columns (16 bytes) and no swizzle.
 bool make_tiled_map_2d_c8(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// Tap-major filter [9][Cout][Cin] bf16: box = 3 taps x box_cout rows x 64 channels, 128 B swizzle.
+bool make_filter_row_map(CUtensorMap* map, const void* base, int Cout, int Cin, uint32_t box_cout);
 // NHWC bf16 tensor, tiled box of box_h x box_w pixels x 64 channels, 128 B swizzle.
 bool make_patch_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, uint32_t box_w, uint32_t box_h);
 // NHWC bf16 tensor read through a 3x3 / pad 1 window: box = `pixels` x 64 channels, 128 B swizzle.

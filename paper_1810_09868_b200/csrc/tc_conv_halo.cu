@@ -13,7 +13,10 @@
 // consecutive rows, 10 rows apart: a K-major operand with a stride of
 // 1280 bytes between 8-row groups, starting (r * 10 + s) rows into the patch.
 // The nine taps are nine MMAs on the same buffer with different start rows.
-// Filter slices (BN x 64 per tap) stream through their own ring.
+// The filter is read from a tap-major copy [9][Cout][Cin], so that one TMA box
+// brings a whole filter row (three taps x BN x 64) into one slot of its own ring:
+// one barrier hand-off per twelve MMAs instead of per four (with four the
+// producer thread, not the tensor pipe, set the pace).
 //
 // Warps: 0 patch producer, 1 MMA issuer + TMEM owner, 2-5 epilogue, 6 filter
 // producer.  Accumulator double-buffered; persistent CTAs; time-limited waits.
@@ -30,15 +33,16 @@ constexpr int PW = 8, PH = 16;                  // output patch
 constexpr int IW = PW + 2, IH = PH + 2;         // input patch with halo
 constexpr int A_BYTES = IW * IH * 128;          // 23040
 constexpr int A_SLOT = 23 * 1024;               // 1024-byte aligned slot
-constexpr int NA = 3;
 constexpr int kThreads = 224;
 
 template <int BN>
 struct HaloTile {
-  static constexpr int B_BYTES = BN * BK * 2;
-  static constexpr int OUT_BYTES = BM * 64 * 2;  // staging tile of the TMA store
+  static constexpr int TAP_BYTES = BN * BK * 2;   // one tap's BN x 64 filter slice
+  static constexpr int B_BYTES = 3 * TAP_BYTES;   // a filter row: three taps
+  static constexpr int NA = BN <= 64 ? 3 : 2;     // input-patch slots
+  static constexpr int OUT_BYTES = BM * 64 * 2;   // staging tile of the TMA store
   static constexpr int kBudget = 227 * 1024 - 4608 - NA * A_SLOT - OUT_BYTES;
-  static constexpr int NB = kBudget / B_BYTES > 12 ? 12 : kBudget / B_BYTES;
+  static constexpr int NB = kBudget / B_BYTES > 4 ? 4 : kBudget / B_BYTES;
   static constexpr int SMEM_BYTES = NA * A_SLOT + NB * B_BYTES + OUT_BYTES + 1024 + 512;
 };
 
@@ -59,6 +63,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_y, HaloArgs a) {
   using T = HaloTile<BN>;
+  constexpr int NA = T::NA;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_base = smem_base + NA * A_SLOT;
@@ -138,10 +143,10 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int n_tile = tile % a.n_tiles;
         for (int cb = 0; cb < a.cin_blocks && ok; ++cb)
-          for (int tap = 0; tap < 9; ++tap) {
+          for (int r = 0; r < 3; ++r) {
             if (!mbar_wait(b_empty(slot), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
             mbar_expect_tx(b_full(slot), T::B_BYTES);
-            tma_load_2d(b_base + slot * T::B_BYTES, &map_w, b_full(slot), tap * a.Cin + cb * BK, n_tile * BN);
+            tma_load_3d(b_base + slot * T::B_BYTES, &map_w, b_full(slot), cb * BK, n_tile * BN, 3 * r);
             ++fills[slot];
             if (++slot == T::NB) { slot = 0; phase ^= 1; }
           }
@@ -170,17 +175,19 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         for (int cb = 0; cb < a.cin_blocks && ok; ++cb) {
           if (!mbar_wait(a_full(aslot), aphase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
           const uint32_t sa = smem_base + aslot * A_SLOT;
-          for (int tap = 0; tap < 9; ++tap) {
+          for (int r = 0; r < 3; ++r) {
             if (!mbar_wait(b_full(bslot), bphase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t sb = b_base + bslot * T::B_BYTES;
-            const int r = tap / 3, s = tap - r * 3;
-            const uint32_t a_tap = sa + (uint32_t)(r * IW + s) * 128u;
-            const uint64_t da = smem_desc_sw128_sbo(a_tap, IW * 128), db = smem_desc_sw128(sb, 16);
-            umma_bf16(d_tmem, da, db, idesc, (cb | tap) != 0 ? 1u : 0u);
 #pragma unroll
-            for (int k = 1; k < BK / 16; ++k)
-              umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
+            for (int s = 0; s < 3; ++s) {
+              const uint32_t sb = b_base + bslot * T::B_BYTES + s * T::TAP_BYTES;
+              const uint32_t a_tap = sa + (uint32_t)(r * IW + s) * 128u;
+              const uint64_t da = smem_desc_sw128_sbo(a_tap, IW * 128), db = smem_desc_sw128(sb, 16);
+              umma_bf16(d_tmem, da, db, idesc, (cb | r | s) != 0 ? 1u : 0u);
+#pragma unroll
+              for (int k = 1; k < BK / 16; ++k)
+                umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
+            }
             umma_commit(b_empty(bslot));
             if (++bslot == T::NB) { bslot = 0; bphase ^= 1; }
           }
@@ -333,19 +340,45 @@ cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
 
 }  // namespace
 
+namespace {
+// forward : out[tap][k][c] = w[k][tap][c]                       (rows k = Cout, columns c = Cin)
+// dgrad   : out[tap][c][k] = w[k][8 - tap][c]  (filter rotated by 180 degrees, channel roles exchanged:
+//           rows c = Cin, columns k = Cout)
+__global__ void tap_major_kernel(const float* __restrict__ w, bf16* __restrict__ out, int Cin, int Cout, int dgrad) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long total = 9L * Cin * Cout;
+  if (i >= total) return;
+  if (!dgrad) {
+    const int c = i % Cin; const long t = i / Cin;
+    const int k = t % Cout, tap = t / Cout;
+    out[i] = __float2bfloat16_rn(w[((long)k * 9 + tap) * Cin + c]);
+  } else {
+    const int k = i % Cout; const long t = i / Cout;
+    const int c = t % Cin, tap = t / Cin;
+    out[i] = __float2bfloat16_rn(w[((long)k * 9 + (8 - tap)) * Cin + c]);
+  }
+}
+}  // namespace
+
+cudaError_t tc_make_tap_major(const float* w, bf16* out, int Cin, int Cout, bool for_dgrad, cudaStream_t st) {
+  const long total = 9L * Cin * Cout;
+  tap_major_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w, out, Cin, Cout, for_dgrad ? 1 : 0);
+  return cudaGetLastError();
+}
+
 bool tc_conv3x3_halo_supported(ConvShape s) {
   return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.Cout <= 128 && s.W % PW == 0 && s.H % PH == 0 && s.W >= 64 &&
          (long)s.N * s.H * s.W < (1L << 31) - 256;
 }
 
-cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out,
+cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
                             bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st) {
   if (!out && !pooled) return cudaErrorInvalidValue;
   if (!tc_conv3x3_halo_supported(s)) return cudaErrorInvalidValue;
   const int BN = s.Cout % 128 == 0 ? 128 : 64;
   CUtensorMap mx, mw;
   if (!make_patch_map(&mx, in, s.N, s.H, s.W, s.Cin, IW, IH)) return cudaErrorInvalidValue;
-  if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
+  if (!make_filter_row_map(&mw, wt_tap_major, s.Cout, s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
   CUtensorMap my = mw;  // only read when there is a full-resolution output
   if (out && !make_patch_map(&my, out, s.N, s.H, s.W, s.Cout, PW, PH)) return cudaErrorInvalidValue;
   HaloArgs a;

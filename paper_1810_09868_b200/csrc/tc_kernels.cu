@@ -84,6 +84,18 @@ bool make_patch_map(CUtensorMap* map, const void* base, int N, int H, int W, int
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_filter_row_map(CUtensorMap* map, const void* base, int Cout, int Cin, uint32_t box_cout) {
+  const TensorMapApi& api = tensor_map_api();
+  if (!api.ok) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)Cin, (cuuint64_t)Cout, 9};
+  cuuint64_t strides[2] = {(cuuint64_t)Cin * 2, (cuuint64_t)Cout * Cin * 2};
+  cuuint32_t box[3] = {64, box_cout, 3};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return api.encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_patch_map_c8(CUtensorMap* map, const void* base, int N, int H, int W, uint32_t box_w, uint32_t box_h) {
   const TensorMapApi& api = tensor_map_api();
   if (!api.ok) return false;

@@ -20,8 +20,11 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
 // The same convolution with the input patch (plus halo) kept in shared memory
 // for all nine taps (tc_conv_halo.cu): the large-image, few-channel layers.
 bool tc_conv3x3_halo_supported(ConvShape s);
+// The filter comes tap-major, [9][Cout][Cin] (tc_make_tap_major builds it from the fp32 [Cout][3][3][Cin]
+// master; for_dgrad gives the rotated, channel-swapped filter of the input gradient, [9][Cin][Cout]).
 // `pooled` (or null) also receives the 2x2 max-pool of the result; `out` may then be null.
-cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out,
+cudaError_t tc_make_tap_major(const float* w, bf16* out, int Cin, int Cout, bool for_dgrad, cudaStream_t st);
+cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
                             bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
 
 // Filter gradient of the same convolution as a GEMM with M = Cout, N = 9*Cin,

@@ -62,6 +62,8 @@ struct vgg19 {
   float *params = nullptr;   // fp32 master, device
   void *params_t = nullptr;  // copy in the storage dtype (aliases params in fp32 mode)
   void *dgrad_w = nullptr;   // rotated filters for layers 2..16, storage dtype
+  bf16 *tap_fwd = nullptr;   // tap-major [9][Cout][Cin] filters of layers 2..16 (halo kernel), at dgrad_off
+  bf16 *tap_bwd = nullptr;   // tap-major rotated filters [9][Cin][Cout] of the same layers
   bf16 *w8 = nullptr;        // first-layer filter padded to [64][10][8] (bf16 tensor-core path)
   int *dev_error = nullptr;
   void *ws = nullptr;
@@ -213,7 +215,7 @@ struct Pass {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       ok(tc_first_conv((const bf16 *)buf(p.x8), n->w8, n->params + c.b_off, (bf16 *)y, s, true, n->dev_error, st), 1);
     } else if (n->use_tc && tc_conv3x3_halo_supported(s)) {
-      ok(tc_conv3x3_halo((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
+      ok(tc_conv3x3_halo((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
                          (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st), 1);
       return;
     } else if (tc_conv_ok(s))
@@ -243,7 +245,7 @@ struct Pass {
       ConvShape t{B, c.H, c.W, c.Cout, c.Cin};  // a 3x3 correlation from Cout to Cin channels
       const T *wr = static_cast<const T *>(n->dgrad_w) + c.dgrad_off;
       if (n->use_tc && tc_conv3x3_halo_supported(t))
-        ok(tc_conv3x3_halo((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr, t,
+        ok(tc_conv3x3_halo((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr, t,
                            false, n->dev_error, st), 1);
       else if (tc_conv_ok(t))
         ok(tc_conv3x3((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
@@ -415,6 +417,12 @@ int upload_params(vgg19 *n, const float *host) {
       CUDA_TRY(n, make_dgrad_filter<float>(n->params + c.w_off, (float *)n->dgrad_w + c.dgrad_off, c.Cin, c.Cout, 0));
   }
   if (n->w8) CUDA_TRY(n, tc_make_first_filter(n->params + n->conv[0].w_off, n->w8, 0));
+  if (n->tap_fwd)
+    for (int l = 1; l < kConvLayers; ++l) {
+      const ConvLayer &c = n->conv[l];
+      CUDA_TRY(n, tc_make_tap_major(n->params + c.w_off, n->tap_fwd + c.dgrad_off, c.Cin, c.Cout, false, 0));
+      CUDA_TRY(n, tc_make_tap_major(n->params + c.w_off, n->tap_bwd + c.dgrad_off, c.Cin, c.Cout, true, 0));
+    }
   CUDA_TRY(n, cudaDeviceSynchronize());
   return VGG19_OK;
 }
@@ -469,6 +477,8 @@ int create_common(const vgg19_config *cfg, vgg19 **out) {
   }
   if (e == cudaSuccess) e = cudaMalloc(&n->dgrad_w, n->n_dgrad * n->elt);
   if (e == cudaSuccess && n->use_tc) e = cudaMalloc(&n->w8, 64 * 80 * sizeof(bf16));
+  if (e == cudaSuccess && n->use_tc) e = cudaMalloc(&n->tap_fwd, n->n_dgrad * sizeof(bf16));
+  if (e == cudaSuccess && n->use_tc) e = cudaMalloc(&n->tap_bwd, n->n_dgrad * sizeof(bf16));
   if (e == cudaSuccess) e = cudaMalloc(&n->dev_error, 256);
   if (e == cudaSuccess) e = cudaMemset(n->dev_error, 0, 256);
   if (e != cudaSuccess) {
@@ -514,6 +524,8 @@ void vgg19_destroy(vgg19_t *n) {
   if (n->params) cudaFree(n->params);
   if (n->dgrad_w) cudaFree(n->dgrad_w);
   if (n->w8) cudaFree(n->w8);
+  if (n->tap_fwd) cudaFree(n->tap_fwd);
+  if (n->tap_bwd) cudaFree(n->tap_bwd);
   if (n->dev_error) cudaFree(n->dev_error);
   delete n;
 }
