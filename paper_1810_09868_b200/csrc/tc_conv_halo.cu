@@ -41,9 +41,10 @@ struct HaloTile {
   static constexpr int B_BYTES = 3 * TAP_BYTES;   // a filter row: three taps
   static constexpr int NA = BN <= 64 ? 3 : 2;     // input-patch slots
   static constexpr int OUT_BYTES = BM * 64 * 2;   // staging tile of the TMA store
-  static constexpr int kBudget = 227 * 1024 - 4608 - NA * A_SLOT - OUT_BYTES;
+  // one staging tile for the output and one for the ReLU-mask tile of the input gradient
+  static constexpr int kBudget = 227 * 1024 - 4608 - NA * A_SLOT - 2 * OUT_BYTES;
   static constexpr int NB = kBudget / B_BYTES > 4 ? 4 : kBudget / B_BYTES;
-  static constexpr int SMEM_BYTES = NA * A_SLOT + NB * B_BYTES + OUT_BYTES + 1024 + 512;
+  static constexpr int SMEM_BYTES = NA * A_SLOT + NB * B_BYTES + 2 * OUT_BYTES + 1024 + 512;
 };
 
 struct HaloArgs {
@@ -61,14 +62,16 @@ struct HaloArgs {
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                       const __grid_constant__ CUtensorMap map_y, HaloArgs a) {
+                       const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_m,
+                       HaloArgs a) {
   using T = HaloTile<BN>;
   constexpr int NA = T::NA;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_base = smem_base + NA * A_SLOT;
   const uint32_t out_smem = b_base + T::NB * T::B_BYTES;  // 1024-byte aligned
-  const uint32_t bars = out_smem + T::OUT_BYTES;
+  const uint32_t mask_smem = out_smem + T::OUT_BYTES;
+  const uint32_t bars = mask_smem + T::OUT_BYTES;
   auto a_full = [&](int s) { return bars + 8u * s; };
   auto a_empty = [&](int s) { return bars + 8u * (NA + s); };
   auto b_full = [&](int s) { return bars + 8u * (2 * NA + s); };
@@ -76,6 +79,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   auto acc_full = [&](int b) { return bars + 8u * (2 * NA + 2 * T::NB + b); };
   auto acc_empty = [&](int b) { return bars + 8u * (2 * NA + 2 * T::NB + 2 + b); };
   const uint32_t drain_bar = bars + 8u * (2 * NA + 2 * T::NB + 4);
+  const uint32_t mask_bar = bars + 8u * (2 * NA + 2 * T::NB + 5);
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ __align__(16) float bias_s[512];  // the layer's bias (zeros when it has none)
@@ -90,6 +94,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     for (int s = 0; s < T::NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 128); }
     mbar_init(drain_bar, 1);
+    mbar_init(mask_bar, 1);
     mbar_fence_init();
     tma_prefetch_desc(&map_x);
     tma_prefetch_desc(&map_w);
@@ -213,6 +218,8 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     // store groups.
     const bool issuer = threadIdx.x == 64;
     uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
+    const uint8_t* mask_srow = smem_raw + (mask_smem - smem_u32(smem_raw)) + row * 128;
+    uint32_t mask_phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
@@ -224,19 +231,25 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       const int th = t % a.tiles_h, img = t / a.tiles_h;
       const int h = th * PH + row / PW;
       const int w = tw * PW + row % PW;
-      const long pixel = ((long)img * a.H + h) * a.W + w;  // always inside the image: H % 16 == 0, W % 8 == 0
       const int c_base = n_tile * BN;
       // 2x2 pooling: a warp holds four patch rows of eight pixels (lane = 8 * row + column), so every
       // window lies inside one warp; the lane of the window's top-left pixel stores the maximum
       const bool pool_lane = (lane & 1) == 0 && (lane & 8) == 0;
       bf16* pool_row = a.pooled ? a.pooled + (((long)img * (a.H / 2) + h / 2) * (a.W / 2) + w / 2) * a.Cout + c_base
                                 : nullptr;
-      const bf16* mask_row = a.mask ? a.mask + pixel * a.Cout + c_base : nullptr;
 #pragma unroll 1
       for (int c64 = 0; c64 < BN; c64 += 64) {
         if (a.out) {
           if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
           named_bar_sync(1, 128);
+        }
+        // input gradient: the ReLU mask (the layer below's output at the same pixels) arrives as one
+        // tiled box in the staging layout; everyone finished reading the previous one before the
+        // barrier above
+        bool mask_ready = false;
+        if (a.mask && issuer) {
+          mbar_expect_tx(mask_bar, T::OUT_BYTES);
+          tma_load_4d(mask_smem, &map_m, mask_bar, c_base + c64, tw * PW, th * PH, img);
         }
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -253,11 +266,15 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
             packed[j >> 1] = *reinterpret_cast<uint32_t*>(&hh);
           }
-          if (mask_row) {
-            const uint4* mp = reinterpret_cast<const uint4*>(mask_row + cc);
+          if (a.mask) {
+            if (!mask_ready) {  // a failed wait leaves the tile unmasked; the error word says so
+              mask_ready = mbar_wait(mask_bar, mask_phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
+              mask_phase ^= 1;
+              mask_ready = true;
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const uint4 m = __ldg(mp + q);
+              const uint4 m = *reinterpret_cast<const uint4*>(mask_srow + (((half * 4 + q) ^ (row & 7)) << 4));
               const uint32_t mw[4] = {m.x, m.y, m.z, m.w};
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
@@ -321,8 +338,8 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 }
 
 template <int BN>
-cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, HaloArgs a,
-                        cudaStream_t st) {
+cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const CUtensorMap& mm,
+                        HaloArgs a, cudaStream_t st) {
   using T = HaloTile<BN>;
   static bool configured = false;
   if (!configured) {
@@ -334,7 +351,7 @@ cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int tiles = a.m_tiles * a.n_tiles;
-  conv3x3_halo_tc_kernel<BN><<<tiles < sms ? tiles : sms, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
+  conv3x3_halo_tc_kernel<BN><<<tiles < sms ? tiles : sms, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
   return cudaGetLastError();
 }
 
@@ -381,6 +398,9 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const floa
   if (!make_filter_row_map(&mw, wt_tap_major, s.Cout, s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
   CUtensorMap my = mw;  // only read when there is a full-resolution output
   if (out && !make_patch_map(&my, out, s.N, s.H, s.W, s.Cout, PW, PH)) return cudaErrorInvalidValue;
+  CUtensorMap mm = mw;  // only read when there is a mask
+  if (mask && !make_patch_map(&mm, mask, s.N, s.H, s.W, s.Cout, PW, PH)) return cudaErrorInvalidValue;
+  if (mask && !out) return cudaErrorInvalidValue;
   HaloArgs a;
   a.N = s.N; a.H = s.H; a.W = s.W;
   a.cin_blocks = s.Cin / 64; a.Cin = s.Cin; a.Cout = s.Cout;
@@ -388,7 +408,7 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const floa
   a.m_tiles = s.N * a.tiles_w * a.tiles_h;
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0; a.bias = bias; a.mask = mask; a.out = out; a.pooled = pooled; a.dev_error = dev_error;
-  return BN == 128 ? launch_halo<128>(mx, mw, my, a, st) : launch_halo<64>(mx, mw, my, a, st);
+  return BN == 128 ? launch_halo<128>(mx, mw, my, mm, a, st) : launch_halo<64>(mx, mw, my, mm, a, st);
 }
 
 }  // namespace vgg
