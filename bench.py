@@ -253,10 +253,7 @@ def run_native(args):
     sampler = ClockSampler(local) if rank == 0 else None
     if sampler:
         sampler.start()
-        with torch.cuda.stream(stream):  # nvidia-smi needs a moment to start sampling: keep the GPU busy meanwhile
-            for _ in range(30):
-                fwd()
-        stream.synchronize()
+        time.sleep(0.6)  # nvidia-smi needs a moment before its first sample
     t_begin = time.time()
     fwd_ms = timed(fwd, args.steps, args.warmup)
     net.sync_status(stream)

@@ -158,6 +158,17 @@ def test_smaller_batch_than_batch_max_and_ragged_sizes():
     net.close()
 
 
+def test_mid_size_image_takes_every_convolution_kernel():
+    # 96x64: layer 2 runs on the halo kernel, 48x32 and below on the general kernel in patch
+    # (48x32) and im2col (24x16, ...) mode
+    p = pkg()
+    params, images, labels = make_inputs(96, 64, 3, True, bias_std=0.05)
+    net = p.Net(96, 64, 3, p.VGG19_BF16, params=params)
+    logits, grads, loss = run_backward(net, images, labels)
+    check_bf16_backward(net, params, images, labels, logits, grads, loss)
+    net.close()
+
+
 def test_graph_replay_is_bit_identical_and_matches_direct_launch():
     p = pkg()
     params, images, _ = make_inputs(32, 32, 2, True)
