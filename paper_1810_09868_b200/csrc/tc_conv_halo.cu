@@ -39,12 +39,12 @@ template <int BN>
 struct HaloTile {
   static constexpr int TAP_BYTES = BN * BK * 2;   // one tap's BN x 64 filter slice
   static constexpr int B_BYTES = 3 * TAP_BYTES;   // a filter row: three taps
-  static constexpr int NA = BN <= 64 ? 3 : 2;     // input-patch slots
-  static constexpr int OUT_BYTES = BM * 64 * 2;   // staging tile of the TMA store
-  // one staging tile for the output and one for the ReLU-mask tile of the input gradient
-  static constexpr int kBudget = 227 * 1024 - 4608 - NA * A_SLOT - 2 * OUT_BYTES;
-  static constexpr int NB = kBudget / B_BYTES > 4 ? 4 : kBudget / B_BYTES;
-  static constexpr int SMEM_BYTES = NA * A_SLOT + NB * B_BYTES + 2 * OUT_BYTES + 1024 + 512;
+  static constexpr int OUT_BYTES = BM * 64 * 2;   // staging tile of the TMA store; a second one holds the mask tile
+  // Shared memory: `na` input-patch slots, the filter region, two staging tiles, barriers.  The filter
+  // region either holds the layer's whole filter slice for this kernel's BN output channels
+  // (cin_blocks x 9 taps, loaded once per CTA: "resident") or is a ring of `nb` filter rows.
+  static constexpr int kFixed = 2 * OUT_BYTES + 1024 + 512;
+  static constexpr int kLimit = 227 * 1024 - 2560;  // static shared memory (bias, flags) comes on top
 };
 
 struct HaloArgs {
@@ -53,6 +53,7 @@ struct HaloArgs {
   int tiles_w, tiles_h, m_tiles, n_tiles;
   int relu;
   const float* bias;
+  int na, nb, resident, b_region_bytes;  // shared-memory plan (see HaloTile)
   const bf16* mask;
   bf16* out;     // full-resolution output, or null when only the pooled output is wanted
   bf16* pooled;  // 2x2 max-pooled output [N][H/2][W/2][Cout], or null
@@ -65,21 +66,22 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                        const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_m,
                        HaloArgs a) {
   using T = HaloTile<BN>;
-  constexpr int NA = T::NA;
+  constexpr int NA = 3, NB = 4;  // most slots a plan may use (barrier numbering)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t b_base = smem_base + NA * A_SLOT;
-  const uint32_t out_smem = b_base + T::NB * T::B_BYTES;  // 1024-byte aligned
+  const uint32_t b_base = smem_base + a.na * A_SLOT;
+  const uint32_t out_smem = b_base + a.b_region_bytes;  // 1024-byte aligned
   const uint32_t mask_smem = out_smem + T::OUT_BYTES;
   const uint32_t bars = mask_smem + T::OUT_BYTES;
   auto a_full = [&](int s) { return bars + 8u * s; };
   auto a_empty = [&](int s) { return bars + 8u * (NA + s); };
   auto b_full = [&](int s) { return bars + 8u * (2 * NA + s); };
-  auto b_empty = [&](int s) { return bars + 8u * (2 * NA + T::NB + s); };
-  auto acc_full = [&](int b) { return bars + 8u * (2 * NA + 2 * T::NB + b); };
-  auto acc_empty = [&](int b) { return bars + 8u * (2 * NA + 2 * T::NB + 2 + b); };
-  const uint32_t drain_bar = bars + 8u * (2 * NA + 2 * T::NB + 4);
-  const uint32_t mask_bar = bars + 8u * (2 * NA + 2 * T::NB + 5);
+  auto b_empty = [&](int s) { return bars + 8u * (2 * NA + NB + s); };
+  auto acc_full = [&](int b) { return bars + 8u * (2 * NA + 2 * NB + b); };
+  auto acc_empty = [&](int b) { return bars + 8u * (2 * NA + 2 * NB + 2 + b); };
+  const uint32_t drain_bar = bars + 8u * (2 * NA + 2 * NB + 4);
+  const uint32_t mask_bar = bars + 8u * (2 * NA + 2 * NB + 5);
+  const uint32_t w_bar = bars + 8u * (2 * NA + 2 * NB + 6);  // resident filter loaded
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ __align__(16) float bias_s[512];  // the layer's bias (zeros when it has none)
@@ -91,10 +93,11 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
-    for (int s = 0; s < T::NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
+    for (int s = 0; s < NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 128); }
     mbar_init(drain_bar, 1);
     mbar_init(mask_bar, 1);
+    mbar_init(w_bar, 1);
     mbar_fence_init();
     tma_prefetch_desc(&map_x);
     tma_prefetch_desc(&map_w);
@@ -126,7 +129,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           mbar_expect_tx(a_full(slot), A_BYTES);
           tma_load_4d(smem_base + slot * A_SLOT, &map_x, a_full(slot), cb * BK, w0 - 1, h0 - 1, img);
           ++fills[slot];
-          if (++slot == NA) { slot = 0; phase ^= 1; }
+          if (++slot == a.na) { slot = 0; phase ^= 1; }
         }
       }
       if (!ok)
@@ -139,13 +142,22 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   } else if (warp == 6) {
     // ---------------- filter producer ----------------
     if (lane == 0) {
-      uint32_t fills[T::NB];
+      uint32_t fills[NB];
 #pragma unroll
-      for (int s = 0; s < T::NB; ++s) fills[s] = 0;
+      for (int s = 0; s < NB; ++s) fills[s] = 0;
       int slot = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      if (a.resident) {
+        // n_tiles == 1: the whole filter for these BN output channels, once
+        mbar_expect_tx(w_bar, (uint32_t)(a.cin_blocks * 3 * T::B_BYTES));
+        for (int cb = 0; cb < a.cin_blocks; ++cb)
+          for (int r = 0; r < 3; ++r)
+            tma_load_3d(b_base + (cb * 3 + r) * T::B_BYTES, &map_w, w_bar, cb * BK, 0, 3 * r);
+        const unsigned long long t0 = global_timer_ns();  // never leave with the copy in flight
+        while (!mbar_try_wait(w_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+      for (int tile = blockIdx.x; tile < total_tiles && ok && !a.resident; tile += gridDim.x) {
         const int n_tile = tile % a.n_tiles;
         for (int cb = 0; cb < a.cin_blocks && ok; ++cb)
           for (int r = 0; r < 3; ++r) {
@@ -153,11 +165,11 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             mbar_expect_tx(b_full(slot), T::B_BYTES);
             tma_load_3d(b_base + slot * T::B_BYTES, &map_w, b_full(slot), cb * BK, n_tile * BN, 3 * r);
             ++fills[slot];
-            if (++slot == T::NB) { slot = 0; phase ^= 1; }
+            if (++slot == a.nb) { slot = 0; phase ^= 1; }
           }
       }
       if (!ok)
-        for (int s = 0; s < T::NB; ++s)
+        for (int s = 0; s < NB; ++s)
           if (fills[s]) {
             const unsigned long long t0 = global_timer_ns();
             while (!mbar_try_wait(b_full(s), (fills[s] - 1) & 1) && global_timer_ns() - t0 < 100000000ull) {}
@@ -171,6 +183,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       uint32_t aphase = 0, bphase = 0;
       int local = 0;
       bool ok = true;
+      if (a.resident) ok = mbar_wait(w_bar, 0, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
         const int buf = local & 1;
         const uint32_t use = (uint32_t)(local >> 1);
@@ -181,7 +194,8 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           if (!mbar_wait(a_full(aslot), aphase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
           const uint32_t sa = smem_base + aslot * A_SLOT;
           for (int r = 0; r < 3; ++r) {
-            if (!mbar_wait(b_full(bslot), bphase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+            if (a.resident) bslot = cb * 3 + r;
+            else if (!mbar_wait(b_full(bslot), bphase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
             tc_fence_after();
 #pragma unroll
             for (int s = 0; s < 3; ++s) {
@@ -193,12 +207,12 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
               for (int k = 1; k < BK / 16; ++k)
                 umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
             }
-            umma_commit(b_empty(bslot));
-            if (++bslot == T::NB) { bslot = 0; bphase ^= 1; }
+            if (!a.resident) umma_commit(b_empty(bslot));
+            if (!a.resident && ++bslot == a.nb) { bslot = 0; bphase ^= 1; }
           }
           if (!ok) break;
           umma_commit(a_empty(aslot));
-          if (++aslot == NA) { aslot = 0; aphase ^= 1; }
+          if (++aslot == a.na) { aslot = 0; aphase ^= 1; }
         }
         if (ok) umma_commit(acc_full(buf));
       }
@@ -341,9 +355,26 @@ template <int BN>
 cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const CUtensorMap& mm,
                         HaloArgs a, cudaStream_t st) {
   using T = HaloTile<BN>;
+  // plan the shared memory: keep the whole filter resident when it fits beside two or three patch slots
+  // (then only the input patches cross the L2-to-SM path, which is what bounds these layers), else
+  // stream filter rows through a ring
+  const int res_bytes = a.cin_blocks * 3 * T::B_BYTES;
+  a.resident = 0;
+  for (int na = 3; na >= 2 && !a.resident; --na)
+    if (a.n_tiles == 1 && na * A_SLOT + res_bytes + T::kFixed <= T::kLimit) {
+      a.resident = 1; a.na = na; a.nb = 0; a.b_region_bytes = res_bytes;
+    }
+  if (!a.resident) {
+    a.na = BN <= 64 ? 3 : 2;
+    int nb = (T::kLimit - T::kFixed - a.na * A_SLOT) / T::B_BYTES;
+    a.nb = nb > 4 ? 4 : nb;
+    if (a.nb < 2) return cudaErrorInvalidValue;
+    a.b_region_bytes = a.nb * T::B_BYTES;
+  }
+  const int smem = a.na * A_SLOT + a.b_region_bytes + T::kFixed;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_halo_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_halo_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::kLimit);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -351,7 +382,7 @@ cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int tiles = a.m_tiles * a.n_tiles;
-  conv3x3_halo_tc_kernel<BN><<<tiles < sms ? tiles : sms, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
+  conv3x3_halo_tc_kernel<BN><<<tiles < sms ? tiles : sms, kThreads, smem, st>>>(mx, mw, my, mm, a);
   return cudaGetLastError();
 }
 
