@@ -43,7 +43,9 @@ struct HaloTile {
   // Shared memory: `na` input-patch slots, the filter region, two staging tiles, barriers.  The filter
   // region either holds the layer's whole filter slice for this kernel's BN output channels
   // (cin_blocks x 9 taps, loaded once per CTA: "resident") or is a ring of `nb` filter rows.
-  static constexpr int kFixed = 2 * OUT_BYTES + 1024 + 512;
+  // two output staging tiles (alternating, so a store can drain while the next chunk is converted),
+  // plus a mask tile for the input gradient
+  static constexpr int fixed_bytes(bool with_mask) { return (with_mask ? 3 : 2) * OUT_BYTES + 1024 + 512; }
   static constexpr int kLimit = 227 * 1024 - 2560;  // static shared memory (bias, flags) comes on top
 };
 
@@ -71,8 +73,8 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_base = smem_base + a.na * A_SLOT;
   const uint32_t out_smem = b_base + a.b_region_bytes;  // 1024-byte aligned
-  const uint32_t mask_smem = out_smem + T::OUT_BYTES;
-  const uint32_t bars = mask_smem + T::OUT_BYTES;
+  const uint32_t mask_smem = out_smem + 2 * T::OUT_BYTES;
+  const uint32_t bars = mask_smem + (a.mask ? T::OUT_BYTES : 0);
   auto a_full = [&](int s) { return bars + 8u * s; };
   auto a_empty = [&](int s) { return bars + 8u * (NA + s); };
   auto b_full = [&](int s) { return bars + 8u * (2 * NA + s); };
@@ -231,7 +233,8 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     // and one TMA store; the pooled output (a quarter of it) is stored directly.  Thread 64 owns the
     // store groups.
     const bool issuer = threadIdx.x == 64;
-    uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
+    uint8_t* stage_row0 = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
+    uint32_t stage_sel = 0;  // which of the two staging tiles the next chunk uses
     const uint8_t* mask_srow = smem_raw + (mask_smem - smem_u32(smem_raw)) + row * 128;
     uint32_t mask_phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
@@ -254,7 +257,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 #pragma unroll 1
       for (int c64 = 0; c64 < BN; c64 += 64) {
         if (a.out) {
-          if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
+          if (issuer) tma_store_wait_read<1>();  // the store before last, which used this staging tile, has read it
           named_bar_sync(1, 128);
         }
         // input gradient: the ReLU mask (the layer below's output at the same pixels) arrives as one
@@ -304,7 +307,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
               const int chunk = half * 4 + q;  // 16-byte chunk of the 128-byte staging row
-              *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) =
+              *reinterpret_cast<uint4*>(stage_row0 + stage_sel * T::OUT_BYTES + ((chunk ^ (row & 7)) << 4)) =
                   make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
             }
           }
@@ -331,9 +334,10 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           fence_async_smem();
           named_bar_sync(1, 128);
           if (issuer) {
-            tma_store_4d(&map_y, out_smem, c_base + c64, tw * PW, th * PH, img);
+            tma_store_4d(&map_y, out_smem + stage_sel * T::OUT_BYTES, c_base + c64, tw * PW, th * PH, img);
             tma_store_commit();
           }
+          stage_sel ^= 1;
         }
       }
       tc_fence_before();
@@ -359,19 +363,20 @@ cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
   // (then only the input patches cross the L2-to-SM path, which is what bounds these layers), else
   // stream filter rows through a ring
   const int res_bytes = a.cin_blocks * 3 * T::B_BYTES;
+  const int fixed = T::fixed_bytes(a.mask != nullptr);
   a.resident = 0;
   for (int na = 3; na >= 2 && !a.resident; --na)
-    if (a.n_tiles == 1 && na * A_SLOT + res_bytes + T::kFixed <= T::kLimit) {
+    if (a.n_tiles == 1 && na * A_SLOT + res_bytes + fixed <= T::kLimit) {
       a.resident = 1; a.na = na; a.nb = 0; a.b_region_bytes = res_bytes;
     }
   if (!a.resident) {
     a.na = BN <= 64 ? 3 : 2;
-    int nb = (T::kLimit - T::kFixed - a.na * A_SLOT) / T::B_BYTES;
+    int nb = (T::kLimit - fixed - a.na * A_SLOT) / T::B_BYTES;
     a.nb = nb > 4 ? 4 : nb;
     if (a.nb < 2) return cudaErrorInvalidValue;
     a.b_region_bytes = a.nb * T::B_BYTES;
   }
-  const int smem = a.na * A_SLOT + a.b_region_bytes + T::kFixed;
+  const int smem = a.na * A_SLOT + a.b_region_bytes + fixed;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(conv3x3_halo_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::kLimit);
