@@ -1,7 +1,9 @@
 // First convolution layer (3 input channels) on tensor cores.
 //
 // With 3 channels a pixel is 6 bytes, below TMA's 16-byte granule, so the image
-// is first copied into an 8-channel tensor (channels 3..7 zero).  The layer is
+// is first copied into an 8-channel tensor (channel 3 one, channels 4..7 zero;
+// the filter is zero there, and the constant channel lets the filter-gradient
+// GEMM produce the bias gradient as one more column).  The layer is
 // then the implicit GEMM  D[pixel][cout] = sum_{tap, c<8} X8[pixel + tap][c] * W8[cout][tap][c]
 // with K = 10 taps x 8 channels = 80 (tap 9 is zero padding so that K is a
 // multiple of the MMA depth 16).  One K step of an MMA is two taps: each tap is
@@ -251,13 +253,13 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   }
 }
 
-// x8[p][0..2] = x[p][0..2], x8[p][3..7] = 0
+// x8[p][0..2] = x[p][0..2], x8[p][3] = 1, x8[p][4..7] = 0
 __global__ void pad_to8_kernel(const bf16* __restrict__ x, bf16* __restrict__ x8, long P) {
   long p = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= P) return;
   const unsigned short* s = reinterpret_cast<const unsigned short*>(x) + p * 3;
   const uint32_t a = s[0], b = s[1], c = s[2];
-  reinterpret_cast<uint4*>(x8)[p] = make_uint4(a | (b << 16), c, 0u, 0u);
+  reinterpret_cast<uint4*>(x8)[p] = make_uint4(a | (b << 16), c | (0x3F80u << 16), 0u, 0u);  // 0x3F80 = bf16 1.0
 }
 
 // w8[k][tap][c] = w[k][tap][c] for tap < 9 and c < 3, else 0

@@ -479,9 +479,16 @@ cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* pa
 // ---- filter gradient of the first layer (3 channels, read from the 8-channel copy) ----
 
 namespace {
-// dW[k][tap][c] = sum over splits of partial[split][k][tap * 8 + c], c < 3
-__global__ void wgrad_c8_finish_kernel(const float* __restrict__ partial, int splits, int Cout, float* dW) {
+// dW[k][tap][c] = sum over splits of partial[split][k][tap * 8 + c], c < 3.  Channel 3 of the
+// 8-channel image is the constant 1, so column (centre tap, channel 3) is sum_pixels dz[pixel][k]:
+// the bias gradient.
+__global__ void wgrad_c8_finish_kernel(const float* __restrict__ partial, int splits, int Cout, float* dW, float* db) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (db && i < Cout) {
+    float s = 0.f;
+    for (int z = 0; z < splits; ++z) s += partial[((long)z * Cout + i) * 80 + 4 * 8 + 3];
+    db[i] = s;
+  }
   if (i >= Cout * 27) return;
   int c = i % 3, tap = (i / 3) % 9, k = i / 27;
   float s = 0.f;
@@ -501,7 +508,7 @@ size_t tc_first_wgrad_scratch_elems(ConvShape s) {
   return (size_t)splits * s.Cout * 80;
 }
 
-cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* partial, ConvShape s, int* dev_error,
+cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* db, float* partial, ConvShape s, int* dev_error,
                            cudaStream_t st) {
   const long P = (long)s.N * s.H * s.W;
   CUtensorMap ma, mb;
@@ -514,7 +521,7 @@ cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* par
   g.dev_error = dev_error; g.ldc = 80; g.partial = partial;
   cudaError_t e = launch_gemm_tc<80, kMnMajor, kMnMajorIm2colC8>(ma, mb, g, 1, splits, st);
   if (e != cudaSuccess) return e;
-  wgrad_c8_finish_kernel<<<(s.Cout * 27 + 255) / 256, 256, 0, st>>>(partial, splits, s.Cout, dW);
+  wgrad_c8_finish_kernel<<<(s.Cout * 27 + 255) / 256, 256, 0, st>>>(partial, splits, s.Cout, dW, db);
   return cudaGetLastError();
 }
 

@@ -55,7 +55,8 @@ cudaError_t tc_make_first_filter(const float* w, bf16* w8, cudaStream_t st);
 cudaError_t tc_first_conv(const bf16* x8, const bf16* w8, const float* bias, bf16* out, ConvShape s, bool relu,
                           int* dev_error, cudaStream_t st);
 size_t tc_first_wgrad_scratch_elems(ConvShape s);
-cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* partial, ConvShape s, int* dev_error,
+// x8 must come from tc_pad_to8 (its constant channel yields db, fp32 [64], when db is not null).
+cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* db, float* partial, ConvShape s, int* dev_error,
                            cudaStream_t st);
 
 }  // namespace vgg

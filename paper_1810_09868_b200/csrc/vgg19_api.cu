@@ -232,9 +232,8 @@ struct Pass {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
     if (first_tc_ok(l, s)) {
-      ok(simt_bias_grad<T>(dz, db, fbuf(p.partial), (long)B * c.H * c.W, c.Cout, st), 2);
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
-      ok(tc_first_wgrad((const bf16 *)buf(p.x8), (const bf16 *)dz, dW, fbuf(p.partial), s, n->dev_error, st), 2);
+      ok(tc_first_wgrad((const bf16 *)buf(p.x8), (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st), 2);
     } else if (n->use_tc && tc_wgrad_supported(s)) {
       ok(simt_bias_grad<T>(dz, db, fbuf(p.partial), (long)B * c.H * c.W, c.Cout, st), 2);
       ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, fbuf(p.partial), s, n->dev_error, st),
