@@ -18,6 +18,11 @@
 // With K split, tiles write raw fp32 partial sums and a second kernel adds the
 // splits in a fixed order and applies bias / ReLU / mask (deterministic).
 // All waits are time-limited (see tc_common.cuh).
+//
+// The filter gradient can also produce the bias gradient db[m] = sum_k A(m, k): a narrow extra MMA
+// multiplies the A tile by a block of ones into 16 spare tensor-memory columns.  The CTAs that share
+// an m tile (one per n tile) take turns, K block by K block, so that the extra issue time is spread
+// evenly; each writes its part of the sum and the finishing kernel adds the parts in a fixed order.
 #include "tc_common.cuh"
 #include "tc_kernels.cuh"
 
@@ -49,6 +54,7 @@ struct GemmArgs {
   const bf16* mask;  // same shape as the output, or null: keep where mask > 0
   int relu;
   int* dev_error;
+  float* db_partial; // column sums of A at db_partial[((split * n_tiles) + n_tile) * M + m], or null
 };
 
 template <int BN>
@@ -58,7 +64,8 @@ template <int BN, int AMODE, int BMODE>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs g) {
   constexpr int STAGE = stage_bytes<BN>();
-  constexpr int TMEM_COLS = BN <= 32 ? 32 : (BN <= 64 ? 64 : (BN <= 128 ? 128 : 256));
+  // 32 spare columns after the tile where the column sums of A can accumulate
+  constexpr int TMEM_COLS = BN + 32 <= 64 ? 64 : (BN + 32 <= 128 ? 128 : (BN + 32 <= 256 ? 256 : 512));
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = smem_base + g.stages * STAGE;
@@ -66,6 +73,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
   const uint32_t acc_bar = bars + 8u * (2 * kMaxStages);
   const uint32_t drain_bar = bars + 8u * (2 * kMaxStages + 1);
+  const uint32_t ones = bars + 256;  // 1 KB of bf16 1.0
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -74,6 +82,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int m0 = m_tile * BM, n0 = n_tile * BN;
   const int kb0 = blockIdx.y * g.kb_per_split;
   const int kb1 = min(g.k_blocks, kb0 + g.kb_per_split);
+  // K blocks kb = n_tile (mod n_tiles) are the ones whose column sums this CTA adds
+  int db_first = kb1;
+  if (g.db_partial) {
+    int r = n_tile - kb0 % g.n_tiles;
+    if (r < 0) r += g.n_tiles;
+    db_first = kb0 + r;
+    if (threadIdx.x >= 64) {
+      const uint32_t t = threadIdx.x - 64;  // 128 threads x 8 bytes
+      asm volatile("st.shared.v2.b32 [%0], {%1, %1};" ::"r"(ones + 8u * t), "r"(0x3F803F80u) : "memory");
+    }
+    fence_async_smem();
+  }
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -164,6 +184,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, AMODE != kKMajor, BMODE != kKMajor);
+      constexpr uint32_t idesc_ones = umma_idesc_bf16(BM, 16, AMODE != kKMajor, false);
+      const uint64_t d_ones = smem_desc_plain(ones, 128, 256);  // every element is 1: the layout is immaterial
+      int db_next = db_first;
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -183,6 +206,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
         for (int k = 1; k < BK / 16; ++k)
           umma_bf16_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), idesc);
+        if (kb == db_next) {
+          umma_bf16(tmem_base + BN, da, d_ones, idesc_ones, kb != db_first ? 1u : 0u);
+#pragma unroll
+          for (int k = 1; k < BK / 16; ++k) umma_bf16_acc(tmem_base + BN, desc_advance(da, k * a_step), d_ones, idesc_ones);
+          db_next += g.n_tiles;
+        }
         umma_commit(empty_bar(stage));
         if (++stage == g.stages) { stage = 0; phase ^= 1; }
       }
@@ -250,6 +279,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
       }
+      if (g.db_partial) {
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)BN, v);
+        tmem_ld_wait();
+        if (row_ok)
+          g.db_partial[((long)blockIdx.y * g.n_tiles + n_tile) * g.M + m] = db_first < kb1 ? __uint_as_float(v[0]) : 0.f;
+      }
     }
   }
 
@@ -265,8 +301,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // out = epilogue(sum over splits of partial[split]), four columns per thread
 __global__ void splitk_finish_kernel(const float* __restrict__ partial, int splits, long MN, int N,
                                      const float* __restrict__ bias, int relu, const bf16* __restrict__ mask,
-                                     bf16* out_h, float* out_f) {
-  const long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+                                     bf16* out_h, float* out_f, const float* __restrict__ db_partial, int db_parts,
+                                     int M, float* db) {
+  const long t = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (db && t < M) {
+    float s = 0.f;
+    for (int z = 0; z < db_parts; ++z) s += db_partial[(long)z * M + t];
+    db[t] = s;
+  }
+  const long i = t * 4;
   if (i >= MN) return;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int z = 0; z < splits; ++z) {
@@ -314,27 +357,37 @@ template <int BN, int AMODE, int BMODE>
 cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArgs g, int m_tiles, int splits,
                            cudaStream_t st) {
   constexpr int STAGE = stage_bytes<BN>();
-  constexpr int max_stages = (227 * 1024 - 2048) / STAGE > kMaxStages ? kMaxStages : (227 * 1024 - 2048) / STAGE;
+  constexpr int kExtra = 1024 + 256 + 1024;  // alignment slack, barriers, block of ones
+  constexpr int max_stages = (227 * 1024 - 3072) / STAGE > kMaxStages ? kMaxStages : (227 * 1024 - 3072) / STAGE;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, AMODE, BMODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         max_stages * STAGE + 1024 + 256);
+                                         max_stages * STAGE + kExtra);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   g.stages = g.kb_per_split < max_stages ? g.kb_per_split : max_stages;
-  const size_t smem = (size_t)g.stages * STAGE + 1024 + 256;
+  const size_t smem = (size_t)g.stages * STAGE + kExtra;
   dim3 grid(m_tiles * g.n_tiles, splits);
   gemm_tc_kernel<BN, AMODE, BMODE><<<grid, kThreads, smem, st>>>(ma, mb, g);
   return cudaGetLastError();
 }
 
 cudaError_t finish(const GemmArgs& g, int splits, const float* bias, bool relu, const bf16* mask, bf16* out_h,
-                   float* out_f, cudaStream_t st) {
+                   float* out_f, cudaStream_t st, float* db = nullptr) {
   const long MN = (long)g.M * g.N;
   splitk_finish_kernel<<<(unsigned)((MN / 4 + 255) / 256), 256, 0, st>>>(g.partial, splits, MN, g.N, bias, relu ? 1 : 0,
-                                                                          mask, out_h, out_f);
+                                                                          mask, out_h, out_f, g.db_partial,
+                                                                          splits * g.n_tiles, g.M, db);
   return cudaGetLastError();
+}
+
+__global__ void db_finish_kernel(const float* __restrict__ db_partial, int parts, int M, float* db) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= M) return;
+  float s = 0.f;
+  for (int z = 0; z < parts; ++z) s += db_partial[(long)z * M + t];
+  db[t] = s;
 }
 
 }  // namespace
@@ -442,18 +495,19 @@ size_t tc_wgrad_scratch_elems(ConvShape s) {
   if (!tc_wgrad_supported(s)) return 0;
   int mt, nt, kb, splits, per;
   wgrad_plan(s, &mt, &nt, &kb, &splits, &per);
-  return (size_t)splits * s.Cout * 9 * s.Cin;
+  return (size_t)splits * s.Cout * 9 * s.Cin + (size_t)splits * nt * s.Cout;
 }
 
-int tc_wgrad_launches(ConvShape s) {
+int tc_wgrad_launches(ConvShape s, bool with_db) {
   int mt, nt, kb, splits, per;
   wgrad_plan(s, &mt, &nt, &kb, &splits, &per);
-  return splits > 1 ? 2 : 1;
+  return splits > 1 || with_db ? 2 : 1;
 }
 
-// dW[k][tap][c] = sum_pixels dz[pixel][k] * x[pixel + tap][c]   (fp32 out, [Cout][9*Cin])
-cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* partial, ConvShape s, int* dev_error,
-                             cudaStream_t st) {
+// dW[k][tap][c] = sum_pixels dz[pixel][k] * x[pixel + tap][c]   (fp32 out, [Cout][9*Cin]);
+// db[k] = sum_pixels dz[pixel][k] when db is not null
+cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* db, float* partial, ConvShape s,
+                             int* dev_error, cudaStream_t st) {
   if (!tc_wgrad_supported(s)) return cudaErrorInvalidValue;
   const long P = (long)s.N * s.H * s.W;
   const int BN = wgrad_bn(s.Cin);
@@ -466,14 +520,20 @@ cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* pa
   g.M = s.Cout; g.N = 9 * s.Cin; g.H = s.H; g.W = s.W; g.Cin = s.Cin;
   g.dev_error = dev_error; g.ldc = g.N;
   if (splits == 1) g.out_f = dW; else g.partial = partial;
+  if (db) g.db_partial = partial + (splits == 1 ? 0 : (size_t)splits * s.Cout * 9 * s.Cin);
   cudaError_t e;
   switch (BN) {
     case 256: e = launch_gemm_tc<256, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
     case 128: e = launch_gemm_tc<128, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
     default: e = launch_gemm_tc<192, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
   }
-  if (e != cudaSuccess || splits == 1) return e;
-  return finish(g, splits, nullptr, false, nullptr, nullptr, dW, st);
+  if (e != cudaSuccess) return e;
+  if (splits == 1) {
+    if (!db) return e;
+    db_finish_kernel<<<(s.Cout + 255) / 256, 256, 0, st>>>(g.db_partial, g.n_tiles, s.Cout, db);
+    return cudaGetLastError();
+  }
+  return finish(g, splits, nullptr, false, nullptr, nullptr, dW, st, db);
 }
 
 // ---- filter gradient of the first layer (3 channels, read from the 8-channel copy) ----

@@ -235,9 +235,8 @@ struct Pass {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       ok(tc_first_wgrad((const bf16 *)buf(p.x8), (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st), 2);
     } else if (n->use_tc && tc_wgrad_supported(s)) {
-      ok(simt_bias_grad<T>(dz, db, fbuf(p.partial), (long)B * c.H * c.W, c.Cout, st), 2);
-      ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, fbuf(p.partial), s, n->dev_error, st),
-         tc_wgrad_launches(s));
+      ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st),
+         tc_wgrad_launches(s, db != nullptr));
     } else
       ok(simt_conv3x3_wgrad<T>(x, dz, dW, db, fbuf(p.partial), s, st), 4);
     if (dx) {
