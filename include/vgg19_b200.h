@@ -53,7 +53,8 @@ typedef enum {
 
 enum {
   VGG19_FLAG_NO_GRAPH = 1,        /* enqueue kernels directly instead of replaying a CUDA graph */
-  VGG19_FLAG_NO_TENSOR_CORES = 2  /* bf16 only: use the CUDA-core kernels for every layer */
+  VGG19_FLAG_NO_TENSOR_CORES = 2, /* bf16 only: use the CUDA-core kernels for every layer */
+  VGG19_FLAG_NO_CTA_PAIRS = 4     /* one CTA per tile everywhere: no two-CTA (cta_group::2) kernels */
 };
 
 typedef enum { VGG19_MODE_FORWARD = 0, VGG19_MODE_BACKWARD = 1 } vgg19_mode;

@@ -1,0 +1,329 @@
+// 3x3 convolution as an implicit GEMM on CTA pairs (tcgen05 cta_group::2) for the layers with many
+// output channels (56x56 images and below).
+//
+//   D[pixel][cout] = sum over (r, s, c) of  X[pixel shifted by (r-1, s-1)][c] * Wt[cout][r][s][c]
+//
+// A cluster of two CTAs computes a 256 (pixels) x BN (output channels) tile with one MMA stream:
+// each CTA stages its own 128 pixels (TMA im2col, zero padding from the out-of-bounds fill) and only
+// HALF of the BN x 64 filter slice per K block, and keeps its 128 accumulator rows in its own tensor
+// memory.  Against one CTA per 128 x BN tile that halves the filter bytes written to and read from
+// shared memory per MMA, which is what bounds the single-CTA kernel (per 128 x 256 x 16 MMA it
+// reads 12 KB and the copy engine writes another 12 KB, against 128 B per cycle of shared memory).
+//
+// Roles per CTA: warp 0 TMA producer (one thread), warp 1 tensor-memory owner and, in the even CTA
+// only, the single MMA-issuing thread; warps 2-5 epilogue (bias, ReLU / ReLU mask, bf16, swizzled
+// staging tile, TMA store).  Barriers the issuer waits on (stage full, accumulator drained) live in
+// the even CTA and receive the peer's signals through the cluster; barriers the issuer signals
+// (stage free, accumulator full) exist in both CTAs and are reached by one multicast commit.
+// Every wait has a time limit; a CTA that gives up drains its copies and MMAs, and both CTAs meet
+// at a cluster barrier before either releases tensor memory or exits.
+#include "tc_common.cuh"
+#include "tc_kernels.cuh"
+
+namespace vgg {
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128;   // pixels per CTA (tensor-memory lanes); the pair's tile has 2 * BM
+constexpr int BK = 64;    // channels per K block (one 128-byte swizzle row)
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int kThreads = 192;
+constexpr int kSmemLimit = 227 * 1024;
+
+template <int BN>
+struct PairTile {
+  static constexpr int B_BYTES = (BN / 2) * BK * 2;  // this CTA's half of the filter slice
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int OUT_BYTES = BM * 64 * 2;      // staging tile of the TMA store
+  static constexpr int STAGES = (kSmemLimit - 4608 - OUT_BYTES) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608 - OUT_BYTES) / STAGE_BYTES;
+  static constexpr int TMEM_COLS = 2 * BN;           // double-buffered accumulator
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + 1024 + 256;
+};
+
+struct PairArgs {
+  int pixels;      // N*H*W
+  int H, W;
+  int cin_blocks;  // Cin / 64
+  int Cout;
+  int m_pairs;     // ceil(pixels / 256)
+  int n_tiles;     // Cout / BN
+  int relu;
+  const float* bias;
+  const bf16* mask;
+  int* dev_error;
+};
+
+template <int BN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                       const __grid_constant__ CUtensorMap map_y, PairArgs a) {
+  using T = PairTile<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t out_smem = smem_base + T::STAGES * T::STAGE_BYTES;
+  const uint32_t bars = out_smem + T::OUT_BYTES;
+  auto full_bar = [&](int s) { return bars + 8u * s; };                       // used in the even CTA
+  auto empty_bar = [&](int s) { return bars + 8u * (T::STAGES + s); };        // both CTAs
+  auto acc_full_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + b); };       // both CTAs
+  auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + 2 + b); };  // used in the even CTA
+  const uint32_t drain_bar = bars + 8u * (2 * T::STAGES + 4);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  __shared__ __align__(16) float bias_s[512];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int k_blocks = 9 * a.cin_blocks;
+  const int total_tiles = a.m_pairs * a.n_tiles;
+
+  for (int i = threadIdx.x; i < a.Cout; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < T::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 256); }
+    mbar_init(drain_bar, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&map_x);
+    tma_prefetch_desc(&map_w);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&tmem_base_slot), T::TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised before anything signals them
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      uint32_t fills[T::STAGES];
+#pragma unroll
+      for (int s = 0; s < T::STAGES; ++s) fills[s] = 0;
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+        const int m_pair = tile / a.n_tiles, n_tile = tile - m_pair * a.n_tiles;
+        // a CTA whose 128 pixels all lie past the end of the tensor (odd tile count) stages the
+        // tensor's first pixels instead: its accumulator rows are never stored
+        int p0 = (2 * m_pair + (int)rank) * BM;
+        if (p0 >= a.pixels) p0 = 0;
+        const int w0 = p0 % a.W, t = p0 / a.W;
+        const int h0 = t % a.H, n0 = t / a.H;
+        const int filter_row = n_tile * BN + (int)rank * (BN / 2);
+        int kb = 0;
+        for (int r = 0; r < 3 && ok; ++r)
+          for (int s = 0; s < 3 && ok; ++s)
+            for (int cb = 0; cb < a.cin_blocks; ++cb, ++kb) {
+              if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
+              const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
+              const uint32_t full = map_to_cta(full_bar(stage), 0);
+              // the even CTA announces the bytes of both CTAs' copies for this stage
+              if (leader) mbar_expect_tx(full_bar(stage), 2 * T::STAGE_BYTES);
+              tma_load_im2col_4d_pair(sa, &map_x, full, cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
+              tma_load_2d_pair(sb, &map_w, full, kb * BK, filter_row);
+              ++fills[stage];
+              if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
+            }
+      }
+      if (!ok) {
+        // let every copy already in flight land before the CTA may go on to exit: the even CTA sees
+        // them on its stage barriers, the peer (whose copies report there too) allows them a millisecond
+        if (leader) {
+          for (int s = 0; s < T::STAGES; ++s)
+            if (fills[s]) {
+              const unsigned long long t0 = global_timer_ns();
+              while (!mbar_try_wait(full_bar(s), (fills[s] - 1) & 1) && global_timer_ns() - t0 < 100000000ull) {}
+            }
+        } else {
+          const unsigned long long t0 = global_timer_ns();
+          while (global_timer_ns() - t0 < 1000000ull) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------- MMA issuer (even CTA only) -------------------------
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc = umma_idesc_bf16(2 * BM, BN, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++local) {
+        const int buf = local & 1;
+        const uint32_t use = (uint32_t)(local >> 1);
+        if (!mbar_wait(acc_empty_bar(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
+          const uint64_t da = smem_desc_sw128(sa, 16), db = smem_desc_sw128(sb, 16);
+          umma_bf16_pair(d_tmem, da, db, idesc, kb != 0 ? 1u : 0u);
+#pragma unroll
+          for (int k = 1; k < BK / 16; ++k)
+            umma_bf16_pair_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
+          umma_commit_pair(empty_bar(stage), 3);  // frees the stage in both CTAs
+          if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit_pair(acc_full_bar(buf), 3);
+      }
+      if (!ok) {
+        umma_commit_pair(drain_bar, 1);  // arrives in this CTA only, once the pair's MMAs are done
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else {
+    // -------------------------------- epilogue --------------------------------
+    const int quarter = warp & 3;  // the tensor-memory lane quarter this warp may read
+    const int row = quarter * 32 + lane;
+    int local = 0;
+    const bool issuer = threadIdx.x == 64;  // owns the TMA store groups
+    uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
+    for (int tile = pair; tile < total_tiles; tile += n_pairs, ++local) {
+      const int buf = local & 1;
+      const uint32_t use = (uint32_t)(local >> 1);
+      const int m_pair = tile / a.n_tiles, n_tile = tile - m_pair * a.n_tiles;
+      const int m_tile = 2 * m_pair + (int)rank;
+      const bool got = mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
+      if (named_bar_or(1, 128, !got)) break;  // all four warps leave together
+      tc_fence_after();
+      const long pixel = (long)m_tile * BM + row;
+      const bool valid = pixel < a.pixels;
+      const bool tile_valid = (long)m_tile * BM < a.pixels;
+      const int c_base = n_tile * BN;
+      const bf16* mask_row = (a.mask && valid) ? a.mask + pixel * a.Cout + c_base : nullptr;
+#pragma unroll 1
+      for (int c64 = 0; c64 < BN && tile_valid; c64 += 64) {
+        if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
+        named_bar_sync(1, 128);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int cc = c64 + half * 32;
+          uint32_t v[32];
+          tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+          tmem_ld_wait();
+          uint32_t packed[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
+            x0 += bias_s[c_base + cc + j]; x1 += bias_s[c_base + cc + j + 1];
+            if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
+            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+            packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          if (mask_row) {
+            const uint4* mp = reinterpret_cast<const uint4*>(mask_row + cc);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 m = __ldg(mp + q);
+              const uint32_t mw[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                // a bf16 is > 0 iff its sign bit is clear and it is not zero
+                const uint32_t lo = mw[e] & 0xFFFFu, hi = mw[e] >> 16;
+                uint32_t keep = 0;
+                if (lo != 0 && !(lo & 0x8000u)) keep |= 0x0000FFFFu;
+                if (hi != 0 && !(hi & 0x8000u)) keep |= 0xFFFF0000u;
+                packed[q * 4 + e] &= keep;
+              }
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int chunk = half * 4 + q;  // 16-byte chunk of the 128-byte staging row
+            *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) =
+                make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+          }
+        }
+        fence_async_smem();
+        named_bar_sync(1, 128);
+        if (issuer) {
+          // rows past the end of the tensor (last tile) are clipped by the copy engine
+          tma_store_2d(&map_y, out_smem, c_base + c64, m_tile * BM);
+          tma_store_commit();
+        }
+      }
+      tc_fence_before();
+      mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));  // 256 arrivals: both CTAs have drained the buffer
+    }
+    if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
+  }
+
+  // Neither CTA may release tensor memory or exit while the other can still signal its barriers,
+  // read its shared memory or write its accumulator.
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, T::TMEM_COLS);
+  }
+}
+
+template <int BN>
+cudaError_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, PairArgs a, cudaStream_t st) {
+  using T = PairTile<BN>;
+  static int max_pairs = 0;  // CTA pairs that can be resident at once
+  if (!max_pairs) {
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_pair_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(sms & ~1));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = T::SMEM_BYTES;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, conv3x3_pair_tc_kernel<BN>, &cfg);
+    if (e != cudaSuccess || n < 1) { cudaGetLastError(); n = sms / 2; }
+    max_pairs = n < sms / 2 ? n : sms / 2;
+  }
+  const int tiles = a.m_pairs * a.n_tiles;
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  conv3x3_pair_tc_kernel<BN><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_conv3x3_pair_supported(ConvShape s) {
+  return s.Cin % 64 == 0 && s.Cout % 256 == 0 && s.Cout <= 512 && s.H >= 2 && s.W >= 2 && s.N >= 1 &&
+         (long)s.N * s.H * s.W < (1L << 31) - 512;
+}
+
+cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out, ConvShape s,
+                            bool relu, int* dev_error, cudaStream_t st) {
+  if (!tc_conv3x3_pair_supported(s)) return cudaErrorInvalidValue;
+  constexpr int BN = 256;
+  CUtensorMap mx, mw, my;
+  if (!make_im2col_map(&mx, in, s.N, s.H, s.W, s.Cin, BM)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, BN / 2)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d(&my, out, (uint64_t)s.N * s.H * s.W, (uint64_t)s.Cout, BM)) return cudaErrorInvalidValue;
+  PairArgs a;
+  a.pixels = s.N * s.H * s.W;
+  a.H = s.H; a.W = s.W;
+  a.cin_blocks = s.Cin / 64;
+  a.Cout = s.Cout;
+  a.m_pairs = (a.pixels + 2 * BM - 1) / (2 * BM);
+  a.n_tiles = s.Cout / BN;
+  a.relu = relu ? 1 : 0;
+  a.bias = bias; a.mask = mask; a.dev_error = dev_error;
+  return launch_pair<BN>(mx, mw, my, a, st);
+}
+
+}  // namespace vgg

@@ -17,6 +17,12 @@ bool tc_conv3x3_supported(ConvShape s);
 cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const bf16* mask,
                        bf16* out, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
 
+// The same convolution on CTA pairs (tc_conv_pair.cu): a cluster of two CTAs per 256-pixel x 256-channel
+// tile, each staging half of the filter slice.  Cout must be a multiple of 256.
+bool tc_conv3x3_pair_supported(ConvShape s);
+cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, const bf16* mask,
+                            bf16* out, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
+
 // The same convolution with the input patch (plus halo) kept in shared memory
 // for all nine taps (tc_conv_halo.cu): the large-image, few-channel layers.
 bool tc_conv3x3_halo_supported(ConvShape s);

@@ -72,6 +72,7 @@ struct vgg19 {
   int launches[2] = {0, 0};
   std::string err;
   bool use_tc = false;
+  bool use_pair = false;  // two-CTA kernels where a layer's shape takes them
 };
 
 namespace {
@@ -201,6 +202,7 @@ struct Pass {
   void ok(cudaError_t e, int k) { if (err == cudaSuccess) err = e; launches += k; }
 
   bool tc_conv_ok(const ConvShape &s) const { return n->use_tc && tc_conv3x3_supported(s); }
+  bool pair_ok(const ConvShape &s) const { return n->use_pair && tc_conv3x3_pair_supported(s); }
   // layer 1 on tensor cores needs the 8-channel image copy, i.e. a planned workspace
   bool first_tc_ok(int l, const ConvShape &s) const {
     return l == 0 && n->use_tc && p.valid && tc_first_conv_supported(s);
@@ -218,7 +220,10 @@ struct Pass {
       ok(tc_conv3x3_halo((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
                          (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st), 1);
       return;
-    } else if (tc_conv_ok(s))
+    } else if (pair_ok(s))
+      ok(tc_conv3x3_pair((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
+                         (bf16 *)y, s, true, n->dev_error, st), 1);
+    else if (tc_conv_ok(s))
       ok(tc_conv3x3((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
                     (bf16 *)y, s, true, n->dev_error, st), 1);
     else
@@ -245,6 +250,9 @@ struct Pass {
       if (n->use_tc && tc_conv3x3_halo_supported(t))
         ok(tc_conv3x3_halo((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr, t,
                            false, n->dev_error, st), 1);
+      else if (pair_ok(t))
+        ok(tc_conv3x3_pair((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
+                           t, false, n->dev_error, st), 1);
       else if (tc_conv_ok(t))
         ok(tc_conv3x3((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
                       t, false, n->dev_error, st), 1);
@@ -446,6 +454,7 @@ int create_common(const vgg19_config *cfg, vgg19 **out) {
   n->cfg = *cfg;
   n->elt = cfg->dtype == VGG19_BF16 ? 2 : 4;
   n->use_tc = cfg->dtype == VGG19_BF16 && !(cfg->flags & VGG19_FLAG_NO_TENSOR_CORES);
+  n->use_pair = n->use_tc && !(cfg->flags & VGG19_FLAG_NO_CTA_PAIRS);
   size_t off = 0, doff = 0;
   int h = cfg->height, w = cfg->width, cin = 3, n_pool = 0;
   for (int l = 0; l < kConvLayers; ++l) {
