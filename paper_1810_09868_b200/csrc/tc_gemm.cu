@@ -57,13 +57,17 @@ struct GemmArgs {
   float* db_partial; // column sums of A at db_partial[((split * n_tiles) + n_tile) * M + m], or null
 };
 
-template <int BN>
-__host__ __device__ constexpr int stage_bytes() { return A_BYTES + BN * BK * 2; }
+// PAIR: two CTAs (a cluster, tcgen05 cta_group::2) compute a 256 x BN tile with one MMA stream; each
+// stages its own 128 rows of A and half of the B tile.
+template <int BN, bool PAIR>
+__host__ __device__ constexpr int stage_bytes() { return A_BYTES + (PAIR ? BN / 2 : BN) * BK * 2; }
 
-template <int BN, int AMODE, int BMODE>
+template <int BN, int AMODE, int BMODE, bool PAIR>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs g) {
-  constexpr int STAGE = stage_bytes<BN>();
+  static_assert(!PAIR || (AMODE == kMnMajor && BMODE == kMnMajorIm2col && BN % 128 == 0), "pairs: filter gradient only");
+  constexpr int STAGE = stage_bytes<BN, PAIR>();
+  constexpr int B_GROUPS = (PAIR ? BN / 2 : BN) / 64;  // 64-column groups of B this CTA stages
   // 32 spare columns after the tile where the column sums of A can accumulate
   constexpr int TMEM_COLS = BN + 32 <= 64 ? 64 : (BN + 32 <= 128 ? 128 : (BN + 32 <= 256 ? 256 : 512));
   extern __shared__ uint8_t smem_raw[];
@@ -78,7 +82,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tile = blockIdx.x / g.n_tiles, n_tile = blockIdx.x - m_tile * g.n_tiles;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // position in the pair; rank 0 issues the MMAs
+  const int tile_index = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int m_tile = (tile_index / g.n_tiles) * (PAIR ? 2 : 1) + (int)rank, n_tile = tile_index % g.n_tiles;
   const int m0 = m_tile * BM, n0 = n_tile * BN;
   const int kb0 = blockIdx.y * g.kb_per_split;
   const int kb1 = min(g.k_blocks, kb0 + g.kb_per_split);
@@ -105,11 +111,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tma_prefetch_desc(&map_b);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
-    tmem_relinquish();
+    if (PAIR) {
+      tmem_alloc_pair(smem_u32(&tmem_base_slot), TMEM_COLS);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();  // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
@@ -123,13 +135,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool ok = true;
       // im2col forms: each 64-column group of the tile is (tap, 64 channels), fixed for the CTA; the
       // pixel a K block starts at advances by 64 per block (no divisions in the loop)
-      int grp_c[BN / 64 > 0 ? BN / 64 : 1], grp_s[BN / 64 > 0 ? BN / 64 : 1], grp_r[BN / 64 > 0 ? BN / 64 : 1];
+      int grp_c[B_GROUPS > 0 ? B_GROUPS : 1], grp_s[B_GROUPS > 0 ? B_GROUPS : 1], grp_r[B_GROUPS > 0 ? B_GROUPS : 1];
       int w0 = 0, h0 = 0, img = 0;
       if (BMODE == kMnMajorIm2col || BMODE == kMnMajorIm2colC8) {
         if (BMODE == kMnMajorIm2col) {
 #pragma unroll
-          for (int q = 0; q < BN / 64; ++q) {
-            const int j = n0 + 64 * q, tap = j / g.Cin;
+          for (int q = 0; q < B_GROUPS; ++q) {
+            const int j = n0 + 64 * ((int)rank * B_GROUPS + q), tap = j / g.Cin;
             grp_c[q] = j - tap * g.Cin; grp_r[q] = tap / 3; grp_s[q] = tap - 3 * (tap / 3);
           }
         }
@@ -141,6 +153,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int kb = kb0; kb < kb1; ++kb) {
         if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, g.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
         const uint32_t sa = smem_base + stage * STAGE, sb = sa + A_BYTES;
+        if (PAIR) {
+          // both CTAs' copies are counted on the issuing CTA's barrier, which announces all their bytes
+          const uint32_t full = map_to_cta(full_bar(stage), 0);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE);
+          tma_load_2d_pair(sa, &map_a, full, m0, kb * BK);
+          tma_load_2d_pair(sa + GROUP_BYTES, &map_a, full, m0 + 64, kb * BK);
+#pragma unroll
+          for (int q = 0; q < B_GROUPS; ++q)
+            tma_load_im2col_4d_pair(sb + q * GROUP_BYTES, &map_b, full, grp_c[q], w0 - 1, h0 - 1, img,
+                                    (uint16_t)grp_s[q], (uint16_t)grp_r[q]);
+          w0 += BK;
+          while (w0 >= g.W) { w0 -= g.W; if (++h0 == g.H) { h0 = 0; ++img; } }
+          ++fills[stage];
+          if (++stage == g.stages) { stage = 0; phase ^= 1; }
+          continue;
+        }
         mbar_expect_tx(full_bar(stage), BMODE == kMnMajorIm2colC8 ? A_BYTES + 9 * 1024 : STAGE);
         if (AMODE == kKMajor) {
           tma_load_2d(sa, &map_a, full_bar(stage), kb * BK, m0);
@@ -173,7 +201,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ++fills[stage];
         if (++stage == g.stages) { stage = 0; phase ^= 1; }
       }
-      if (!ok) {
+      if (!ok && rank != 0) {
+        // the peer's copies report to the issuing CTA's barriers: allow them a millisecond to land
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 1000000ull) {}
+      } else if (!ok) {
         for (int s = 0; s < g.stages; ++s)
           if (fills[s]) {
             const unsigned long long t0 = global_timer_ns();
@@ -182,9 +214,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, AMODE != kKMajor, BMODE != kKMajor);
-      constexpr uint32_t idesc_ones = umma_idesc_bf16(BM, 16, AMODE != kKMajor, false);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(PAIR ? 2 * BM : BM, BN, AMODE != kKMajor, BMODE != kKMajor);
+      constexpr uint32_t idesc_ones = umma_idesc_bf16(PAIR ? 2 * BM : BM, 16, AMODE != kKMajor, false);
       const uint64_t d_ones = smem_desc_plain(ones, 128, 256);  // every element is 1: the layout is immaterial
       int db_next = db_first;
       int stage = 0;
@@ -202,23 +234,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint64_t db = BMODE == kKMajor          ? smem_desc_sw128(sb, 16)
                             : BMODE == kMnMajorIm2colC8 ? smem_desc_plain(sb, 128, 1024)
                                                         : smem_desc_sw128(sb, GROUP_BYTES);
-        umma_bf16(tmem_base, da, db, idesc, kb > kb0 ? 1u : 0u);
+        if (PAIR) {
+          umma_bf16_pair(tmem_base, da, db, idesc, kb > kb0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 1; k < BK / 16; ++k)
-          umma_bf16_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), idesc);
-        if (kb == db_next) {
-          umma_bf16(tmem_base + BN, da, d_ones, idesc_ones, kb != db_first ? 1u : 0u);
+          for (int k = 1; k < BK / 16; ++k)
+            umma_bf16_pair_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), idesc);
+          if (kb == db_next) {
+            umma_bf16_pair(tmem_base + BN, da, d_ones, idesc_ones, kb != db_first ? 1u : 0u);
 #pragma unroll
-          for (int k = 1; k < BK / 16; ++k) umma_bf16_acc(tmem_base + BN, desc_advance(da, k * a_step), d_ones, idesc_ones);
-          db_next += g.n_tiles;
+            for (int k = 1; k < BK / 16; ++k)
+              umma_bf16_pair_acc(tmem_base + BN, desc_advance(da, k * a_step), d_ones, idesc_ones);
+            db_next += g.n_tiles;
+          }
+          umma_commit_pair(empty_bar(stage), 3);  // frees the stage in both CTAs
+        } else {
+          umma_bf16(tmem_base, da, db, idesc, kb > kb0 ? 1u : 0u);
+#pragma unroll
+          for (int k = 1; k < BK / 16; ++k)
+            umma_bf16_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), idesc);
+          if (kb == db_next) {
+            umma_bf16(tmem_base + BN, da, d_ones, idesc_ones, kb != db_first ? 1u : 0u);
+#pragma unroll
+            for (int k = 1; k < BK / 16; ++k) umma_bf16_acc(tmem_base + BN, desc_advance(da, k * a_step), d_ones, idesc_ones);
+            db_next += g.n_tiles;
+          }
+          umma_commit(empty_bar(stage));
         }
-        umma_commit(empty_bar(stage));
         if (++stage == g.stages) { stage = 0; phase ^= 1; }
       }
       if (ok) {
-        umma_commit(acc_bar);
+        if (PAIR) umma_commit_pair(acc_bar, 3); else umma_commit(acc_bar);
       } else {
-        umma_commit(drain_bar);
+        if (PAIR) umma_commit_pair(drain_bar, 1); else umma_commit(drain_bar);
         const unsigned long long t0 = global_timer_ns();
         while (!mbar_try_wait(drain_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
       }
@@ -291,10 +338,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   tc_fence_before();
   __syncthreads();
+  // a pair meets before either CTA releases tensor memory or exits: until then the peer may still
+  // signal this CTA's barriers, and the issuing CTA's MMAs read the peer's shared memory
+  if (PAIR) cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
@@ -344,8 +394,8 @@ int sm_count() {
 
 // K split: as many CTAs as fit in one wave (one CTA per SM: a second, partial wave would leave most
 // SMs idle for its whole duration), never an empty split.
-void plan_split(int mn_tiles, int k_blocks, int* splits, int* kb_per_split) {
-  int want = sm_count() / mn_tiles;
+void plan_split(int mn_tiles, int k_blocks, int* splits, int* kb_per_split, int ctas_per_tile = 1) {
+  int want = sm_count() / ctas_per_tile / mn_tiles;
   if (want < 1) want = 1;
   if (want > k_blocks) want = k_blocks;
   int per = (k_blocks + want - 1) / want;
@@ -353,23 +403,36 @@ void plan_split(int mn_tiles, int k_blocks, int* splits, int* kb_per_split) {
   *splits = (k_blocks + per - 1) / per;
 }
 
-template <int BN, int AMODE, int BMODE>
+// m_tiles counts tiles of 128 rows, or of 256 rows (CTA pairs) with PAIR
+template <int BN, int AMODE, int BMODE, bool PAIR = false>
 cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArgs g, int m_tiles, int splits,
                            cudaStream_t st) {
-  constexpr int STAGE = stage_bytes<BN>();
+  constexpr int STAGE = stage_bytes<BN, PAIR>();
   constexpr int kExtra = 1024 + 256 + 1024;  // alignment slack, barriers, block of ones
   constexpr int max_stages = (227 * 1024 - 3072) / STAGE > kMaxStages ? kMaxStages : (227 * 1024 - 3072) / STAGE;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, AMODE, BMODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, AMODE, BMODE, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          max_stages * STAGE + kExtra);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   g.stages = g.kb_per_split < max_stages ? g.kb_per_split : max_stages;
   const size_t smem = (size_t)g.stages * STAGE + kExtra;
+  if (PAIR) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * m_tiles * g.n_tiles, splits);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, AMODE, BMODE, PAIR>, ma, mb, g);
+  }
   dim3 grid(m_tiles * g.n_tiles, splits);
-  gemm_tc_kernel<BN, AMODE, BMODE><<<grid, kThreads, smem, st>>>(ma, mb, g);
+  gemm_tc_kernel<BN, AMODE, BMODE, PAIR><<<grid, kThreads, smem, st>>>(ma, mb, g);
   return cudaGetLastError();
 }
 
@@ -478,12 +541,16 @@ cudaError_t tc_dense_dw(const bf16* dY, const bf16* X, float* dW, int M, int In,
 namespace {
 // 9*Cin columns in tiles of whole 64-channel groups: 256 or 128 wide, and 192 (three taps) for 64 channels
 int wgrad_bn(int Cin) { return Cin % 256 == 0 ? 256 : (Cin % 128 == 0 ? 128 : 192); }
-void wgrad_plan(ConvShape s, int* m_tiles, int* n_tiles, int* k_blocks, int* splits, int* per) {
+// CTA pairs take 256 output channels per tile
+bool wgrad_pair(ConvShape s, bool pairs) { return pairs && s.Cout % 256 == 0 && s.Cin % 128 == 0; }
+// m_tiles: tiles of 128 output channels, or of 256 with CTA pairs
+void wgrad_plan(ConvShape s, bool pairs, int* m_tiles, int* n_tiles, int* k_blocks, int* splits, int* per) {
   const long P = (long)s.N * s.H * s.W;
-  *m_tiles = (s.Cout + BM - 1) / BM;
+  const bool pair = wgrad_pair(s, pairs);
+  *m_tiles = pair ? s.Cout / 256 : (s.Cout + BM - 1) / BM;
   *n_tiles = 9 * s.Cin / wgrad_bn(s.Cin);
   *k_blocks = (int)((P + BK - 1) / BK);
-  plan_split(*m_tiles * *n_tiles, *k_blocks, splits, per);
+  plan_split(*m_tiles * *n_tiles, *k_blocks, splits, per, pair ? 2 : 1);
 }
 }  // namespace
 
@@ -491,23 +558,23 @@ bool tc_wgrad_supported(ConvShape s) {
   return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.H >= 2 && s.W >= 2 && (long)s.N * s.H * s.W < (1L << 31) - 256;
 }
 
-size_t tc_wgrad_scratch_elems(ConvShape s) {
+size_t tc_wgrad_scratch_elems(ConvShape s, bool pairs) {
   if (!tc_wgrad_supported(s)) return 0;
   int mt, nt, kb, splits, per;
-  wgrad_plan(s, &mt, &nt, &kb, &splits, &per);
+  wgrad_plan(s, pairs, &mt, &nt, &kb, &splits, &per);
   return (size_t)splits * s.Cout * 9 * s.Cin + (size_t)splits * nt * s.Cout;
 }
 
-int tc_wgrad_launches(ConvShape s, bool with_db) {
+int tc_wgrad_launches(ConvShape s, bool with_db, bool pairs) {
   int mt, nt, kb, splits, per;
-  wgrad_plan(s, &mt, &nt, &kb, &splits, &per);
+  wgrad_plan(s, pairs, &mt, &nt, &kb, &splits, &per);
   return splits > 1 || with_db ? 2 : 1;
 }
 
 // dW[k][tap][c] = sum_pixels dz[pixel][k] * x[pixel + tap][c]   (fp32 out, [Cout][9*Cin]);
 // db[k] = sum_pixels dz[pixel][k] when db is not null
 cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* db, float* partial, ConvShape s,
-                             int* dev_error, cudaStream_t st) {
+                             int* dev_error, cudaStream_t st, bool pairs) {
   if (!tc_wgrad_supported(s)) return cudaErrorInvalidValue;
   const long P = (long)s.N * s.H * s.W;
   const int BN = wgrad_bn(s.Cin);
@@ -516,15 +583,22 @@ cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* db
   if (!make_im2col_map(&mb, x, s.N, s.H, s.W, s.Cin, 64)) return cudaErrorInvalidValue;
   GemmArgs g{};
   int m_tiles, splits;
-  wgrad_plan(s, &m_tiles, &g.n_tiles, &g.k_blocks, &splits, &g.kb_per_split);
+  wgrad_plan(s, pairs, &m_tiles, &g.n_tiles, &g.k_blocks, &splits, &g.kb_per_split);
   g.M = s.Cout; g.N = 9 * s.Cin; g.H = s.H; g.W = s.W; g.Cin = s.Cin;
   g.dev_error = dev_error; g.ldc = g.N;
   if (splits == 1) g.out_f = dW; else g.partial = partial;
   if (db) g.db_partial = partial + (splits == 1 ? 0 : (size_t)splits * s.Cout * 9 * s.Cin);
   cudaError_t e;
+  const bool pair = wgrad_pair(s, pairs);
   switch (BN) {
-    case 256: e = launch_gemm_tc<256, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
-    case 128: e = launch_gemm_tc<128, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
+    case 256:
+      e = pair ? launch_gemm_tc<256, kMnMajor, kMnMajorIm2col, true>(ma, mb, g, m_tiles, splits, st)
+               : launch_gemm_tc<256, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st);
+      break;
+    case 128:
+      e = pair ? launch_gemm_tc<128, kMnMajor, kMnMajorIm2col, true>(ma, mb, g, m_tiles, splits, st)
+               : launch_gemm_tc<128, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st);
+      break;
     default: e = launch_gemm_tc<192, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
   }
   if (e != cudaSuccess) return e;

@@ -37,11 +37,13 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const floa
 // K = pixels (both operands read transposed, x through the im2col window):
 // dW fp32 [Cout][3][3][Cin]; db fp32 [Cout] = column sums of dz from the same GEMM (a block of
 // ones as a second B operand), or null.  partial: fp32 scratch of tc_wgrad_scratch_elems().
+// pairs: let CTA pairs (256 output channels per tile, each CTA staging half of the x tile) take the
+// shapes that allow it; the scratch size and launch count are asked for with the same value.
 bool tc_wgrad_supported(ConvShape s);
-size_t tc_wgrad_scratch_elems(ConvShape s);
-int tc_wgrad_launches(ConvShape s, bool with_db);
+size_t tc_wgrad_scratch_elems(ConvShape s, bool pairs = true);
+int tc_wgrad_launches(ConvShape s, bool with_db, bool pairs = true);
 cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* db, float* partial, ConvShape s,
-                             int* dev_error, cudaStream_t st);
+                             int* dev_error, cudaStream_t st, bool pairs = true);
 
 // Dense layers on the same GEMM kernel.  X [M][In], W [Out][In], dY [M][Out].
 bool tc_dense_supported(int M, int In, int Out);

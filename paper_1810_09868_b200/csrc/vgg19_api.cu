@@ -129,7 +129,7 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
     }
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
     size_t pe = simt_wgrad_scratch_elems(s);
-    size_t te = tc_wgrad_scratch_elems(s);
+    size_t te = tc_wgrad_scratch_elems(s, n->use_pair);
     if (te > pe) pe = te;
     if (pe > max_partial) max_partial = pe;
   }
@@ -240,8 +240,8 @@ struct Pass {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       ok(tc_first_wgrad((const bf16 *)buf(p.x8), (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st), 2);
     } else if (n->use_tc && tc_wgrad_supported(s)) {
-      ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st),
-         tc_wgrad_launches(s, db != nullptr));
+      ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st, n->use_pair),
+         tc_wgrad_launches(s, db != nullptr, n->use_pair));
     } else
       ok(simt_conv3x3_wgrad<T>(x, dz, dW, db, fbuf(p.partial), s, st), 4);
     if (dx) {
