@@ -286,7 +286,7 @@ def run_native(args):
         bwd()  # leaves the batch-100 activations of every layer in the workspace
     stream.synchronize()
     layers = time_conv_layers(pkg, net, torch, stream)
-    # dominant kernel: conv3x3_tc_kernel<256>, the 12 launches of layers 5..16 (about half the pass)
+    # dominant kernel: conv3x3_pair_tc_kernel<256>, the 12 launches of layers 5..16 (60 % of the pass)
     dom = [t for t in layers if t[0] >= 5]
     conv_ms = sum(ms for _, ms, _, _ in dom)
     conv_flop = sum(f for _, _, f, _ in dom)
@@ -297,8 +297,8 @@ def run_native(args):
     per_layer = {f"conv{l}": {"ms": round(ms, 4), "tflops": round(f / (ms * 1e-3) / 1e12, 1), "path": path}
                  for l, ms, f, path in layers}
     # dram__bytes_read+write of one launch of this kernel on layer 6 (56x56, 256->256), captured with
-    # ncu at batch 48 (112.9 MB) and scaled by the pixel count to the batch-100 launch timed here
-    traffic = 112.87e6 * BATCH / 48
+    # ncu at batch 48 (113.7 MB) and scaled by the pixel count to the batch-100 launch timed here
+    traffic = 113.70e6 * BATCH / 48
 
     n_fwd = pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_FORWARD)
     cpu_rate, cpu_dt = oracle_forward_rate(args.cpu_images)
@@ -323,8 +323,8 @@ def run_native(args):
                     "launches_per_step": pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_BACKWARD)},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": traffic,
-                     "kernel": "conv3x3_tc_kernel<256>: 3x3 convolution forward as a tcgen05 implicit GEMM, "
-                               "layers 5..16 (12 launches per pass), algorithmic flops / summed launch time",
+                     "kernel": "conv3x3_pair_tc_kernel<256>: 3x3 convolution forward as a tcgen05 cta_group::2 implicit "
+                               "GEMM on CTA pairs, layers 5..16 (12 launches per pass), algorithmic flops / summed launch time",
                      "traffic_note": "DRAM bytes of the layer-6 launch (algorithmic: 160.6 MB in + 160.6 MB out "
                                      "+ 1.2 MB filter at batch 100); the output is still in L2 when the launch ends",
                      "peak_source": f"{pk['source']} burst bf16 GEMM (kernel timed alone per layer)",
