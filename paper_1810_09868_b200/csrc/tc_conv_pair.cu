@@ -52,7 +52,27 @@ struct PairArgs {
   const float* bias;
   const bf16* mask;
   int* dev_error;
+  // Tail split.  The first main_tiles tiles are whole rounds of the resident pairs; the rest (fewer
+  // than half a round) are each cut into tail_splits ranges of tail_kb K blocks so that the last
+  // round keeps every pair busy for a fraction of a tile's time.  Those work items leave raw fp32
+  // sums in `partial` ([split][tail_rows][Cout], rows counted from pixel tail_row0) for
+  // pair_tail_finish_kernel.  main_tiles = all tiles when there is no tail.
+  int main_tiles, tail_splits, tail_kb;
+  int tail_row0, tail_rows;
+  float* partial;
 };
+
+// One unit of a pair's work: a whole tile (split < 0) or a range of a tail tile's K blocks.
+struct Work {
+  int tile, kb0, kb1, split;
+};
+__device__ __forceinline__ Work get_work(int w, const PairArgs& a, int k_blocks) {
+  if (w < a.main_tiles) return Work{w, 0, k_blocks, -1};
+  const int j = w - a.main_tiles;
+  const int t = j / a.tail_splits, z = j - t * a.tail_splits;
+  const int kb0 = z * a.tail_kb;
+  return Work{a.main_tiles + t, kb0, min(k_blocks, kb0 + a.tail_kb), z};
+}
 
 template <int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
@@ -77,7 +97,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const bool leader = rank == 0;
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int k_blocks = 9 * a.cin_blocks;
-  const int total_tiles = a.m_pairs * a.n_tiles;
+  const int total_work = a.main_tiles + (a.m_pairs * a.n_tiles - a.main_tiles) * a.tail_splits;
 
   for (int i = threadIdx.x; i < a.Cout; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
   if (threadIdx.x == 0) {
@@ -108,8 +128,9 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
-        const int m_pair = tile / a.n_tiles, n_tile = tile - m_pair * a.n_tiles;
+      for (int w = pair; w < total_work && ok; w += n_pairs) {
+        const Work wk = get_work(w, a, k_blocks);
+        const int m_pair = wk.tile / a.n_tiles, n_tile = wk.tile - m_pair * a.n_tiles;
         // a CTA whose 128 pixels all lie past the end of the tensor (odd tile count) stages the
         // tensor's first pixels instead: its accumulator rows are never stored
         int p0 = (2 * m_pair + (int)rank) * BM;
@@ -117,20 +138,21 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const int w0 = p0 % a.W, t = p0 / a.W;
         const int h0 = t % a.H, n0 = t / a.H;
         const int filter_row = n_tile * BN + (int)rank * (BN / 2);
-        int kb = 0;
-        for (int r = 0; r < 3 && ok; ++r)
-          for (int s = 0; s < 3 && ok; ++s)
-            for (int cb = 0; cb < a.cin_blocks; ++cb, ++kb) {
-              if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
-              const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
-              const uint32_t full = map_to_cta(full_bar(stage), 0);
-              // the even CTA announces the bytes of both CTAs' copies for this stage
-              if (leader) mbar_expect_tx(full_bar(stage), 2 * T::STAGE_BYTES);
-              tma_load_im2col_4d_pair(sa, &map_x, full, cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
-              tma_load_2d_pair(sb, &map_w, full, kb * BK, filter_row);
-              ++fills[stage];
-              if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
-            }
+        // K block kb = (tap (r, s), channel block cb), channel blocks fastest
+        const int tap0 = wk.kb0 / a.cin_blocks;
+        int cb = wk.kb0 - tap0 * a.cin_blocks, r = tap0 / 3, s = tap0 - 3 * (tap0 / 3);
+        for (int kb = wk.kb0; kb < wk.kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
+          const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
+          const uint32_t full = map_to_cta(full_bar(stage), 0);
+          // the even CTA announces the bytes of both CTAs' copies for this stage
+          if (leader) mbar_expect_tx(full_bar(stage), 2 * T::STAGE_BYTES);
+          tma_load_im2col_4d_pair(sa, &map_x, full, cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
+          tma_load_2d_pair(sb, &map_w, full, kb * BK, filter_row);
+          ++fills[stage];
+          if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
+          if (++cb == a.cin_blocks) { cb = 0; if (++s == 3) { s = 0; ++r; } }
+        }
       }
       if (!ok) {
         // let every copy already in flight land before the CTA may go on to exit: the even CTA sees
@@ -155,18 +177,19 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++local) {
+      for (int w = pair; w < total_work && ok; w += n_pairs, ++local) {
+        const Work wk = get_work(w, a, k_blocks);
         const int buf = local & 1;
         const uint32_t use = (uint32_t)(local >> 1);
         if (!mbar_wait(acc_empty_bar(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = wk.kb0; kb < wk.kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
           const uint64_t da = smem_desc_sw128(sa, 16), db = smem_desc_sw128(sb, 16);
-          umma_bf16_pair(d_tmem, da, db, idesc, kb != 0 ? 1u : 0u);
+          umma_bf16_pair(d_tmem, da, db, idesc, kb != wk.kb0 ? 1u : 0u);
 #pragma unroll
           for (int k = 1; k < BK / 16; ++k)
             umma_bf16_pair_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
@@ -188,10 +211,11 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     int local = 0;
     const bool issuer = threadIdx.x == 64;  // owns the TMA store groups
     uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
-    for (int tile = pair; tile < total_tiles; tile += n_pairs, ++local) {
+    for (int w = pair; w < total_work; w += n_pairs, ++local) {
+      const Work wk = get_work(w, a, k_blocks);
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
-      const int m_pair = tile / a.n_tiles, n_tile = tile - m_pair * a.n_tiles;
+      const int m_pair = wk.tile / a.n_tiles, n_tile = wk.tile - m_pair * a.n_tiles;
       const int m_tile = 2 * m_pair + (int)rank;
       const bool got = mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
       if (named_bar_or(1, 128, !got)) break;  // all four warps leave together
@@ -201,6 +225,25 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       const bool tile_valid = (long)m_tile * BM < a.pixels;
       const int c_base = n_tile * BN;
       const bf16* mask_row = (a.mask && valid) ? a.mask + pixel * a.Cout + c_base : nullptr;
+      if (wk.split >= 0) {
+        // part of a tail tile's K range: raw sums, one row per thread, for the finishing kernel
+        float* dst = a.partial + ((size_t)wk.split * a.tail_rows + (size_t)(pixel - a.tail_row0)) * a.Cout + c_base;
+#pragma unroll 1
+        for (int cc = 0; cc < BN && tile_valid; cc += 32) {
+          uint32_t v[32];
+          tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+          tmem_ld_wait();
+          if (valid) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(dst + cc + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                     __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+          }
+        }
+        tc_fence_before();
+        mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
+        continue;
+      }
 #pragma unroll 1
       for (int c64 = 0; c64 < BN && tile_valid; c64 += 64) {
         if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
@@ -270,10 +313,50 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   }
 }
 
+// out[row][c] = epilogue(sum over splits of partial[split][row][c]) for the rows of the tail tiles
+// (out, mask already point at the first tail row); eight channels per thread, splits added in order.
+__global__ void pair_tail_finish_kernel(const float* __restrict__ partial, int splits, long elems, int Cout,
+                                        const float* __restrict__ bias, int relu, const bf16* __restrict__ mask,
+                                        bf16* __restrict__ out) {
+  const long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  if (i >= elems) return;
+  float x[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int z = 0; z < splits; ++z) {
+    const float4 p0 = *reinterpret_cast<const float4*>(partial + (long)z * elems + i);
+    const float4 p1 = *reinterpret_cast<const float4*>(partial + (long)z * elems + i + 4);
+    x[0] += p0.x; x[1] += p0.y; x[2] += p0.z; x[3] += p0.w;
+    x[4] += p1.x; x[5] += p1.y; x[6] += p1.z; x[7] += p1.w;
+  }
+  const int c = (int)(i % Cout);
+  uint32_t packed[4];
+#pragma unroll
+  for (int e = 0; e < 8; e += 2) {
+    float x0 = x[e], x1 = x[e + 1];
+    if (bias) { x0 += bias[c + e]; x1 += bias[c + e + 1]; }
+    if (relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
+    __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+    packed[e >> 1] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  if (mask) {
+    const uint4 m = *reinterpret_cast<const uint4*>(mask + i);
+    const uint32_t mw[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint32_t lo = mw[e] & 0xFFFFu, hi = mw[e] >> 16;
+      uint32_t keep = 0;
+      if (lo != 0 && !(lo & 0x8000u)) keep |= 0x0000FFFFu;
+      if (hi != 0 && !(hi & 0x8000u)) keep |= 0xFFFF0000u;
+      packed[e] &= keep;
+    }
+  }
+  *reinterpret_cast<uint4*>(out + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+}
+
+// CTA pairs of this kernel that can be resident at once (one pair per two SMs at most)
 template <int BN>
-cudaError_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, PairArgs a, cudaStream_t st) {
+cudaError_t resident_pairs(int* out) {
   using T = PairTile<BN>;
-  static int max_pairs = 0;  // CTA pairs that can be resident at once
+  static int max_pairs = 0;
   if (!max_pairs) {
     cudaError_t e = cudaFuncSetAttribute(conv3x3_pair_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
     if (e != cudaSuccess) return e;
@@ -292,12 +375,13 @@ cudaError_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
     e = cudaOccupancyMaxActiveClusters(&n, conv3x3_pair_tc_kernel<BN>, &cfg);
     if (e != cudaSuccess || n < 1) { cudaGetLastError(); n = sms / 2; }
     max_pairs = n < sms / 2 ? n : sms / 2;
+    if (max_pairs < 1) max_pairs = 1;
   }
-  const int tiles = a.m_pairs * a.n_tiles;
-  const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  conv3x3_pair_tc_kernel<BN><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
-  return cudaGetLastError();
+  *out = max_pairs;
+  return cudaSuccess;
 }
+
+constexpr int kTailMaxPairs = 128;  // bound used to size the tail scratch (SMs / 2 on any device this runs on)
 
 }  // namespace
 
@@ -306,10 +390,17 @@ bool tc_conv3x3_pair_supported(ConvShape s) {
          (long)s.N * s.H * s.W < (1L << 31) - 512;
 }
 
+size_t tc_conv3x3_pair_scratch_elems(ConvShape s) {
+  // at most one work item per resident pair, each 256 rows x 256 columns of fp32
+  return tc_conv3x3_pair_supported(s) ? (size_t)kTailMaxPairs * 2 * BM * 256 : 0;
+}
+
 cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out, ConvShape s,
-                            bool relu, int* dev_error, cudaStream_t st) {
+                            bool relu, int* dev_error, cudaStream_t st, float* partial, int* launches) {
+  if (launches) *launches = 0;
   if (!tc_conv3x3_pair_supported(s)) return cudaErrorInvalidValue;
   constexpr int BN = 256;
+  using T = PairTile<BN>;
   CUtensorMap mx, mw, my;
   if (!make_im2col_map(&mx, in, s.N, s.H, s.W, s.Cin, BM)) return cudaErrorInvalidValue;
   if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, BN / 2)) return cudaErrorInvalidValue;
@@ -323,7 +414,41 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0;
   a.bias = bias; a.mask = mask; a.dev_error = dev_error;
-  return launch_pair<BN>(mx, mw, my, a, st);
+  int cap = 0;
+  cudaError_t e = resident_pairs<BN>(&cap);
+  if (e != cudaSuccess) return e;
+  const int tiles = a.m_pairs * a.n_tiles, k_blocks = 9 * a.cin_blocks;
+  a.main_tiles = tiles; a.tail_splits = 1; a.tail_kb = k_blocks; a.tail_row0 = 0; a.tail_rows = 0; a.partial = nullptr;
+  // Whole rounds of `cap` tiles, then a tail of fewer than half a round: cut each tail tile's K range
+  // so that the last round occupies (nearly) every pair for 1/splits of a tile's time.
+  const int rounds = tiles / cap, left = tiles - rounds * cap;
+  if (partial && rounds >= 1 && left > 0 && 2 * left <= cap && cap <= kTailMaxPairs && (rounds * cap) % a.n_tiles == 0) {
+    int splits = cap / left;
+    if (splits > k_blocks) splits = k_blocks;
+    const int per = (k_blocks + splits - 1) / splits;
+    splits = (k_blocks + per - 1) / per;
+    // The pieces cost a second kernel and a round trip of fp32 partial sums (about the time of 50 K
+    // blocks at batch 100): only worth it when the shortened round saves more than that.
+    if (splits >= 2 && k_blocks - per >= 56) {
+      a.main_tiles = rounds * cap;
+      a.tail_splits = splits; a.tail_kb = per;
+      a.tail_row0 = (a.main_tiles / a.n_tiles) * 2 * BM;
+      a.tail_rows = a.pixels - a.tail_row0;
+      a.partial = partial;
+    }
+  }
+  const int work = a.main_tiles + (tiles - a.main_tiles) * a.tail_splits;
+  const int pairs = work < cap ? work : cap;
+  conv3x3_pair_tc_kernel<BN><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
+  e = cudaGetLastError();
+  if (launches) *launches = 1;
+  if (e != cudaSuccess || !a.partial) return e;
+  const long elems = (long)a.tail_rows * a.Cout;
+  const size_t row_off = (size_t)a.tail_row0 * a.Cout;
+  pair_tail_finish_kernel<<<(unsigned)((elems / 8 + 255) / 256), 256, 0, st>>>(
+      partial, a.tail_splits, elems, a.Cout, bias, a.relu, mask ? mask + row_off : nullptr, out + row_off);
+  if (launches) *launches = 2;
+  return cudaGetLastError();
 }
 
 }  // namespace vgg

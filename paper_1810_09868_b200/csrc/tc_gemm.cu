@@ -68,8 +68,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   static_assert(!PAIR || (AMODE == kMnMajor && BMODE == kMnMajorIm2col && BN % 128 == 0), "pairs: filter gradient only");
   constexpr int STAGE = stage_bytes<BN, PAIR>();
   constexpr int B_GROUPS = (PAIR ? BN / 2 : BN) / 64;  // 64-column groups of B this CTA stages
-  // 32 spare columns after the tile where the column sums of A can accumulate
-  constexpr int TMEM_COLS = BN + 32 <= 64 ? 64 : (BN + 32 <= 128 ? 128 : (BN + 32 <= 256 ? 256 : 512));
+  // filter gradient: 32 spare columns after the tile where the column sums of A can accumulate.  The
+  // dense layers need none, and with 256 columns instead of 512 two of their CTAs share an SM.
+  constexpr int COLS = BN + (BMODE == kMnMajorIm2col ? 32 : 0);
+  constexpr int TMEM_COLS = COLS <= 64 ? 64 : (COLS <= 128 ? 128 : (COLS <= 256 ? 256 : 512));
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = smem_base + g.stages * STAGE;
@@ -90,7 +92,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int kb1 = min(g.k_blocks, kb0 + g.kb_per_split);
   // K blocks kb = n_tile (mod n_tiles) are the ones whose column sums this CTA adds
   int db_first = kb1;
-  if (g.db_partial) {
+  if (BMODE == kMnMajorIm2col && g.db_partial) {
     int r = n_tile - kb0 % g.n_tiles;
     if (r < 0) r += g.n_tiles;
     db_first = kb0 + r;
@@ -326,7 +328,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
       }
-      if (g.db_partial) {
+      if (BMODE == kMnMajorIm2col && g.db_partial) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)BN, v);
         tmem_ld_wait();

@@ -19,9 +19,15 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
 
 // The same convolution on CTA pairs (tc_conv_pair.cu): a cluster of two CTAs per 256-pixel x 256-channel
 // tile, each staging half of the filter slice.  Cout must be a multiple of 256.
+// partial (or null): fp32 scratch of tc_conv3x3_pair_scratch_elems() elements.  With it, when the tile count
+// leaves a last round less than half full, the tiles of that round are cut along K over all the
+// pairs and a second kernel adds the pieces (in a fixed order) and applies the epilogue.
+// launches (or null) receives the number of kernels launched (1 or 2).
 bool tc_conv3x3_pair_supported(ConvShape s);
+size_t tc_conv3x3_pair_scratch_elems(ConvShape s);
 cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, const bf16* mask,
-                            bf16* out, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
+                            bf16* out, ConvShape s, bool relu, int* dev_error, cudaStream_t st,
+                            float* partial = nullptr, int* launches = nullptr);
 
 // The same convolution with the input patch (plus halo) kept in shared memory
 // for all nine taps (tc_conv_halo.cu): the large-image, few-channel layers.

@@ -117,7 +117,7 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   int pi = 0;
-  size_t max_act = 0, max_low = 0, max_partial = 0;
+  size_t max_act = 0, max_low = 0, max_partial = 0, conv_fwd_partial = 0;
   for (int l = 0; l < kConvLayers; ++l) {
     const ConvLayer &c = n->conv[l];
     size_t a = (size_t)B * c.H * c.W * c.Cout;
@@ -132,6 +132,13 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
     size_t te = tc_wgrad_scratch_elems(s, n->use_pair);
     if (te > pe) pe = te;
     if (pe > max_partial) max_partial = pe;
+    // tail-split scratch of the two-CTA convolution (forward, and input gradient with the channels swapped)
+    if (n->use_pair) {
+      size_t fe = tc_conv3x3_pair_scratch_elems(s), de = tc_conv3x3_pair_scratch_elems(ConvShape{B, c.H, c.W, c.Cout, c.Cin});
+      if (fe > conv_fwd_partial) conv_fwd_partial = fe;
+      if (fe > max_partial) max_partial = fe;
+      if (de > max_partial) max_partial = de;
+    }
   }
   p.x8 = take(n->use_tc ? (size_t)B * n->cfg.height * n->cfg.width * 16 : 0);
   {
@@ -149,6 +156,7 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
     if (e > dense_partial) dense_partial = e;
   }
   if (1024 * 512 > max_partial) max_partial = 1024 * 512;  // bias-gradient column sums
+  if (conv_fwd_partial > dense_partial) dense_partial = conv_fwd_partial;
   if (mode == VGG19_MODE_FORWARD) p.partial = take(dense_partial * 4);
   if (dense_partial > max_partial) max_partial = dense_partial;
   if (mode == VGG19_MODE_BACKWARD) {
@@ -195,6 +203,10 @@ struct Pass {
   int launches = 0;
   cudaError_t err = cudaSuccess;
   bool keep_activations = true;  // false in a forward-only pass: nothing will read a pre-pool output again
+  // Whether a forward convolution may cut the tiles of its last round along K.  That changes the fp32
+  // summation order of the images in those tiles with the batch size, so a training pass, whose ReLU and
+  // pooling decisions should not depend on what else is in the batch, keeps it off for its forward half.
+  bool forward_tail_split = true;
 
   T *buf(size_t off) const { return reinterpret_cast<T *>(static_cast<char *>(n->ws) + off); }
   float *fbuf(size_t off) const { return reinterpret_cast<float *>(static_cast<char *>(n->ws) + off); }
@@ -220,10 +232,12 @@ struct Pass {
       ok(tc_conv3x3_halo((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
                          (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st), 1);
       return;
-    } else if (pair_ok(s))
+    } else if (pair_ok(s)) {
+      int k = 1;
       ok(tc_conv3x3_pair((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
-                         (bf16 *)y, s, true, n->dev_error, st), 1);
-    else if (tc_conv_ok(s))
+                         (bf16 *)y, s, true, n->dev_error, st, p.valid && forward_tail_split ? fbuf(p.partial) : nullptr, &k), 0);
+      launches += k;
+    } else if (tc_conv_ok(s))
       ok(tc_conv3x3((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
                     (bf16 *)y, s, true, n->dev_error, st), 1);
     else
@@ -250,10 +264,12 @@ struct Pass {
       if (n->use_tc && tc_conv3x3_halo_supported(t))
         ok(tc_conv3x3_halo((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr, t,
                            false, n->dev_error, st), 1);
-      else if (pair_ok(t))
+      else if (pair_ok(t)) {
+        int k = 1;
         ok(tc_conv3x3_pair((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
-                           t, false, n->dev_error, st), 1);
-      else if (tc_conv_ok(t))
+                           t, false, n->dev_error, st, p.valid ? fbuf(p.partial) : nullptr, &k), 0);
+        launches += k;
+      } else if (tc_conv_ok(t))
         ok(tc_conv3x3((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
                       t, false, n->dev_error, st), 1);
       else
@@ -358,7 +374,13 @@ int check_batch(vgg19 *n, int batch, int mode, size_t extra) {
 template <typename T>
 int enqueue(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st, int *launches) {
   Pass<T> pass{n, make_plan(n, a.batch, mode), st};
-  if (mode == VGG19_MODE_FORWARD) { pass.keep_activations = false; pass.forward(a); } else pass.backward(a);
+  if (mode == VGG19_MODE_FORWARD) {
+    pass.keep_activations = false;
+    pass.forward(a);
+  } else {
+    pass.forward_tail_split = false;
+    pass.backward(a);
+  }
   if (launches) *launches = pass.launches;
   n->launches[mode] = pass.launches;
   if (pass.err != cudaSuccess)

@@ -89,3 +89,43 @@ def test_conv_layer_backward(net224, layer, S, Cin, Cout):
     if dx is not None:
         ref = oracle.round_bf16(oracle.conv3x3_dgrad(dz, Wt))
         assert rel_l2(dx.float().cpu().numpy(), ref) <= 1e-3
+
+
+@pytest.mark.parametrize("layer,S,Cin,Cout", [(13, 14, 512, 512), (9, 28, 256, 512)])
+def test_conv_layer_tail_round_batch100(layer, S, Cin, Cout):
+    """At batch 100 the tile count of these layers leaves a last round of CTA pairs less than half full;
+    where that saves enough (layer 13 forward and input gradient, layer 9 input gradient) its tiles
+    are cut along K over all pairs and summed by a second kernel.  The images in those tiles (the
+    last of the batch) and a few from whole rounds are checked against the checker, forward and
+    input gradient, and the whole batch against the one-CTA-per-tile kernels."""
+    import paper_1810_09868_b200 as p
+    B = 100
+    params = si.vgg19_params(224, 224, seed=0, bias_std=0.1, bf16_exact=True)
+    x = layer_input(layer, B, S, Cin)
+    dz = si.normal(B * S * S * Cout, seed=200 + layer, stddev=1e-3, bf16_exact=True).reshape(B, S, S, Cout)
+    xd = torch.from_numpy(x).to(DEV).to(torch.bfloat16)
+    dzd = torch.from_numpy(dz).to(DEV).to(torch.bfloat16)
+    sample = [0, 50, 96, 97, 98, 99]
+    outs = {}
+    for flags in (0, p.binding.VGG19_FLAG_NO_CTA_PAIRS):
+        net = p.Net(224, 224, B, p.VGG19_BF16, params=params, flags=flags)
+        y = torch.full((B, S, S, Cout), float("nan"), dtype=torch.bfloat16, device=DEV)
+        dx = torch.full((B, S, S, Cin), float("nan"), dtype=torch.bfloat16, device=DEV)
+        dw = torch.empty((Cout, 3, 3, Cin), dtype=torch.float32, device=DEV)
+        db = torch.empty((Cout,), dtype=torch.float32, device=DEV)
+        p.vgg19_conv_layer_forward(net.handle, layer, xd, B, y, None, torch.cuda.current_stream())
+        p.vgg19_conv_layer_backward(net.handle, layer, xd, dzd, B, dw, db, dx, torch.cuda.current_stream())
+        net.sync_status()
+        outs[flags] = (y.float().cpu().numpy(), dx.float().cpu().numpy())
+        Wt, b = layer_params(p, net, params, layer)
+        net.close()
+    y, dx = outs[0]
+    assert np.isfinite(y).all() and np.isfinite(dx).all()
+    ref_y = oracle.round_bf16(oracle.relu_fwd(oracle.conv3x3_fwd(x[sample], Wt, b)))
+    ref_dx = oracle.round_bf16(oracle.conv3x3_dgrad(dz[sample], Wt))
+    for row, i in enumerate(sample):
+        assert rel_l2(y[i], ref_y[row]) <= 1e-3, i
+        assert rel_l2(dx[i], ref_dx[row]) <= 1e-3, i
+    # against the single-CTA kernels over the whole batch: rare one-ulp rounding flips only
+    assert rel_l2(y, outs[p.binding.VGG19_FLAG_NO_CTA_PAIRS][0]) <= 1e-3
+    assert rel_l2(dx, outs[p.binding.VGG19_FLAG_NO_CTA_PAIRS][1]) <= 1e-3
