@@ -20,6 +20,12 @@
 //
 // Warps: 0 patch producer, 1 MMA issuer + TMEM owner, 2-5 epilogue, 6 filter
 // producer.  Accumulator double-buffered; persistent CTAs; time-limited waits.
+//
+// PAIR: two CTAs (a cluster, tcgen05 cta_group::2) work as one: each loads the patch of its own
+// tile and HALF of the filter's output channels, the even CTA issues MMAs of 256 rows (both
+// patches) whose B operand the hardware gathers from both CTAs, and each CTA finds its 128
+// accumulator rows in its own tensor memory.  With 128 output channels one CTA's MMA reads 8 KB of
+// shared memory per 64 cycles, all the bandwidth there is; as a pair it reads 6 KB.
 #include "tc_common.cuh"
 #include "tc_kernels.cuh"
 
@@ -34,10 +40,12 @@ constexpr int IW = PW + 2, IH = PH + 2;         // input patch with halo
 constexpr int A_BYTES = IW * IH * 128;          // 23040
 constexpr int A_SLOT = 23 * 1024;               // 1024-byte aligned slot
 constexpr int kThreads = 224;
+constexpr int kMaxPatchSlots = 6;
 
-template <int BN>
+template <int BN, bool PAIR>
 struct HaloTile {
-  static constexpr int TAP_BYTES = BN * BK * 2;   // one tap's BN x 64 filter slice
+  static constexpr int BNH = PAIR ? BN / 2 : BN;  // filter rows (output channels) this CTA stages per tap
+  static constexpr int TAP_BYTES = BNH * BK * 2;  // one tap's slice of the filter
   static constexpr int B_BYTES = 3 * TAP_BYTES;   // a filter row: three taps
   static constexpr int OUT_BYTES = BM * 64 * 2;   // staging tile of the TMA store; a second one holds the mask tile
   // Shared memory: `na` input-patch slots, the filter region, two staging tiles, barriers.  The filter
@@ -62,13 +70,16 @@ struct HaloArgs {
   int* dev_error;
 };
 
-template <int BN>
+template <int BN, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_m,
                        HaloArgs a) {
-  using T = HaloTile<BN>;
-  constexpr int NA = 3, NB = 4;  // most slots a plan may use (barrier numbering)
+  using T = HaloTile<BN, PAIR>;
+  constexpr int NA = kMaxPatchSlots, NB = 4;  // most slots a plan may use (barrier numbering)
+  // Accumulator buffers in tensor memory.  A tile here lasts a microsecond or two, about as long as
+  // the hand-off to the epilogue and back takes, so two buffers leave the tensor pipe waiting.
+  constexpr int NACC = 4;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_base = smem_base + a.na * A_SLOT;
@@ -80,23 +91,29 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   auto b_full = [&](int s) { return bars + 8u * (2 * NA + s); };
   auto b_empty = [&](int s) { return bars + 8u * (2 * NA + NB + s); };
   auto acc_full = [&](int b) { return bars + 8u * (2 * NA + 2 * NB + b); };
-  auto acc_empty = [&](int b) { return bars + 8u * (2 * NA + 2 * NB + 2 + b); };
-  const uint32_t drain_bar = bars + 8u * (2 * NA + 2 * NB + 4);
-  const uint32_t mask_bar = bars + 8u * (2 * NA + 2 * NB + 5);
-  const uint32_t w_bar = bars + 8u * (2 * NA + 2 * NB + 6);  // resident filter loaded
+  auto acc_empty = [&](int b) { return bars + 8u * (2 * NA + 2 * NB + NACC + b); };
+  const uint32_t drain_bar = bars + 8u * (2 * NA + 2 * NB + 2 * NACC);
+  const uint32_t mask_bar = bars + 8u * (2 * NA + 2 * NB + 2 * NACC + 1);
+  const uint32_t w_bar = bars + 8u * (2 * NA + 2 * NB + 2 * NACC + 2);  // resident filter loaded
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ __align__(16) float bias_s[512];  // the layer's bias (zeros when it has none)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = a.m_tiles * a.n_tiles;
+  // Work units: tiles, or with PAIR two tiles side by side in the tile order (m_tiles is even).
+  // Barriers the MMA issuer waits on (patch, filter, accumulator drained) are the even CTA's.
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int first_unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int unit_stride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int total_units = (PAIR ? a.m_tiles / 2 : a.m_tiles) * a.n_tiles;
+  auto unit_m_tile = [&](int u) { return PAIR ? 2 * (u / a.n_tiles) + (int)rank : u / a.n_tiles; };
 
   for (int i = threadIdx.x; i < a.Cout; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
     for (int s = 0; s < NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 128); }
+    for (int b = 0; b < NACC; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), PAIR ? 2 : 128); }
     mbar_init(drain_bar, 1);
     mbar_init(mask_bar, 1);
     mbar_init(w_bar, 1);
@@ -105,11 +122,17 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     tma_prefetch_desc(&map_w);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
-    tmem_relinquish();
+    if (PAIR) {
+      tmem_alloc_pair(smem_u32(&tmem_base_slot), NACC * BN);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(&tmem_base_slot), NACC * BN);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();  // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
@@ -122,19 +145,29 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       int slot = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m_tile = tile / a.n_tiles;
+      for (int unit = first_unit; unit < total_units && ok; unit += unit_stride) {
+        const int m_tile = unit_m_tile(unit);
         const int tw = m_tile % a.tiles_w, t = m_tile / a.tiles_w;
         const int w0 = tw * PW, h0 = (t % a.tiles_h) * PH, img = t / a.tiles_h;
         for (int cb = 0; cb < a.cin_blocks; ++cb) {
           if (!mbar_wait(a_empty(slot), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
-          mbar_expect_tx(a_full(slot), A_BYTES);
-          tma_load_4d(smem_base + slot * A_SLOT, &map_x, a_full(slot), cb * BK, w0 - 1, h0 - 1, img);
+          if (PAIR) {
+            // both CTAs' patches are counted on the even CTA's barrier, which announces all their bytes
+            if (rank == 0) mbar_expect_tx(a_full(slot), 2 * A_BYTES);
+            tma_load_4d_pair(smem_base + slot * A_SLOT, &map_x, map_to_cta(a_full(slot), 0), cb * BK, w0 - 1, h0 - 1, img);
+          } else {
+            mbar_expect_tx(a_full(slot), A_BYTES);
+            tma_load_4d(smem_base + slot * A_SLOT, &map_x, a_full(slot), cb * BK, w0 - 1, h0 - 1, img);
+          }
           ++fills[slot];
           if (++slot == a.na) { slot = 0; phase ^= 1; }
         }
       }
-      if (!ok)
+      if (!ok && rank != 0) {
+        // the peer's copies report to the even CTA's barriers: allow them a millisecond to land
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 1000000ull) {}
+      } else if (!ok)
         for (int s = 0; s < NA; ++s)
           if (fills[s]) {
             const unsigned long long t0 = global_timer_ns();
@@ -150,27 +183,49 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       int slot = 0;
       uint32_t phase = 0;
       bool ok = true;
+      const int row_in_tile = (int)rank * T::BNH;  // this CTA's output channels within the BN of a tile
       if (a.resident) {
-        // n_tiles == 1: the whole filter for these BN output channels, once
-        mbar_expect_tx(w_bar, (uint32_t)(a.cin_blocks * 3 * T::B_BYTES));
-        for (int cb = 0; cb < a.cin_blocks; ++cb)
-          for (int r = 0; r < 3; ++r)
-            tma_load_3d(b_base + (cb * 3 + r) * T::B_BYTES, &map_w, w_bar, cb * BK, 0, 3 * r);
-        const unsigned long long t0 = global_timer_ns();  // never leave with the copy in flight
-        while (!mbar_try_wait(w_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+        // n_tiles == 1: the whole filter for these output channels, once
+        if (PAIR) {
+          const uint32_t wb = map_to_cta(w_bar, 0);
+          if (rank == 0) mbar_expect_tx(w_bar, (uint32_t)(2 * a.cin_blocks * 3 * T::B_BYTES));
+          for (int cb = 0; cb < a.cin_blocks; ++cb)
+            for (int r = 0; r < 3; ++r)
+              tma_load_3d_pair(b_base + (cb * 3 + r) * T::B_BYTES, &map_w, wb, cb * BK, row_in_tile, 3 * r);
+        } else {
+          mbar_expect_tx(w_bar, (uint32_t)(a.cin_blocks * 3 * T::B_BYTES));
+          for (int cb = 0; cb < a.cin_blocks; ++cb)
+            for (int r = 0; r < 3; ++r)
+              tma_load_3d(b_base + (cb * 3 + r) * T::B_BYTES, &map_w, w_bar, cb * BK, 0, 3 * r);
+        }
+        // never leave with the copy in flight.  (The peer of a pair cannot see the even CTA's barrier;
+        // its epilogue does not finish before MMAs that needed this filter have.)
+        if (rank == 0) {
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(w_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+        }
       }
-      for (int tile = blockIdx.x; tile < total_tiles && ok && !a.resident; tile += gridDim.x) {
-        const int n_tile = tile % a.n_tiles;
+      for (int unit = first_unit; unit < total_units && ok && !a.resident; unit += unit_stride) {
+        const int n_tile = unit % a.n_tiles;
         for (int cb = 0; cb < a.cin_blocks && ok; ++cb)
           for (int r = 0; r < 3; ++r) {
             if (!mbar_wait(b_empty(slot), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
-            mbar_expect_tx(b_full(slot), T::B_BYTES);
-            tma_load_3d(b_base + slot * T::B_BYTES, &map_w, b_full(slot), cb * BK, n_tile * BN, 3 * r);
+            if (PAIR) {
+              if (rank == 0) mbar_expect_tx(b_full(slot), 2 * T::B_BYTES);
+              tma_load_3d_pair(b_base + slot * T::B_BYTES, &map_w, map_to_cta(b_full(slot), 0), cb * BK,
+                               n_tile * BN + row_in_tile, 3 * r);
+            } else {
+              mbar_expect_tx(b_full(slot), T::B_BYTES);
+              tma_load_3d(b_base + slot * T::B_BYTES, &map_w, b_full(slot), cb * BK, n_tile * BN, 3 * r);
+            }
             ++fills[slot];
             if (++slot == a.nb) { slot = 0; phase ^= 1; }
           }
       }
-      if (!ok)
+      if (!ok && rank != 0) {
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 1000000ull) {}
+      } else if (!ok)
         for (int s = 0; s < NB; ++s)
           if (fills[s]) {
             const unsigned long long t0 = global_timer_ns();
@@ -179,16 +234,16 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, 0, 0);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(PAIR ? 2 * BM : BM, BN, 0, 0);
       int aslot = 0, bslot = 0;
       uint32_t aphase = 0, bphase = 0;
       int local = 0;
       bool ok = true;
       if (a.resident) ok = mbar_wait(w_bar, 0, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
-        const int buf = local & 1;
-        const uint32_t use = (uint32_t)(local >> 1);
+      for (int unit = first_unit; unit < total_units && ok; unit += unit_stride, ++local) {
+        const int buf = local % NACC;
+        const uint32_t use = (uint32_t)(local / NACC);
         if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
@@ -204,22 +259,29 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
               const uint32_t sb = b_base + bslot * T::B_BYTES + s * T::TAP_BYTES;
               const uint32_t a_tap = sa + (uint32_t)(r * IW + s) * 128u;
               const uint64_t da = smem_desc_sw128_sbo(a_tap, IW * 128), db = smem_desc_sw128(sb, 16);
-              umma_bf16(d_tmem, da, db, idesc, (cb | r | s) != 0 ? 1u : 0u);
+              if (PAIR) {
+                umma_bf16_pair(d_tmem, da, db, idesc, (cb | r | s) != 0 ? 1u : 0u);
 #pragma unroll
-              for (int k = 1; k < BK / 16; ++k)
-                umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
+                for (int k = 1; k < BK / 16; ++k)
+                  umma_bf16_pair_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
+              } else {
+                umma_bf16(d_tmem, da, db, idesc, (cb | r | s) != 0 ? 1u : 0u);
+#pragma unroll
+                for (int k = 1; k < BK / 16; ++k)
+                  umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
+              }
             }
-            if (!a.resident) umma_commit(b_empty(bslot));
+            if (!a.resident) { if (PAIR) umma_commit_pair(b_empty(bslot), 3); else umma_commit(b_empty(bslot)); }
             if (!a.resident && ++bslot == a.nb) { bslot = 0; bphase ^= 1; }
           }
           if (!ok) break;
-          umma_commit(a_empty(aslot));
+          if (PAIR) umma_commit_pair(a_empty(aslot), 3); else umma_commit(a_empty(aslot));
           if (++aslot == a.na) { aslot = 0; aphase ^= 1; }
         }
-        if (ok) umma_commit(acc_full(buf));
+        if (ok) { if (PAIR) umma_commit_pair(acc_full(buf), 3); else umma_commit(acc_full(buf)); }
       }
       if (!ok) {
-        umma_commit(drain_bar);
+        if (PAIR) umma_commit_pair(drain_bar, 1); else umma_commit(drain_bar);
         const unsigned long long t0 = global_timer_ns();
         while (!mbar_try_wait(drain_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
       }
@@ -237,10 +299,10 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     uint32_t stage_sel = 0;  // which of the two staging tiles the next chunk uses
     const uint8_t* mask_srow = smem_raw + (mask_smem - smem_u32(smem_raw)) + row * 128;
     uint32_t mask_phase = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
-      const int buf = local & 1;
-      const uint32_t use = (uint32_t)(local >> 1);
-      const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
+    for (int unit = first_unit; unit < total_units; unit += unit_stride, ++local) {
+      const int buf = local % NACC;
+      const uint32_t use = (uint32_t)(local / NACC);
+      const int m_tile = unit_m_tile(unit), n_tile = unit % a.n_tiles;
       const bool got = mbar_wait(acc_full(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
       if (named_bar_or(1, 128, !got)) break;  // all four warps leave together
       tc_fence_after();
@@ -341,53 +403,80 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         }
       }
       tc_fence_before();
-      mbar_arrive(acc_empty(buf));
+      if (PAIR) {
+        // one arrival per CTA, on the even CTA's barrier: an arrival that crosses the cluster costs far
+        // more than a local one, and a tile here lasts a microsecond or two
+        named_bar_sync(1, 128);
+        if (issuer) mbar_arrive_cluster(map_to_cta(acc_empty(buf), 0));
+      } else {
+        mbar_arrive(acc_empty(buf));
+      }
     }
     if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }
 
   tc_fence_before();
   __syncthreads();
+  // a pair meets before either CTA releases tensor memory or exits: until then the peer may still
+  // signal this CTA's barriers, and the even CTA's MMAs read the peer's shared memory
+  if (PAIR) cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 2 * BN);
+    if (PAIR) tmem_dealloc_pair(tmem_base, NACC * BN); else tmem_dealloc(tmem_base, NACC * BN);
   }
 }
 
-template <int BN>
+template <int BN, bool PAIR>
 cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const CUtensorMap& mm,
                         HaloArgs a, cudaStream_t st) {
-  using T = HaloTile<BN>;
+  using T = HaloTile<BN, PAIR>;
   // plan the shared memory: keep the whole filter resident when it fits beside two or three patch slots
   // (then only the input patches cross the L2-to-SM path, which is what bounds these layers), else
   // stream filter rows through a ring
   const int res_bytes = a.cin_blocks * 3 * T::B_BYTES;
   const int fixed = T::fixed_bytes(a.mask != nullptr);
   a.resident = 0;
-  for (int na = 3; na >= 2 && !a.resident; --na)
+  for (int na = kMaxPatchSlots; na >= 2 && !a.resident; --na)
     if (a.n_tiles == 1 && na * A_SLOT + res_bytes + fixed <= T::kLimit) {
       a.resident = 1; a.na = na; a.nb = 0; a.b_region_bytes = res_bytes;
     }
   if (!a.resident) {
-    a.na = BN <= 64 ? 3 : 2;
-    int nb = (T::kLimit - fixed - a.na * A_SLOT) / T::B_BYTES;
-    a.nb = nb > 4 ? 4 : nb;
-    if (a.nb < 2) return cudaErrorInvalidValue;
+    // filter ring of up to four rows (never fewer than two), the rest for patch slots
+    int nb = 4;
+    while (nb > 2 && 2 * A_SLOT + nb * T::B_BYTES + fixed > T::kLimit) --nb;
+    a.nb = nb;
+    int na = (T::kLimit - fixed - nb * T::B_BYTES) / A_SLOT;
+    a.na = na > kMaxPatchSlots ? kMaxPatchSlots : na;
+    if (a.na < 2) return cudaErrorInvalidValue;
     a.b_region_bytes = a.nb * T::B_BYTES;
   }
   const int smem = a.na * A_SLOT + a.b_region_bytes + fixed;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_halo_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::kLimit);
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_halo_tc_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::kLimit);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (PAIR) {
+    const int units = (a.m_tiles / 2) * a.n_tiles;
+    const int pairs = units < sms / 2 ? units : sms / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, conv3x3_halo_tc_kernel<BN, PAIR>, mx, mw, my, mm, a);
+  }
   const int tiles = a.m_tiles * a.n_tiles;
-  conv3x3_halo_tc_kernel<BN><<<tiles < sms ? tiles : sms, kThreads, smem, st>>>(mx, mw, my, mm, a);
+  conv3x3_halo_tc_kernel<BN, PAIR><<<tiles < sms ? tiles : sms, kThreads, smem, st>>>(mx, mw, my, mm, a);
   return cudaGetLastError();
 }
 
@@ -425,13 +514,16 @@ bool tc_conv3x3_halo_supported(ConvShape s) {
 }
 
 cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
-                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st) {
+                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, bool pairs) {
   if (!out && !pooled) return cudaErrorInvalidValue;
   if (!tc_conv3x3_halo_supported(s)) return cudaErrorInvalidValue;
   const int BN = s.Cout % 128 == 0 ? 128 : 64;
+  // CTA pairs take two tiles at a time.  They pay with 128 output channels, where one CTA's MMAs are
+  // bound by shared-memory reads; with 64 they measure the same as single CTAs, which are kept there.
+  const bool pair = pairs && BN == 128 && (s.N * (s.W / PW) * (s.H / PH)) % 2 == 0;
   CUtensorMap mx, mw;
   if (!make_patch_map(&mx, in, s.N, s.H, s.W, s.Cin, IW, IH)) return cudaErrorInvalidValue;
-  if (!make_filter_row_map(&mw, wt_tap_major, s.Cout, s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
+  if (!make_filter_row_map(&mw, wt_tap_major, s.Cout, s.Cin, (uint32_t)(pair ? BN / 2 : BN))) return cudaErrorInvalidValue;
   CUtensorMap my = mw;  // only read when there is a full-resolution output
   if (out && !make_patch_map(&my, out, s.N, s.H, s.W, s.Cout, PW, PH)) return cudaErrorInvalidValue;
   CUtensorMap mm = mw;  // only read when there is a mask
@@ -444,7 +536,8 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const floa
   a.m_tiles = s.N * a.tiles_w * a.tiles_h;
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0; a.bias = bias; a.mask = mask; a.out = out; a.pooled = pooled; a.dev_error = dev_error;
-  return BN == 128 ? launch_halo<128>(mx, mw, my, mm, a, st) : launch_halo<64>(mx, mw, my, mm, a, st);
+  if (pair) return launch_halo<128, true>(mx, mw, my, mm, a, st);
+  return BN == 128 ? launch_halo<128, false>(mx, mw, my, mm, a, st) : launch_halo<64, false>(mx, mw, my, mm, a, st);
 }
 
 }  // namespace vgg

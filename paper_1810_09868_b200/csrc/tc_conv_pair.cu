@@ -103,7 +103,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < T::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 256); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 2); }
     mbar_init(drain_bar, 1);
     mbar_fence_init();
     tma_prefetch_desc(&map_x);
@@ -241,7 +241,8 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           }
         }
         tc_fence_before();
-        mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
+        named_bar_sync(1, 128);
+        if (issuer) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
         continue;
       }
 #pragma unroll 1
@@ -296,7 +297,8 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         }
       }
       tc_fence_before();
-      mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));  // 256 arrivals: both CTAs have drained the buffer
+      named_bar_sync(1, 128);
+      if (issuer) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));  // one arrival per CTA of the pair
     }
     if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }

@@ -36,8 +36,10 @@ bool tc_conv3x3_halo_supported(ConvShape s);
 // master; for_dgrad gives the rotated, channel-swapped filter of the input gradient, [9][Cin][Cout]).
 // `pooled` (or null) also receives the 2x2 max-pool of the result; `out` may then be null.
 cudaError_t tc_make_tap_major(const float* w, bf16* out, int Cin, int Cout, bool for_dgrad, cudaStream_t st);
+// pairs: work as CTA pairs (two tiles at a time, each CTA staging half of the filter's output channels)
+// when the tile count is even.
 cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
-                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
+                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, bool pairs = true);
 
 // Filter gradient of the same convolution as a GEMM with M = Cout, N = 9*Cin,
 // K = pixels (both operands read transposed, x through the im2col window):

@@ -230,7 +230,7 @@ struct Pass {
       ok(tc_first_conv((const bf16 *)buf(p.x8), n->w8, n->params + c.b_off, (bf16 *)y, s, true, n->dev_error, st), 1);
     } else if (n->use_tc && tc_conv3x3_halo_supported(s)) {
       ok(tc_conv3x3_halo((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
-                         (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st), 1);
+                         (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st, n->use_pair), 1);
       return;
     } else if (pair_ok(s)) {
       int k = 1;
@@ -263,7 +263,7 @@ struct Pass {
       const T *wr = static_cast<const T *>(n->dgrad_w) + c.dgrad_off;
       if (n->use_tc && tc_conv3x3_halo_supported(t))
         ok(tc_conv3x3_halo((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr, t,
-                           false, n->dev_error, st), 1);
+                           false, n->dev_error, st, n->use_pair), 1);
       else if (pair_ok(t)) {
         int k = 1;
         ok(tc_conv3x3_pair((const bf16 *)dz, (const bf16 *)wr, nullptr, (const bf16 *)mask, (bf16 *)dx,
