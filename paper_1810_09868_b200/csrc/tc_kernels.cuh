@@ -41,6 +41,13 @@ cudaError_t tc_make_tap_major(const float* w, bf16* out, int Cin, int Cout, bool
 cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
                             bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, bool pairs = true);
 
+// The same convolution for 64 output channels (tc_conv_rowshift.cu): the three taps of a filter row
+// share one 128 x 192 x 16 MMA, and the epilogue adds the three column-shifted partial sums.  Same
+// arguments as tc_conv3x3_halo; W must be a multiple of 14 and H of 8.
+bool tc_conv3x3_rowshift_supported(ConvShape s);
+cudaError_t tc_conv3x3_rowshift(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
+                                bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
+
 // Filter gradient of the same convolution as a GEMM with M = Cout, N = 9*Cin,
 // K = pixels (both operands read transposed, x through the im2col window):
 // dW fp32 [Cout][3][3][Cin]; db fp32 [Cout] = column sums of dz from the same GEMM (a block of

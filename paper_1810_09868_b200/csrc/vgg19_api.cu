@@ -228,6 +228,10 @@ struct Pass {
     if (first_tc_ok(l, s)) {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       ok(tc_first_conv((const bf16 *)buf(p.x8), n->w8, n->params + c.b_off, (bf16 *)y, s, true, n->dev_error, st), 1);
+    } else if (n->use_tc && tc_conv3x3_rowshift_supported(s)) {
+      ok(tc_conv3x3_rowshift((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
+                             (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st), 1);
+      return;
     } else if (n->use_tc && tc_conv3x3_halo_supported(s)) {
       ok(tc_conv3x3_halo((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
                          (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st, n->use_pair), 1);
@@ -261,7 +265,10 @@ struct Pass {
     if (dx) {
       ConvShape t{B, c.H, c.W, c.Cout, c.Cin};  // a 3x3 correlation from Cout to Cin channels
       const T *wr = static_cast<const T *>(n->dgrad_w) + c.dgrad_off;
-      if (n->use_tc && tc_conv3x3_halo_supported(t))
+      if (n->use_tc && tc_conv3x3_rowshift_supported(t))
+        ok(tc_conv3x3_rowshift((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr,
+                               t, false, n->dev_error, st), 1);
+      else if (n->use_tc && tc_conv3x3_halo_supported(t))
         ok(tc_conv3x3_halo((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr, t,
                            false, n->dev_error, st, n->use_pair), 1);
       else if (pair_ok(t)) {
