@@ -19,8 +19,11 @@
 // Roles and pipeline are those of the general convolution kernel: warp 0 TMA
 // producer, warp 1 MMA issuer and TMEM owner, then epilogue warps; double-buffered
 // accumulator; persistent CTAs; time-limited waits.  The main loop is five MMAs
-// per tile, so the epilogue sets the pace: eight epilogue warps, two per TMEM lane
-// quarter, each converting and storing 32 of the 64 output channels of its rows.
+// per tile, so the epilogue sets the pace: two groups of eight epilogue warps take
+// alternate tiles (each group its own accumulator buffer, staging tile and named
+// barrier), so that one tile's chain of wait, tensor-memory load, conversion, staging
+// and store overlaps the next tile's; within a group two warps per TMEM lane quarter
+// each convert and store 32 of the 64 output channels of their rows.
 #include "tc_common.cuh"
 #include "tc_kernels.cuh"
 
@@ -37,7 +40,8 @@ constexpr int W_TAP_BYTES = BN * 16;      // 64 output channels x 8 channels
 constexpr int W_BYTES = 10 * W_TAP_BYTES;
 constexpr int OUT_TILE_BYTES = BM * BN * 2;  // 16 KB staging tile for the TMA store, two of them
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_TILE_BYTES + W_BYTES + 1024 + 256;
-constexpr int kThreads = 320;  // producer, MMA issuer, eight epilogue warps (two per TMEM lane quarter)
+constexpr int kThreads = 576;  // producer, MMA issuer, two groups of eight epilogue warps
+constexpr int kGroupThreads = 256;
 
 constexpr int PW = 8, PH = 16, IW = PW + 2, IH = PH + 2;  // patch mode: output patch and input patch with halo
 constexpr int PATCH_BYTES = IW * IH * 16;                 // 2880
@@ -185,22 +189,27 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       }
     }
   } else {
-    const int quarter = warp & 3;
+    const int group = (warp - 2) >> 3;            // which of the two accumulator buffers / staging tiles
+    const int quarter = warp & 3;                 // the TMEM lane quarter this warp may read
     const int row = quarter * 32 + lane;
-    int local = 0;
-    for (int tile = blockIdx.x; tile < a.m_tiles; tile += gridDim.x, ++local) {
-      const int buf = local & 1;
-      const uint32_t use = (uint32_t)(local >> 1);
-      const bool got = mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
-      // the store that last used this tile's staging buffer must have read it before anyone refills it;
-      // the barrier doubles as the vote that lets all eight warps leave together if any wait failed
-      if (threadIdx.x == 64) tma_store_wait_read<1>();
-      if (named_bar_or(1, 256, !got)) break;
+    const int cc = (((warp - 2) >> 2) & 1) * 32;  // this warp's 32 of the 64 output channels
+    const int bar_id = 1 + group;
+    const bool issuer = threadIdx.x == 64 + group * kGroupThreads;  // owns the group's store groups
+    const uint32_t stage_out = out_smem + (uint32_t)group * OUT_TILE_BYTES;
+    uint32_t use = 0;  // tiles this group has taken
+    for (int tile = blockIdx.x + group * gridDim.x; tile < a.m_tiles; tile += 2 * gridDim.x, ++use) {
+      const bool got = mbar_wait(acc_full_bar(group), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
+      // the group's previous store must have read the staging tile before anyone refills it; the
+      // barrier doubles as the vote that lets the group's warps leave together if any wait failed
+      if (issuer) tma_store_wait_read<0>();
+      if (named_bar_or(bar_id, kGroupThreads, !got)) break;
       tc_fence_after();
-      const int cc = ((warp - 2) >> 2) * 32;  // warps 2-5 take channels 0..31, warps 6-9 channels 32..63
       uint32_t v[32];
-      tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+      tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(group * BN + cc), v);
       tmem_ld_wait();
+      // the accumulator is in registers: the MMA issuer may have the buffer back
+      tc_fence_before();
+      mbar_arrive(acc_empty_bar(group));
       uint32_t packed[16];
 #pragma unroll
       for (int j = 0; j < 32; j += 2) {
@@ -212,9 +221,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       }
       if (a.patch) {
         // the tile leaves through shared memory and one TMA store (whole 128-byte lines) instead of
-        // 256 threads writing 64-byte pieces of their own rows; two staging tiles alternate
-        const uint32_t stage_out = out_smem + (uint32_t)(local & 1) * OUT_TILE_BYTES;
-        const bool issuer = threadIdx.x == 64;  // first epilogue thread owns the store groups
+        // 256 threads writing 64-byte pieces of their own rows
         uint8_t* dst = smem_raw + (stage_out - smem_u32(smem_raw)) + row * 128;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -223,7 +230,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
               make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
         }
         fence_async_smem();
-        named_bar_sync(1, 256);
+        named_bar_sync(bar_id, kGroupThreads);
         if (issuer) {
           const int tw = tile % a.tiles_w, t = tile / a.tiles_w;
           tma_store_4d(&map_y, stage_out, 0, tw * PW, (t % a.tiles_h) * PH, t / a.tiles_h);
@@ -238,10 +245,8 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             op[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
         }
       }
-      tc_fence_before();
-      mbar_arrive(acc_empty_bar(buf));
     }
-    if (threadIdx.x == 64) tma_store_wait_all();  // shared memory must outlive the stores that read it
+    if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }
 
   tc_fence_before();

@@ -10,7 +10,10 @@
 // (TMA im2col) with the pixel index as k: that is the filter gradient
 //   dW[cout][tap][c] = sum_pixels dz[pixel][cout] * x[pixel shifted by tap][c].
 // A fourth form does the same for the 8-channel copy of the 3-channel image
-// (16-byte rows, no swizzle; the tile's 80 columns are 10 taps x 8 channels).
+// (16-byte rows, no swizzle; the tile's 80 columns are 10 taps x 8 channels).  There the copy
+// engine, at nine small boxes per K block, sets the pace, so a K block is 128 pixels instead of 64:
+// A's second 64 x 64 box holds the next 64 pixels instead of output channels 64..127 (the layer has
+// 64), which leaves accumulator rows 64..127 meaningless and unread.
 //
 // One CTA computes one 128 x BN tile over its share of K (grid.y splits K):
 //   warp 0 TMA producer, warp 1 TMEM owner + single-thread MMA issuer, warps
@@ -60,7 +63,10 @@ struct GemmArgs {
 // PAIR: two CTAs (a cluster, tcgen05 cta_group::2) compute a 256 x BN tile with one MMA stream; each
 // stages its own 128 rows of A and half of the B tile.
 template <int BN, bool PAIR>
-__host__ __device__ constexpr int stage_bytes() { return A_BYTES + (PAIR ? BN / 2 : BN) * BK * 2; }
+__host__ __device__ constexpr int stage_bytes() {
+  // BN = 80 is the 8-channel form, whose K blocks are 128 pixels: ten taps x 128 pixels x 16 bytes
+  return BN == 80 ? A_BYTES + 10 * 2048 : A_BYTES + (PAIR ? BN / 2 : BN) * BK * 2;
+}
 
 template <int BN, int AMODE, int BMODE, bool PAIR>
 __global__ void __launch_bounds__(kThreads)
@@ -147,7 +153,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             grp_c[q] = j - tap * g.Cin; grp_r[q] = tap / 3; grp_s[q] = tap - 3 * (tap / 3);
           }
         }
-        const long p0 = (long)kb0 * BK;
+        const long p0 = (long)kb0 * (BMODE == kMnMajorIm2colC8 ? 2 * BK : BK);
         w0 = (int)(p0 % g.W);
         const long t = p0 / g.W;
         h0 = (int)(t % g.H); img = (int)(t / g.H);
@@ -171,9 +177,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (++stage == g.stages) { stage = 0; phase ^= 1; }
           continue;
         }
-        mbar_expect_tx(full_bar(stage), BMODE == kMnMajorIm2colC8 ? A_BYTES + 9 * 1024 : STAGE);
+        mbar_expect_tx(full_bar(stage), BMODE == kMnMajorIm2colC8 ? A_BYTES + 9 * 2048 : STAGE);
         if (AMODE == kKMajor) {
           tma_load_2d(sa, &map_a, full_bar(stage), kb * BK, m0);
+        } else if (BMODE == kMnMajorIm2colC8) {
+          tma_load_2d(sa, &map_a, full_bar(stage), m0, kb * 2 * BK);
+          tma_load_2d(sa + GROUP_BYTES, &map_a, full_bar(stage), m0, kb * 2 * BK + BK);
         } else {
           tma_load_2d(sa, &map_a, full_bar(stage), m0, kb * BK);
           tma_load_2d(sa + GROUP_BYTES, &map_a, full_bar(stage), m0 + 64, kb * BK);
@@ -189,15 +198,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tma_load_im2col_4d(sb + q * GROUP_BYTES, &map_b, full_bar(stage), grp_c[q], w0 - 1, h0 - 1, img,
                                (uint16_t)grp_s[q], (uint16_t)grp_r[q]);
         } else {
-          // nine taps of the 8-channel image, 64 pixels x 16 bytes each; the tenth slot (columns
+          // nine taps of the 8-channel image, 128 pixels x 16 bytes each; the tenth slot (columns
           // 72..79 of the tile, never stored) is left as it is
 #pragma unroll
           for (int tap = 0; tap < 9; ++tap)
-            tma_load_im2col_4d(sb + tap * 1024, &map_b, full_bar(stage), 0, w0 - 1, h0 - 1, img, (uint16_t)(tap % 3),
+            tma_load_im2col_4d(sb + tap * 2048, &map_b, full_bar(stage), 0, w0 - 1, h0 - 1, img, (uint16_t)(tap % 3),
                                (uint16_t)(tap / 3));
         }
         if (BMODE == kMnMajorIm2col || BMODE == kMnMajorIm2colC8) {
-          w0 += BK;
+          w0 += BMODE == kMnMajorIm2colC8 ? 2 * BK : BK;
           while (w0 >= g.W) { w0 -= g.W; if (++h0 == g.H) { h0 = 0; ++img; } }
         }
         ++fills[stage];
@@ -229,12 +238,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tc_fence_after();
         const uint32_t sa = smem_base + stage * STAGE, sb = sa + A_BYTES;
         // K-major: 16 k = 32 bytes along the swizzled row.  MN-major: 16 k = 16 rows = 2048 bytes.
-        // 8-channel form: 16 k = 16 rows of 16 bytes; 8-row groups 128 bytes apart, taps 1024 bytes apart.
+        // 8-channel form: 16 k = 16 rows of 16 bytes; 8-row groups 128 bytes apart, taps 2048 bytes apart;
+        // eight K steps per block, A's two boxes being consecutive in shared memory.
         constexpr uint32_t a_step = AMODE == kKMajor ? 32 : 2048;
         constexpr uint32_t b_step = BMODE == kKMajor ? 32 : (BMODE == kMnMajorIm2colC8 ? 256 : 2048);
         const uint64_t da = AMODE == kKMajor ? smem_desc_sw128(sa, 16) : smem_desc_sw128(sa, GROUP_BYTES);
         const uint64_t db = BMODE == kKMajor          ? smem_desc_sw128(sb, 16)
-                            : BMODE == kMnMajorIm2colC8 ? smem_desc_plain(sb, 128, 1024)
+                            : BMODE == kMnMajorIm2colC8 ? smem_desc_plain(sb, 128, 2048)
                                                         : smem_desc_sw128(sb, GROUP_BYTES);
         if (PAIR) {
           umma_bf16_pair(tmem_base, da, db, idesc, kb > kb0 ? 1u : 0u);
@@ -250,9 +260,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
           umma_commit_pair(empty_bar(stage), 3);  // frees the stage in both CTAs
         } else {
+          constexpr int k_steps = BMODE == kMnMajorIm2colC8 ? 2 * BK / 16 : BK / 16;
           umma_bf16(tmem_base, da, db, idesc, kb > kb0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 1; k < BK / 16; ++k)
+          for (int k = 1; k < k_steps; ++k)
             umma_bf16_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), idesc);
           if (kb == db_next) {
             umma_bf16(tmem_base + BN, da, d_ones, idesc_ones, kb != db_first ? 1u : 0u);
@@ -618,22 +629,30 @@ namespace {
 // dW[k][tap][c] = sum over splits of partial[split][k][tap * 8 + c], c < 3.  Channel 3 of the
 // 8-channel image is the constant 1, so column (centre tap, channel 3) is sum_pixels dz[pixel][k]:
 // the bias gradient.
+// One warp per output: lanes take the splits round-robin and a butterfly adds the lanes (a fixed order).
 __global__ void wgrad_c8_finish_kernel(const float* __restrict__ partial, int splits, int Cout, float* dW, float* db) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (db && i < Cout) {
-    float s = 0.f;
-    for (int z = 0; z < splits; ++z) s += partial[((long)z * Cout + i) * 80 + 4 * 8 + 3];
-    db[i] = s;
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  const int n_dw = Cout * 27;
+  if (i >= n_dw + Cout) return;  // whole warps leave together
+  long col;
+  float* dst;
+  if (i < n_dw) {
+    const int c = i % 3, tap = (i / 3) % 9, k = i / 27;
+    col = (long)k * 80 + tap * 8 + c;
+    dst = dW + i;
+  } else {
+    col = (long)(i - n_dw) * 80 + 4 * 8 + 3;
+    dst = db ? db + (i - n_dw) : nullptr;
   }
-  if (i >= Cout * 27) return;
-  int c = i % 3, tap = (i / 3) % 9, k = i / 27;
   float s = 0.f;
-  for (int z = 0; z < splits; ++z) s += partial[((long)z * Cout + k) * 80 + tap * 8 + c];
-  dW[i] = s;
+  for (int z = lane; z < splits; z += 32) s += partial[(long)z * Cout * 80 + col];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0 && dst) *dst = s;
 }
 void wgrad_c8_plan(ConvShape s, int* k_blocks, int* splits, int* per) {
   const long P = (long)s.N * s.H * s.W;
-  *k_blocks = (int)((P + BK - 1) / BK);
+  *k_blocks = (int)((P + 2 * BK - 1) / (2 * BK));  // K blocks of 128 pixels
   plan_split(1, *k_blocks, splits, per);
 }
 }  // namespace
@@ -649,7 +668,7 @@ cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* db,
   const long P = (long)s.N * s.H * s.W;
   CUtensorMap ma, mb;
   if (!make_tiled_map_2d(&ma, dz, (uint64_t)P, (uint64_t)s.Cout, 64)) return cudaErrorInvalidValue;
-  if (!make_im2col_map_c8(&mb, x8, s.N, s.H, s.W, 64)) return cudaErrorInvalidValue;
+  if (!make_im2col_map_c8(&mb, x8, s.N, s.H, s.W, 128)) return cudaErrorInvalidValue;
   GemmArgs g{};
   int splits;
   wgrad_c8_plan(s, &g.k_blocks, &splits, &g.kb_per_split);
@@ -657,7 +676,7 @@ cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* db,
   g.dev_error = dev_error; g.ldc = 80; g.partial = partial;
   cudaError_t e = launch_gemm_tc<80, kMnMajor, kMnMajorIm2colC8>(ma, mb, g, 1, splits, st);
   if (e != cudaSuccess) return e;
-  wgrad_c8_finish_kernel<<<(s.Cout * 27 + 255) / 256, 256, 0, st>>>(partial, splits, s.Cout, dW, db);
+  wgrad_c8_finish_kernel<<<(s.Cout * 28 * 32 + 255) / 256, 256, 0, st>>>(partial, splits, s.Cout, dW, db);
   return cudaGetLastError();
 }
 
