@@ -374,6 +374,8 @@ const TensorMapApi& tensor_map_api();
 
 // [rows][cols] bf16 row-major matrix, box = box_rows x 64 columns, 128 B swizzle.
 bool make_tiled_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// [rows][cols] fp32 row-major matrix, box = box_rows x 32 columns (128 bytes), 128 B swizzle.
+bool make_tiled_map_2d_f32(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 // Same with a box of box_rows x 8 columns (16 bytes) and no swizzle.
 bool make_tiled_map_2d_c8(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 // Tap-major filter [9][Cout][Cin] bf16: box = 3 taps x box_cout rows x 64 channels, 128 B swizzle.

@@ -58,7 +58,9 @@ struct GemmArgs {
   int relu;
   int* dev_error;
   float* db_partial; // column sums of A at db_partial[((split * n_tiles) + n_tile) * M + m], or null
+  int tma_store;     // fp32 output (partial or out_f, no bias / ReLU / mask) leaves through staging tiles and map_c
 };
+constexpr int kStoreStagingBytes = 2 * BM * 128;  // two tiles of 128 rows x 32 fp32
 
 // PAIR: two CTAs (a cluster, tcgen05 cta_group::2) compute a 256 x BN tile with one MMA stream; each
 // stages its own 128 rows of A and half of the B tile.
@@ -70,7 +72,8 @@ __host__ __device__ constexpr int stage_bytes() {
 
 template <int BN, int AMODE, int BMODE, bool PAIR>
 __global__ void __launch_bounds__(kThreads)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs g) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_c, GemmArgs g) {
   static_assert(!PAIR || (AMODE == kMnMajor && BMODE == kMnMajorIm2col && BN % 128 == 0), "pairs: filter gradient only");
   constexpr int STAGE = stage_bytes<BN, PAIR>();
   constexpr int B_GROUPS = (PAIR ? BN / 2 : BN) / 64;  // 64-column groups of B this CTA stages
@@ -80,7 +83,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   constexpr int TMEM_COLS = COLS <= 64 ? 64 : (COLS <= 128 ? 128 : (COLS <= 256 ? 256 : 512));
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bars = smem_base + g.stages * STAGE;
+  const uint32_t store_smem = smem_base + g.stages * STAGE;  // 1024-byte aligned: stages are multiples of 1 KB
+  const uint32_t bars = store_smem + (g.tma_store ? kStoreStagingBytes : 0);
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
   const uint32_t acc_bar = bars + 8u * (2 * kMaxStages);
@@ -287,7 +291,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int quarter = warp & 3;
     const int m = m0 + quarter * 32 + lane;
     const bool row_ok = m < g.M;
-    if (mbar_wait(acc_bar, 0, &abort_flag, g.dev_error, kDevTimeoutAccum)) {
+    const bool got_acc = mbar_wait(acc_bar, 0, &abort_flag, g.dev_error, kDevTimeoutAccum);
+    if (got_acc && g.tma_store) {
+      // Raw fp32 tile, 32 columns (one 128-byte line per row) at a time through two alternating
+      // 128-byte-swizzled staging tiles and TMA stores: whole lines instead of 128 threads each
+      // writing 16-byte pieces of their own rows.  Rows and columns past the tensor are clipped.
+      tc_fence_after();
+      const bool issuer = threadIdx.x == 64;
+      const int row = quarter * 32 + lane;
+      const int row0 = (g.partial ? (int)blockIdx.y * g.M : 0) + m0;
+#pragma unroll 1
+      for (int cc = 0; cc < BN; cc += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)cc, v);
+        tmem_ld_wait();
+        const uint32_t tile = store_smem + (uint32_t)((cc >> 5) & 1) * (BM * 128);
+        if (issuer) tma_store_wait_read<1>();  // the store before last has read this staging tile
+        named_bar_sync(1, 128);
+        uint8_t* dst = smem_raw + (tile - smem_u32(smem_raw)) + row * 128;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(dst + ((q ^ (row & 7)) << 4)) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        fence_async_smem();
+        named_bar_sync(1, 128);
+        if (issuer && n0 + cc < g.N) {
+          tma_store_2d(&map_c, tile, n0 + cc, row0);
+          tma_store_commit();
+        }
+      }
+      if (issuer) tma_store_wait_all();
+    }
+    if (got_acc && !g.tma_store) {
       tc_fence_after();
 #pragma unroll 1
       for (int cc = 0; cc < BN; cc += 32) {
@@ -339,6 +373,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
       }
+    }
+    if (got_acc) {
       if (BMODE == kMnMajorIm2col && g.db_partial) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)BN, v);
@@ -422,16 +458,30 @@ cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArg
                            cudaStream_t st) {
   constexpr int STAGE = stage_bytes<BN, PAIR>();
   constexpr int kExtra = 1024 + 256 + 1024;  // alignment slack, barriers, block of ones
-  constexpr int max_stages = (227 * 1024 - 3072) / STAGE > kMaxStages ? kMaxStages : (227 * 1024 - 3072) / STAGE;
+  // Raw fp32 output (split-K partial sums, or a result without bias / ReLU / mask) leaves by TMA store
+  // where whole 128-row boxes cannot run into rows that belong to someone else: a single result
+  // matrix (the copy engine clips at its end), or partial sums stacked per split with M a multiple
+  // of 128, or M = 64 (box of 64 rows).
+  float* target = g.partial ? g.partial : g.out_f;
+  const bool plain = !g.bias && !g.relu && !g.mask && !g.out_h && target != nullptr;
+  const long out_rows = g.partial ? (long)splits * g.M : g.M;
+  const int out_cols = g.partial ? g.N : (int)g.ldc;
+  CUtensorMap mc = ma;  // unused unless tma_store
+  g.tma_store = 0;
+  if (plain && out_cols % 4 == 0 && (!g.partial || g.M % BM == 0 || g.M == 64) &&
+      make_tiled_map_2d_f32(&mc, target, (uint64_t)out_rows, (uint64_t)out_cols, g.M == 64 ? 64 : BM))
+    g.tma_store = 1;
+  constexpr int kBudget = 227 * 1024 - 3072 - kStoreStagingBytes;
+  constexpr int max_stages = kBudget / STAGE > kMaxStages ? kMaxStages : kBudget / STAGE;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, AMODE, BMODE, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         max_stages * STAGE + kExtra);
+                                         max_stages * STAGE + kExtra + kStoreStagingBytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   g.stages = g.kb_per_split < max_stages ? g.kb_per_split : max_stages;
-  const size_t smem = (size_t)g.stages * STAGE + kExtra;
+  const size_t smem = (size_t)g.stages * STAGE + kExtra + (g.tma_store ? kStoreStagingBytes : 0);
   if (PAIR) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * m_tiles * g.n_tiles, splits);
@@ -442,10 +492,10 @@ cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArg
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, AMODE, BMODE, PAIR>, ma, mb, g);
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, AMODE, BMODE, PAIR>, ma, mb, mc, g);
   }
   dim3 grid(m_tiles * g.n_tiles, splits);
-  gemm_tc_kernel<BN, AMODE, BMODE, PAIR><<<grid, kThreads, smem, st>>>(ma, mb, g);
+  gemm_tc_kernel<BN, AMODE, BMODE, PAIR><<<grid, kThreads, smem, st>>>(ma, mb, mc, g);
   return cudaGetLastError();
 }
 

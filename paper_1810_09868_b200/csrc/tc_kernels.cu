@@ -68,6 +68,18 @@ bool make_tiled_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64
   return tiled_map(map, base, rows, cols, 64, box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+bool make_tiled_map_2d_f32(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  const TensorMapApi& api = tensor_map_api();
+  if (!api.ok) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 4};
+  cuuint32_t box[2] = {32, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return api.encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_tiled_map_2d_c8(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
   return tiled_map(map, base, rows, cols, 8, box_rows, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
