@@ -39,6 +39,7 @@ BATCH = 100
 CONV = [(224, 3, 64), (224, 64, 64), (112, 64, 128), (112, 128, 128), (56, 128, 256), (56, 256, 256),
         (56, 256, 256), (56, 256, 256), (28, 256, 512), (28, 512, 512), (28, 512, 512), (28, 512, 512),
         (14, 512, 512), (14, 512, 512), (14, 512, 512), (14, 512, 512)]
+TRAIN_LR = 1e-6
 FWD_FLOP_PER_IMAGE = sum(2 * s * s * co * 9 * ci for s, ci, co in CONV) + 2 * (25088 * 4096 + 4096 * 4096 + 4096 * 1000)
 
 
@@ -114,6 +115,18 @@ def slowest_rank_ms(ms, world, device="cpu"):
     t = torch.tensor([ms], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def average_gradients(grads, world):
+    """Data-parallel exchange of a training step: every rank ends with the mean of the ranks'
+    gradients, i.e. the gradient of the mean loss over the whole job's batch (each rank's loss is
+    the mean over its own, equally sized, batch).  One all-reduce on the default process group."""
+    if world == 1:
+        return grads
+    import torch.distributed as dist
+    dist.all_reduce(grads, op=dist.ReduceOp.SUM)
+    grads /= world
+    return grads
 
 
 def aggregate_images_per_s(world, batch_per_rank, steps, slowest_ms):
@@ -250,6 +263,12 @@ def run_native(args):
     fwd = lambda: pkg.vgg19_forward(net.handle, x, BATCH, logits, None, stream)
     bwd = lambda: pkg.vgg19_backward(net.handle, x, y, BATCH, grads, loss, None, stream)
 
+    def train():
+        # forward + backward, the gradient all-reduce over the ranks (N > 1), one SGD step
+        pkg.vgg19_backward(net.handle, x, y, BATCH, grads, loss, None, stream)
+        average_gradients(grads, world)
+        pkg.vgg19_sgd_step(net.handle, grads, TRAIN_LR, stream)
+
     sampler = ClockSampler(local) if rank == 0 else None
     if sampler:
         sampler.start()
@@ -261,6 +280,11 @@ def run_native(args):
     bwd_ms = timed(bwd, bwd_steps, max(3, args.warmup))
     t_end = time.time()
     clocks = sampler.stop(t_begin, t_end) if sampler else None
+    net.sync_status(stream)
+
+    # training step last: it moves the weights (by a learning rate small enough to keep them sane)
+    train_steps = max(3, args.steps // 2)
+    train_ms = timed(train, train_steps, 3)
     net.sync_status(stream)
 
     # end to end: pinned host images in, logits out, through the host-buffer entry point
@@ -321,6 +345,10 @@ def run_native(args):
         "fwd_bwd": {"value": world * BATCH * bwd_steps / (bwd_ms * 1e-3), "unit": "images/s", "steps": bwd_steps,
                     "ms_per_step": bwd_ms / bwd_steps,
                     "launches_per_step": pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_BACKWARD)},
+        "train_step": {"value": world * BATCH * train_steps / (train_ms * 1e-3), "unit": "images/s", "steps": train_steps,
+                       "ms_per_step": train_ms / train_steps, "lr": TRAIN_LR,
+                       "what": "forward + backward + " + ("NCCL all-reduce of the 143.7 M fp32 gradients + " if world > 1 else "")
+                               + "SGD update of the fp32 master, bf16 and filter copies"},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": traffic,
                      "kernel": "conv3x3_pair_tc_kernel<256>: 3x3 convolution forward as a tcgen05 cta_group::2 implicit "

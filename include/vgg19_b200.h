@@ -118,6 +118,16 @@ int vgg19_forward(vgg19_t *net, const void *images, int32_t batch, float *logits
 int vgg19_backward(vgg19_t *net, const void *images, const int32_t *labels, int32_t batch,
                    float *grads, float *loss, float *logits, void *stream);
 
+/* One step of plain gradient descent, parameter <- parameter - lr * gradient, on the
+ * fp32 master copy, with the bf16 copy and every filter copy the kernels read
+ * (rotated, tap-major, padded) rebuilt on the same stream.  The paper fuses "the
+ * training loop" with the two passes into one executable (introduction and
+ * conclusion) without naming the optimiser; plain SGD is the reading taken.
+ * grads: device fp32, vgg19_param_count() elements, in parameter order (what
+ * vgg19_backward wrote).  Asynchronous on `stream`; passes enqueued later on the
+ * same stream see the new parameters.  Graphs recorded earlier stay valid. */
+int vgg19_sgd_step(vgg19_t *net, const float *grads, float lr, void *stream);
+
 /* HOST-buffer convenience wrappers: copy images (and labels) to the device,
  * run the pass, copy the results back and wait for the stream.  The bound
  * workspace must hold vgg19_workspace_bytes(net, batch, mode) +

@@ -381,6 +381,13 @@ def backward(steps, params, images, labels=None, n_total=None, grads=None, loss_
     return loss, grads, logits
 
 
+def sgd_step(params, grads, lr):
+    """One step of plain gradient descent, w <- w - lr * dL/dw, in fp64.  The paper
+    fuses "the training loop" with the two passes (introduction, conclusion) and
+    names no optimiser; this is the reading taken."""
+    return np.asarray(params, dtype=np.float64).ravel() - float(lr) * np.asarray(grads, dtype=np.float64).ravel()
+
+
 def vgg19_forward(params, images, storage=None):
     return forward(vgg19_steps(), params, images, storage=storage)
 

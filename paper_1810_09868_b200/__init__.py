@@ -55,6 +55,10 @@ class Net:
         binding.vgg19_backward(self.handle, images, labels, B, grads, loss, logits, stream)
         return grads, loss
 
+    def sgd_step(self, grads, lr, stream=None):
+        """parameters <- parameters - lr * grads, on the device, with every derived filter copy rebuilt."""
+        binding.vgg19_sgd_step(self.handle, grads, lr, stream or self._torch.cuda.current_stream(self.device))
+
     def saved_tensor(self, batch, mode, index):
         """View of a stored activation inside the workspace (no copy)."""
         off, dims = binding.vgg19_saved_tensor(self.handle, batch, mode, index)

@@ -91,6 +91,10 @@ cudaError_t softmax_xent(const float* logits, const int32_t* labels, float* prob
 // fp32 -> T copy (weights), and the dgrad filter: wt_t[c][r][s][k] = w[k][2-r][2-s][c].
 template <typename T>
 cudaError_t convert_f32(const float* src, T* dst, size_t n, cudaStream_t st);
+// params -= lr * grads (fp32 master, in place); params_t (the storage-type copy, or null when T is
+// float and the master is the copy) receives the rounded result in the same pass.
+template <typename T>
+cudaError_t sgd_update(float* params, const float* grads, T* params_t, float lr, size_t n, cudaStream_t st);
 template <typename T>
 cudaError_t make_dgrad_filter(const float* w, T* wt_t, int Cin, int Cout, cudaStream_t st);
 

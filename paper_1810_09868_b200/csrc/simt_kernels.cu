@@ -542,6 +542,33 @@ cudaError_t convert_f32(const float* src, T* dst, size_t n, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// p -= lr * g on the fp32 master copy, and the storage-type copy follows in the same pass
+// (four elements per thread where the count allows; the tail one at a time).
+template <typename T>
+__global__ void sgd_update_kernel(float* __restrict__ p, const float* __restrict__ g, T* __restrict__ pt, float lr,
+                                  size_t n) {
+  const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i + 3 < n) {
+    float4 w = *reinterpret_cast<float4*>(p + i);
+    const float4 d = *reinterpret_cast<const float4*>(g + i);
+    w.x = fmaf(-lr, d.x, w.x); w.y = fmaf(-lr, d.y, w.y); w.z = fmaf(-lr, d.z, w.z); w.w = fmaf(-lr, d.w, w.w);
+    *reinterpret_cast<float4*>(p + i) = w;
+    if (pt) { pt[i] = from_f32<T>(w.x); pt[i + 1] = from_f32<T>(w.y); pt[i + 2] = from_f32<T>(w.z); pt[i + 3] = from_f32<T>(w.w); }
+  } else {
+    for (size_t k = i; k < n; ++k) {
+      const float w = fmaf(-lr, g[k], p[k]);
+      p[k] = w;
+      if (pt) pt[k] = from_f32<T>(w);
+    }
+  }
+}
+
+template <typename T>
+cudaError_t sgd_update(float* params, const float* grads, T* params_t, float lr, size_t n, cudaStream_t st) {
+  sgd_update_kernel<T><<<(unsigned)((n / 4 + 256) / 256), 256, 0, st>>>(params, grads, params_t, lr, n);
+  return cudaGetLastError();
+}
+
 // wt_t[c][r][s][k] = w[k][2-r][2-s][c]: the filter rotated by 180 degrees with
 // the channel roles exchanged, so that the input gradient is itself a 3x3
 // correlation of dz (appendix row "reverse").
@@ -581,6 +608,7 @@ cudaError_t make_dgrad_filter(const float* w, T* wt_t, int Cin, int Cout, cudaSt
   template cudaError_t softmax_xent<T>(const float*, const int32_t*, float*, T*, float*, float*,     \
                                        int, int, cudaStream_t);                                      \
   template cudaError_t convert_f32<T>(const float*, T*, size_t, cudaStream_t);                       \
+  template cudaError_t sgd_update<T>(float*, const float*, T*, float, size_t, cudaStream_t);         \
   template cudaError_t make_dgrad_filter<T>(const float*, T*, int, int, cudaStream_t);
 
 INSTANTIATE(float)

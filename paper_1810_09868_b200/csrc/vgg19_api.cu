@@ -440,24 +440,32 @@ void drop_graphs(vgg19 *n) {
   n->graphs.clear();
 }
 
-int upload_params(vgg19 *n, const float *host) {
-  CUDA_TRY(n, cudaMemcpy(n->params, host, n->n_params * 4, cudaMemcpyHostToDevice));
+// The filter copies the kernels read besides the storage-type parameters (rotated filters of the input
+// gradients, tap-major filters, the padded first-layer filter), rebuilt from the fp32 master on `st`.
+int refresh_filter_copies(vgg19 *n, cudaStream_t st) {
   const bool h = n->cfg.dtype == VGG19_BF16;
-  if (h) CUDA_TRY(n, convert_f32<bf16>(n->params, (bf16 *)n->params_t, n->n_params, 0));
   for (int l = 1; l < kConvLayers; ++l) {
     const ConvLayer &c = n->conv[l];
     if (h)
-      CUDA_TRY(n, make_dgrad_filter<bf16>(n->params + c.w_off, (bf16 *)n->dgrad_w + c.dgrad_off, c.Cin, c.Cout, 0));
+      CUDA_TRY(n, make_dgrad_filter<bf16>(n->params + c.w_off, (bf16 *)n->dgrad_w + c.dgrad_off, c.Cin, c.Cout, st));
     else
-      CUDA_TRY(n, make_dgrad_filter<float>(n->params + c.w_off, (float *)n->dgrad_w + c.dgrad_off, c.Cin, c.Cout, 0));
+      CUDA_TRY(n, make_dgrad_filter<float>(n->params + c.w_off, (float *)n->dgrad_w + c.dgrad_off, c.Cin, c.Cout, st));
   }
-  if (n->w8) CUDA_TRY(n, tc_make_first_filter(n->params + n->conv[0].w_off, n->w8, 0));
+  if (n->w8) CUDA_TRY(n, tc_make_first_filter(n->params + n->conv[0].w_off, n->w8, st));
   if (n->tap_fwd)
     for (int l = 1; l < kConvLayers; ++l) {
       const ConvLayer &c = n->conv[l];
-      CUDA_TRY(n, tc_make_tap_major(n->params + c.w_off, n->tap_fwd + c.dgrad_off, c.Cin, c.Cout, false, 0));
-      CUDA_TRY(n, tc_make_tap_major(n->params + c.w_off, n->tap_bwd + c.dgrad_off, c.Cin, c.Cout, true, 0));
+      CUDA_TRY(n, tc_make_tap_major(n->params + c.w_off, n->tap_fwd + c.dgrad_off, c.Cin, c.Cout, false, st));
+      CUDA_TRY(n, tc_make_tap_major(n->params + c.w_off, n->tap_bwd + c.dgrad_off, c.Cin, c.Cout, true, st));
     }
+  return VGG19_OK;
+}
+
+int upload_params(vgg19 *n, const float *host) {
+  CUDA_TRY(n, cudaMemcpy(n->params, host, n->n_params * 4, cudaMemcpyHostToDevice));
+  if (n->cfg.dtype == VGG19_BF16) CUDA_TRY(n, convert_f32<bf16>(n->params, (bf16 *)n->params_t, n->n_params, 0));
+  int rc = refresh_filter_copies(n, 0);
+  if (rc != VGG19_OK) return rc;
   CUDA_TRY(n, cudaDeviceSynchronize());
   return VGG19_OK;
 }
@@ -605,6 +613,18 @@ int vgg19_set_params(vgg19_t *n, const float *host) {
   if (!n || !host) return VGG19_ERR_ARG;
   CUDA_TRY(n, cudaDeviceSynchronize());
   return upload_params(n, host);
+}
+
+int vgg19_sgd_step(vgg19_t *n, const float *grads, float lr, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!grads || !(lr == lr)) return fail(n, VGG19_ERR_ARG, "null gradient or NaN learning rate");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the parameter buffers keep their addresses, so recorded graphs stay valid
+  if (n->cfg.dtype == VGG19_BF16)
+    CUDA_TRY(n, sgd_update<bf16>(n->params, grads, (bf16 *)n->params_t, lr, n->n_params, st));
+  else
+    CUDA_TRY(n, sgd_update<float>(n->params, grads, (float *)nullptr, lr, n->n_params, st));
+  return refresh_filter_copies(n, st);
 }
 
 size_t vgg19_workspace_bytes(const vgg19_t *n, int32_t batch, int32_t mode) {

@@ -255,3 +255,34 @@ def test_host_buffer_entry_points():
     torch.cuda.synchronize()
     assert torch.equal(grads.cpu(), grads_host) and float(loss) == float(loss_host)
     net.close()
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_sgd_step_updates_every_copy_of_the_parameters(bf16):
+    """One gradient-descent step on the device against the checker's w - lr * g, then a second
+    forward + backward pass with the updated parameters against the checker: every copy of the
+    filters the kernels read (storage type, rotated, tap-major, padded) must have followed."""
+    p = pkg()
+    B, lr = 2, 0.05
+    params, images, labels = make_inputs(32, 32, B, bf16, bias_std=0.1)
+    net = p.Net(32, 32, B, p.VGG19_BF16 if bf16 else p.VGG19_FP32, params=params)
+    logits0, grads, _ = run_backward(net, images, labels)
+    net.sgd_step(torch.from_numpy(grads).to(DEV), lr)
+    net.sync_status()
+    new = np.empty_like(params)
+    p.vgg19_get_params(net.handle, new)
+    want = oracle.sgd_step(params, grads, lr)
+    assert rel_l2(new, want) <= 1e-6
+    assert rel_l2(new, params) > 1e-4  # the step moved the parameters
+    logits1, grads1, loss1 = run_backward(net, images, labels)
+    assert rel_l2(logits1, logits0) > 1e-3
+    if bf16:
+        # the device computes with the bf16 rounding of its fp32 master copy
+        used = oracle.round_bf16(new.astype(np.float64)).astype(np.float32)
+        check_bf16_backward(net, used, images, labels, logits1, grads1, loss1)
+    else:
+        o_loss, o_grads, o_logits = oracle.backward(oracle.vgg19_steps(), new.astype(np.float64), images, labels)
+        assert rel_l2(logits1, o_logits) <= 1e-4
+        assert abs(loss1 - o_loss) <= 1e-4 * abs(o_loss)
+        check_grads(net, grads1, o_grads, 2e-4)
+    net.close()

@@ -1,6 +1,9 @@
 """The N > 1 path of bench.py on CPU: two gloo ranks, each with its own timing;
 the reported time is the slowest rank's and the throughput counts every rank's
-batch (the forward pass shards over the batch with no collective)."""
+batch (the forward pass shards over the batch with no collective).  The
+training step's one exchange, the gradient all-reduce, is checked with the CPU
+checker standing in for the device: the mean of the ranks' half-batch gradients
+is the whole batch's gradient, and every rank takes the same SGD step."""
 import os
 import sys
 
@@ -44,3 +47,42 @@ def test_single_rank_needs_no_process_group():
     import bench
     assert bench.slowest_rank_ms(7.5, 1) == 7.5
     assert bench.aggregate_images_per_s(1, 100, 20, 100.0) == 20000.0
+
+
+def _grad_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import numpy as np
+    import bench
+    import oracle
+    from test_oracle_pins import TINY, tiny_inputs
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    params, x, labels = tiny_inputs(N=4)
+    half = slice(2 * rank, 2 * rank + 2)  # this rank's shard of the batch
+    _, g, _ = oracle.backward(TINY, params, x[half], labels[half])
+    t = torch.from_numpy(g.copy())
+    bench.average_gradients(t, world)
+    out[rank] = oracle.sgd_step(params, t.numpy(), 0.1)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_average_to_the_whole_batch_gradient():
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import numpy as np
+    import oracle
+    from test_oracle_pins import TINY, tiny_inputs
+    world = 2
+    port = 31500 + os.getpid() % 2000
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_grad_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    params, x, labels = tiny_inputs(N=4)
+    _, g_all, _ = oracle.backward(TINY, params, x, labels)
+    want = oracle.sgd_step(params, g_all, 0.1)
+    assert np.array_equal(res[0], res[1])  # replicas stay identical
+    assert np.allclose(res[0], want, rtol=1e-12, atol=1e-14)

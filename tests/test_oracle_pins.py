@@ -316,6 +316,22 @@ def test_finite_differences_on_a_tiny_net():
     assert np.count_nonzero(grads) > 0.5 * grads.size
 
 
+def test_sgd_step_closed_form_and_descent():
+    # quadratic L = a w^2 / 2: gradient a w, so a step gives w (1 - lr a), k steps w (1 - lr a)^k
+    w, a, lr = np.array([3.0, -1.5]), 2.0, 0.1
+    assert np.allclose(oracle.sgd_step(w, a * w, lr), [2.4, -1.2], rtol=0, atol=1e-15)
+    for _ in range(5):
+        w = oracle.sgd_step(w, a * w, lr)
+    assert np.allclose(w, np.array([3.0, -1.5]) * 0.8 ** 5, rtol=1e-14)
+    # on the tiny net a small step along the negative gradient lowers the loss by about lr |g|^2
+    params, x, labels = tiny_inputs()
+    loss, grads, _ = oracle.backward(TINY, params, x, labels)
+    lr = 1e-4
+    after = oracle.cross_entropy(oracle.forward(TINY, oracle.sgd_step(params, grads, lr), x), labels)
+    assert after < loss
+    assert abs((loss - after) - lr * float(grads @ grads)) <= 1e-2 * lr * float(grads @ grads)
+
+
 def torch_net(steps, params, x, labels):
     shapes = oracle.param_shapes(steps, x.shape[1], x.shape[2], x.shape[3])
     t = torch.from_numpy(params.copy()).requires_grad_(True)
