@@ -318,6 +318,17 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_
   return d;
 }
 
+// The general form: leading byte offset and stride byte offset both given (128-byte swizzle).
+__device__ __forceinline__ uint64_t smem_desc_sw128_full(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
 // Same for a K-major operand whose 8-row groups are `sbo_bytes` apart (rows of a
 // group still 128 bytes apart).  The start address may be any multiple of 128
 // bytes inside a 1024-byte-aligned buffer: the 128-byte swizzle is a function

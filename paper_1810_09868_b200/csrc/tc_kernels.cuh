@@ -60,6 +60,13 @@ int tc_wgrad_launches(ConvShape s, bool with_db, bool pairs = true);
 cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* db, float* partial, ConvShape s,
                              int* dev_error, cudaStream_t st, bool pairs = true);
 
+// The same filter gradient for layers with few channels (at most four 64 x 64 channel blocks), from
+// tiled patches of x and dz instead of im2col boxes (tc_wgrad_patch.cu); always two launches.
+bool tc_wgrad_patch_supported(ConvShape s);
+size_t tc_wgrad_patch_scratch_elems(ConvShape s);
+cudaError_t tc_conv3x3_wgrad_patch(const bf16* x, const bf16* dz, float* dW, float* db, float* partial, ConvShape s,
+                                   int* dev_error, cudaStream_t st);
+
 // Dense layers on the same GEMM kernel.  X [M][In], W [Out][In], dY [M][Out].
 bool tc_dense_supported(int M, int In, int Out);
 size_t tc_dense_scratch_elems(int M, int In, int Out);

@@ -131,6 +131,7 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
     size_t pe = simt_wgrad_scratch_elems(s);
     size_t te = tc_wgrad_scratch_elems(s, n->use_pair);
     if (te > pe) pe = te;
+    if (n->use_tc && tc_wgrad_patch_scratch_elems(s) > pe) pe = tc_wgrad_patch_scratch_elems(s);
     if (pe > max_partial) max_partial = pe;
     // tail-split scratch of the two-CTA convolution (forward, and input gradient with the channels swapped)
     if (n->use_pair) {
@@ -257,6 +258,8 @@ struct Pass {
     if (first_tc_ok(l, s)) {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       ok(tc_first_wgrad((const bf16 *)buf(p.x8), (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st), 2);
+    } else if (n->use_tc && tc_wgrad_patch_supported(s)) {
+      ok(tc_conv3x3_wgrad_patch((const bf16 *)x, (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st), 2);
     } else if (n->use_tc && tc_wgrad_supported(s)) {
       ok(tc_conv3x3_wgrad((const bf16 *)x, (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st, n->use_pair),
          tc_wgrad_launches(s, db != nullptr, n->use_pair));
