@@ -140,6 +140,19 @@ int vgg19_forward_host(vgg19_t *net, const void *host_images, int32_t batch, flo
 int vgg19_backward_host(vgg19_t *net, const void *host_images, const int32_t *host_labels,
                         int32_t batch, float *host_grads, float *host_loss, void *stream);
 
+/* vgg19_forward_host without the wait: the upload runs on a stream of the
+ * library's own into one of two staging slots (taken in turn), the pass and the
+ * download of its results are enqueued on `stream`, and the call returns.  A
+ * caller that enqueues batch after batch gets the upload of the next batch
+ * overlapped with the pass of the current one - how a serving loop would feed
+ * the executable of section 7.2.  host_images must stay untouched, and the
+ * results are not in host_logits / host_probs, until `stream` has been waited
+ * for (vgg19_sync_status); with more than two calls in flight the library orders
+ * the reuse of a slot itself.  stream must not be the legacy default stream.
+ * Needs the same workspace as vgg19_forward_host (vgg19_io_bytes counts both slots). */
+int vgg19_forward_host_async(vgg19_t *net, const void *host_images, int32_t batch, float *host_logits,
+                             float *host_probs, void *stream);
+
 /* Single convolution layer (3x3, pad 1, stride 1) + bias + ReLU, optionally
  * followed by the 2x2 max-pool, on caller-supplied device tensors in the
  * config's dtype; the per-layer building block of section 7.2, exposed for

@@ -21,7 +21,7 @@ VGG19_MODE_FORWARD, VGG19_MODE_BACKWARD = 0, 1
 EXPORTS = (
     "vgg19_create", "vgg19_create_from_params", "vgg19_destroy", "vgg19_param_count", "vgg19_param_info",
     "vgg19_get_params", "vgg19_set_params", "vgg19_workspace_bytes", "vgg19_bind_workspace",
-    "vgg19_forward", "vgg19_backward", "vgg19_sgd_step", "vgg19_io_bytes", "vgg19_forward_host", "vgg19_backward_host",
+    "vgg19_forward", "vgg19_backward", "vgg19_sgd_step", "vgg19_io_bytes", "vgg19_forward_host", "vgg19_forward_host_async", "vgg19_backward_host",
     "vgg19_conv_layer_forward", "vgg19_conv_layer_backward", "vgg19_saved_tensor", "vgg19_conv_wgrad_static", "vgg19_sync_status", "vgg19_launch_count",
     "vgg19_describe", "vgg19_last_error",
 )
@@ -72,6 +72,7 @@ def load():
         "vgg19_sgd_step": ([vp, vp, ctypes.c_float, vp], ctypes.c_int),
         "vgg19_io_bytes": ([vp, i32, i32], sz),
         "vgg19_forward_host": ([vp, vp, i32, vp, vp, vp], ctypes.c_int),
+        "vgg19_forward_host_async": ([vp, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_backward_host": ([vp, vp, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_forward": ([vp, i32, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_backward": ([vp, i32, vp, vp, i32, vp, vp, vp, vp], ctypes.c_int),
@@ -182,6 +183,11 @@ def vgg19_backward(net, images, labels, batch, grads, loss=None, logits=None, st
 def vgg19_forward_host(net, host_images, batch, host_logits, host_probs=None, stream=None):
     return _check(net, load().vgg19_forward_host(net, _ptr(host_images), batch, _ptr(host_logits),
                                                   _ptr(host_probs), _stream(stream)))
+
+
+def vgg19_forward_host_async(net, host_images, batch, host_logits, host_probs=None, stream=None):
+    return _check(net, load().vgg19_forward_host_async(net, _ptr(host_images), batch, _ptr(host_logits),
+                                                        _ptr(host_probs), _stream(stream)))
 
 
 def vgg19_backward_host(net, host_images, host_labels, batch, host_grads, host_loss=None, stream=None):

@@ -73,6 +73,12 @@ struct vgg19 {
   std::string err;
   bool use_tc = false;
   bool use_pair = false;  // two-CTA kernels where a layer's shape takes them
+  // vgg19_forward_host_async: two staging slots, a stream of the library's own for the uploads, and per
+  // slot an event for "images uploaded" and one for "the pass that used the slot has finished"
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_uploaded[2] = {nullptr, nullptr}, ev_consumed[2] = {nullptr, nullptr};
+  bool slot_used[2] = {false, false};
+  unsigned next_slot = 0;
 };
 
 namespace {
@@ -574,6 +580,11 @@ void vgg19_destroy(vgg19_t *n) {
   if (n->tap_fwd) cudaFree(n->tap_fwd);
   if (n->tap_bwd) cudaFree(n->tap_bwd);
   if (n->dev_error) cudaFree(n->dev_error);
+  if (n->copy_stream) cudaStreamDestroy(n->copy_stream);
+  for (int i = 0; i < 2; ++i) {
+    if (n->ev_uploaded[i]) cudaEventDestroy(n->ev_uploaded[i]);
+    if (n->ev_consumed[i]) cudaEventDestroy(n->ev_consumed[i]);
+  }
   delete n;
 }
 
@@ -637,7 +648,9 @@ size_t vgg19_workspace_bytes(const vgg19_t *n, int32_t batch, int32_t mode) {
 
 size_t vgg19_io_bytes(const vgg19_t *n, int32_t batch, int32_t mode) {
   if (!n || batch < 1 || batch > n->cfg.batch_max || (mode != 0 && mode != 1)) return 0;
-  return make_plan(n, batch, mode).io_total;
+  // the forward staging area is doubled: vgg19_forward_host_async alternates between two slots
+  const Plan p = make_plan(n, batch, mode);
+  return mode == VGG19_MODE_FORWARD ? 2 * p.io_total : p.io_total;
 }
 
 int vgg19_bind_workspace(vgg19_t *n, void *ws, size_t bytes) {
@@ -693,6 +706,45 @@ int vgg19_forward_host(vgg19_t *n, const void *host_images, int32_t batch, float
   if (host_logits) CUDA_TRY(n, cudaMemcpyAsync(host_logits, logits, out_bytes, cudaMemcpyDeviceToHost, st));
   if (host_probs) CUDA_TRY(n, cudaMemcpyAsync(host_probs, probs, out_bytes, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(n, cudaStreamSynchronize(st));
+  return VGG19_OK;
+}
+
+int vgg19_forward_host_async(vgg19_t *n, const void *host_images, int32_t batch, float *host_logits,
+                             float *host_probs, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!host_images) return fail(n, VGG19_ERR_ARG, "host_images must not be null");
+  int rc = check_batch(n, batch, VGG19_MODE_FORWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  Plan p = make_plan(n, batch, VGG19_MODE_FORWARD);
+  rc = check_batch(n, batch, VGG19_MODE_FORWARD, 2 * p.io_total);
+  if (rc != VGG19_OK) return rc;
+  if (!n->copy_stream) {
+    CUDA_TRY(n, cudaStreamCreateWithFlags(&n->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+      CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_uploaded[i], cudaEventDisableTiming));
+      CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_consumed[i], cudaEventDisableTiming));
+    }
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const unsigned slot = n->next_slot++ & 1u;
+  char *base = static_cast<char *>(n->ws) + (size_t)slot * p.io_total;
+  size_t img_bytes = (size_t)batch * n->cfg.height * n->cfg.width * 3 * n->elt;
+  // upload on the library's stream, as soon as the pass that last read this slot is done: it overlaps
+  // whatever `stream` is still computing
+  if (n->slot_used[slot]) CUDA_TRY(n, cudaStreamWaitEvent(n->copy_stream, n->ev_consumed[slot], 0));
+  CUDA_TRY(n, cudaMemcpyAsync(base + p.io_images, host_images, img_bytes, cudaMemcpyHostToDevice, n->copy_stream));
+  CUDA_TRY(n, cudaEventRecord(n->ev_uploaded[slot], n->copy_stream));
+  CUDA_TRY(n, cudaStreamWaitEvent(st, n->ev_uploaded[slot], 0));
+  float *logits = reinterpret_cast<float *>(base + p.io_logits);
+  float *probs = host_probs ? reinterpret_cast<float *>(base + p.io_probs) : nullptr;
+  PassArgs a{base + p.io_images, nullptr, logits, probs, nullptr, nullptr, batch};
+  rc = run_pass(n, VGG19_MODE_FORWARD, a, st);
+  if (rc != VGG19_OK) return rc;
+  size_t out_bytes = (size_t)batch * kClasses * 4;
+  if (host_logits) CUDA_TRY(n, cudaMemcpyAsync(host_logits, logits, out_bytes, cudaMemcpyDeviceToHost, st));
+  if (host_probs) CUDA_TRY(n, cudaMemcpyAsync(host_probs, probs, out_bytes, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(n, cudaEventRecord(n->ev_consumed[slot], st));
+  n->slot_used[slot] = true;
   return VGG19_OK;
 }
 

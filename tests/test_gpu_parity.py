@@ -286,3 +286,28 @@ def test_sgd_step_updates_every_copy_of_the_parameters(bf16):
         assert abs(loss1 - o_loss) <= 1e-4 * abs(o_loss)
         check_grads(net, grads1, o_grads, 2e-4)
     net.close()
+
+
+def test_async_host_entry_point_matches_the_blocking_one():
+    """Five batches in flight through vgg19_forward_host_async (two staging slots, uploads on the
+    library's own stream) give bit for bit the logits of vgg19_forward_host on the same images."""
+    p = pkg()
+    B = 3
+    params, _, _ = make_inputs(32, 32, B, True)
+    net = p.Net(32, 32, B, p.VGG19_BF16, params=params, mode=p.VGG19_MODE_FORWARD, host_io=True)
+    stream = torch.cuda.Stream()
+    batches = [torch.from_numpy(si.images(B, 32, 32, seed=10 + i, bf16_exact=True)).to(torch.bfloat16).pin_memory()
+               for i in range(5)]
+    want = []
+    for x in batches:
+        out = torch.empty(B, 1000, dtype=torch.float32).pin_memory()
+        p.vgg19_forward_host(net.handle, x, B, out, None, stream)
+        want.append(out.clone())
+    got = [torch.full((B, 1000), float("nan"), dtype=torch.float32).pin_memory() for _ in batches]
+    for x, out in zip(batches, got):
+        p.vgg19_forward_host_async(net.handle, x, B, out, None, stream)
+    net.sync_status(stream)
+    for g, w in zip(got, want):
+        assert torch.equal(g, w)
+    assert not torch.equal(want[0], want[1])
+    net.close()
