@@ -509,18 +509,24 @@ cudaError_t tc_make_tap_major(const float* w, bf16* out, int Cin, int Cout, bool
 }
 
 bool tc_conv3x3_halo_supported(ConvShape s) {
-  return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.Cout <= 128 && s.W % PW == 0 && s.H % PH == 0 && s.W >= 64 &&
-         (long)s.N * s.H * s.W < (1L << 31) - 256;
+  return tc_conv3x3_halo_supported_unpooled(s) && s.H % PH == 0 && s.W >= 64;
+}
+
+// Without a pooled output the image height need not be a whole number of patches: the copy engine
+// zero-fills the rows a last patch reads past the image and clips the rows it would store there.
+bool tc_conv3x3_halo_supported_unpooled(ConvShape s) {
+  return s.Cin % 64 == 0 && s.Cout % 64 == 0 && s.Cout <= 128 && s.W % PW == 0 && s.H >= PH && s.W >= 56 &&
+         (long)s.N * (s.H + PH) * s.W < (1L << 31) - 256;
 }
 
 cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
                             bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, bool pairs) {
   if (!out && !pooled) return cudaErrorInvalidValue;
-  if (!tc_conv3x3_halo_supported(s)) return cudaErrorInvalidValue;
+  if (!(pooled ? tc_conv3x3_halo_supported(s) : tc_conv3x3_halo_supported_unpooled(s))) return cudaErrorInvalidValue;
   const int BN = s.Cout % 128 == 0 ? 128 : 64;
   // CTA pairs take two tiles at a time.  They pay with 128 output channels, where one CTA's MMAs are
   // bound by shared-memory reads; with 64 they measure the same as single CTAs, which are kept there.
-  const bool pair = pairs && BN == 128 && (s.N * (s.W / PW) * (s.H / PH)) % 2 == 0;
+  const bool pair = pairs && BN == 128 && (s.N * (s.W / PW) * ((s.H + PH - 1) / PH)) % 2 == 0;
   CUtensorMap mx, mw;
   if (!make_patch_map(&mx, in, s.N, s.H, s.W, s.Cin, IW, IH)) return cudaErrorInvalidValue;
   if (!make_filter_row_map(&mw, wt_tap_major, s.Cout, s.Cin, (uint32_t)(pair ? BN / 2 : BN))) return cudaErrorInvalidValue;
@@ -532,7 +538,7 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const floa
   HaloArgs a;
   a.N = s.N; a.H = s.H; a.W = s.W;
   a.cin_blocks = s.Cin / 64; a.Cin = s.Cin; a.Cout = s.Cout;
-  a.tiles_w = s.W / PW; a.tiles_h = s.H / PH;
+  a.tiles_w = s.W / PW; a.tiles_h = (s.H + PH - 1) / PH;
   a.m_tiles = s.N * a.tiles_w * a.tiles_h;
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0; a.bias = bias; a.mask = mask; a.out = out; a.pooled = pooled; a.dev_error = dev_error;

@@ -32,6 +32,7 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
 // The same convolution with the input patch (plus halo) kept in shared memory
 // for all nine taps (tc_conv_halo.cu): the large-image, few-channel layers.
 bool tc_conv3x3_halo_supported(ConvShape s);
+bool tc_conv3x3_halo_supported_unpooled(ConvShape s);  // shapes it takes when no pooled output is asked for
 // The filter comes tap-major, [9][Cout][Cin] (tc_make_tap_major builds it from the fp32 [Cout][3][3][Cin]
 // master; for_dgrad gives the rotated, channel-swapped filter of the input gradient, [9][Cin][Cout]).
 // `pooled` (or null) also receives the 2x2 max-pool of the result; `out` may then be null.

@@ -277,7 +277,7 @@ struct Pass {
       if (n->use_tc && tc_conv3x3_rowshift_supported(t))
         ok(tc_conv3x3_rowshift((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr,
                                t, false, n->dev_error, st), 1);
-      else if (n->use_tc && tc_conv3x3_halo_supported(t))
+      else if (n->use_tc && tc_conv3x3_halo_supported_unpooled(t))
         ok(tc_conv3x3_halo((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr, t,
                            false, n->dev_error, st, n->use_pair), 1);
       else if (pair_ok(t)) {
