@@ -331,8 +331,8 @@ def run_native(args):
     per_layer = {f"conv{l}": {"ms": round(ms, 4), "tflops": round(f / (ms * 1e-3) / 1e12, 1), "path": path}
                  for l, ms, f, path in layers}
     # dram__bytes_read+write of one launch of this kernel on layer 6 (56x56, 256->256), captured with
-    # ncu at batch 48 (113.7 MB) and scaled by the pixel count to the batch-100 launch timed here
-    traffic = 113.70e6 * BATCH / 48
+    # ncu at batch 48 (113.5 MB) and scaled by the pixel count to the batch-100 launch timed here
+    traffic = 113.47e6 * BATCH / 48
 
     n_fwd = pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_FORWARD)
     cpu_rate, cpu_dt = oracle_forward_rate(args.cpu_images)
