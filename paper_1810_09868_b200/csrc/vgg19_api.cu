@@ -879,11 +879,26 @@ int vgg19_describe(const vgg19_t *n, char *out, size_t cap) {
     const ConvLayer &c = n->conv[l];
     ConvShape sh{n->cfg.batch_max, c.H, c.W, c.Cin, c.Cout};
     ConvShape sd{n->cfg.batch_max, c.H, c.W, c.Cout, c.Cin};
+    // the kernel each pass picks for this layer, in the order the scheduler tries them
+    const char *fwd = !n->use_tc ? "simt"
+                      : l == 0 ? (tc_first_conv_supported(sh) ? "tcgen05:first-layer" : "simt")
+                      : tc_conv3x3_rowshift_supported(sh) ? "tcgen05:row-shift"
+                      : tc_conv3x3_halo_supported(sh) ? (n->use_pair && c.Cout == 128 ? "tcgen05:halo-pair" : "tcgen05:halo")
+                      : n->use_pair && tc_conv3x3_pair_supported(sh) ? "tcgen05:pair"
+                      : tc_conv3x3_supported(sh) ? "tcgen05:im2col" : "simt";
+    const char *dgrad = l == 0 ? "none"
+                        : !n->use_tc ? "simt"
+                        : tc_conv3x3_rowshift_supported(sd) ? "tcgen05:row-shift"
+                        : tc_conv3x3_halo_supported_unpooled(sd) ? (n->use_pair && c.Cin == 128 ? "tcgen05:halo-pair" : "tcgen05:halo")
+                        : n->use_pair && tc_conv3x3_pair_supported(sd) ? "tcgen05:pair"
+                        : tc_conv3x3_supported(sd) ? "tcgen05:im2col" : "simt";
+    const char *wgrad = !n->use_tc ? "simt"
+                        : l == 0 ? (tc_first_conv_supported(sh) ? "tcgen05:gemm-8ch" : "simt")
+                        : tc_wgrad_patch_supported(sh) ? "tcgen05:patch"
+                        : tc_wgrad_supported(sh) ? (n->use_pair && c.Cin % 256 == 0 && c.Cout % 256 == 0 ? "tcgen05:gemm-pair" : "tcgen05:gemm")
+                        : "simt";
     snprintf(line, sizeof line, "conv%-2d %3dx%-3d %3d->%-3d +bias +relu%s  fwd=%s dgrad=%s wgrad=%s\n",
-             l + 1, c.H, c.W, c.Cin, c.Cout, c.pool_after ? " +maxpool2x2" : "",
-             n->use_tc && (tc_conv3x3_supported(sh) || (l == 0 && tc_first_conv_supported(sh))) ? "tcgen05" : "simt",
-             l == 0 ? "none" : (n->use_tc && tc_conv3x3_supported(sd) ? "tcgen05" : "simt"),
-             n->use_tc && (tc_wgrad_supported(sh) || (l == 0 && tc_first_conv_supported(sh))) ? "tcgen05" : "simt");
+             l + 1, c.H, c.W, c.Cin, c.Cout, c.pool_after ? " +maxpool2x2" : "", fwd, dgrad, wgrad);
     s += line;
   }
   for (int i = 0; i < kFcLayers; ++i) {
