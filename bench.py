@@ -6,14 +6,17 @@ One "step" is one forward pass of the whole network on a batch of 100
 224x224x3 bf16 images (the paper's headline shape, figure "Timings for the
 VGG19 forward pass", N=100).  Rank 0 prints ONE JSON line: images/s with the
 inputs resident in HBM (`value`), the same through the host-buffer entry point
-with copies inside the timed region (`e2e`), the forward+backward training-step
-throughput (`fwd_bwd`), the roofline of the dominant kernel (the tensor-core
-implicit-GEMM convolution, timed per layer with CUDA events), and the fp64 CPU
-checker timed on a bounded sample (`cpu_baseline`).
+with copies inside the timed region (`e2e`), the forward+backward throughput
+(`fwd_bwd`) and that of a whole training step with the SGD update
+(`train_step`), the roofline of the dominant kernel (the tensor-core
+implicit-GEMM convolution on CTA pairs, timed per layer with CUDA events), the
+achieved bandwidth of the largest memory-bound kernel (`hbm_bound`), and the
+fp64 CPU checker timed on a bounded sample (`cpu_baseline`).
 
 With N > 1 (torchrun) every rank runs the same batch-100 pass on its own GPU:
 the path shards over the batch with no collective in the forward pass, so the
-aggregate is N * 100 images per step over the slowest rank's time.
+aggregate is N * 100 images per step over the slowest rank's time; the training
+step adds its one exchange, an all-reduce of the gradients.
 
 --impl reference times the CPU checker itself (rank 0 only).
 """
@@ -188,7 +191,7 @@ def time_conv_layers(pkg, net, torch, stream, reps=5):
     scratch = torch.empty(BATCH * 224 * 224 * 64, dtype=torch.bfloat16, device=net.device)
     for l, (s, ci, co) in enumerate(CONV):
         if l == 0:
-            continue  # 3 input channels: HBM-bound CUDA-core kernel, not the tensor-core one
+            continue  # 3 input channels: bound by writing its output (see time_first_layer)
         prev = l - 1
         x = net.saved_tensor(BATCH, pkg.VGG19_MODE_BACKWARD, prev)
         if x.shape[1] != s:  # a pool sits between: input is the pooled tensor
@@ -207,6 +210,24 @@ def time_conv_layers(pkg, net, torch, stream, reps=5):
         ms = sum(a.elapsed_time(b) for a, b in evs) / reps
         out.append((l + 1, ms, 2.0 * BATCH * s * s * co * 9 * ci, path))
     return out
+
+
+def time_first_layer(pkg, net, torch, stream, x, reps=5):
+    """conv1_1 (3 -> 64 channels), the pass's largest memory-bound kernel: CUDA-event time of the layer
+    (channel-padding copy + convolution) and the algorithmic bytes it has to move: the 3-channel image in,
+    the 64-channel activation out."""
+    y = torch.empty(BATCH, H, W, 64, dtype=torch.bfloat16, device=net.device)
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            pkg.vgg19_conv_layer_forward(net.handle, 1, x, BATCH, y, None, stream)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in evs:
+            a.record(stream)
+            pkg.vgg19_conv_layer_forward(net.handle, 1, x, BATCH, y, None, stream)
+            b.record(stream)
+    stream.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in evs) / reps
+    return ms, BATCH * H * W * (3 + 64) * 2
 
 
 def run_native(args):
@@ -320,6 +341,7 @@ def run_native(args):
         bwd()  # leaves the batch-100 activations of every layer in the workspace
     stream.synchronize()
     layers = time_conv_layers(pkg, net, torch, stream)
+    first_ms, first_bytes = time_first_layer(pkg, net, torch, stream, x)
     # dominant kernel: conv3x3_pair_tc_kernel<256>, the 12 launches of layers 5..16 (60 % of the pass)
     dom = [t for t in layers if t[0] >= 5]
     conv_ms = sum(ms for _, ms, _, _ in dom)
@@ -370,6 +392,10 @@ def run_native(args):
                      "all_conv_layers_2_16": {"tflops": all_flop / (all_ms * 1e-3) / 1e12,
                                               "frac": all_flop / (all_ms * 1e-3) / 1e12 / peak},
                      "per_layer": per_layer},
+        "hbm_bound": {"kernel": "conv1_1 forward (pad_to8_kernel + conv3x3_c8_tc_kernel): 3-channel image in, 64-channel activation out",
+                      "ms": round(first_ms, 4), "achieved": first_bytes / (first_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
+                      "unit": "GB/s", "frac": first_bytes / (first_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                      "peak_source": f"{pk['source']} copy bandwidth"},
         "cpu_baseline": {"value": cpu_rate, "unit": "images/s", "cores": os.cpu_count(), "kind": "oracle",
                          "sample": f"forward of {args.cpu_images} of the 100 images, {cpu_dt:.1f} s"},
         "context": {"paper_tpuv2_core_s_per_batch100": 0.23, "paper_xeon_4114_flux_cpu_s_per_batch100": 52.4},
