@@ -69,8 +69,8 @@ typedef struct {
 
 /* Build a network whose parameters are the seeded He-normal set (weights
  * N(0, 2/fan_in), biases 0) drawn on the host from `seed` and uploaded.  The
- * library owns the parameters.  (North-star entry point "vgg19_create from a
- * seeded weight set"; the paper itself used trained weights, section 7.2.) */
+ * library owns the parameters.  (The paper itself used trained weights,
+ * section 7.2; a seeded random set stands in for them.) */
 int vgg19_create(const vgg19_config *cfg, uint64_t seed, vgg19_t **out);
 
 /* Same, from a caller-supplied flat fp32 HOST buffer of vgg19_param_count()
@@ -113,8 +113,7 @@ int vgg19_forward(vgg19_t *net, const void *images, int32_t batch, float *logits
  * [batch] in [0,1000).  grads: device fp32, vgg19_param_count() elements,
  * fully overwritten with d(loss)/d(parameter), loss = mean cross-entropy.
  * loss: device fp32 scalar or NULL.  logits: device fp32 [batch][1000] or
- * NULL.  The batch argument is an addition to the spec signature, which
- * leaves the batch size implicit. */
+ * NULL.  batch: number of images in this call, at most the config's batch_max. */
 int vgg19_backward(vgg19_t *net, const void *images, const int32_t *labels, int32_t batch,
                    float *grads, float *loss, float *logits, void *stream);
 
