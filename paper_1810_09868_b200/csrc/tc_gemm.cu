@@ -410,8 +410,17 @@ __global__ void splitk_finish_kernel(const float* __restrict__ partial, int spli
   }
   const long i = t * 4;
   if (i >= MN) return;
+  // independent loads, issued several at a time; the additions stay in split order
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int z = 0; z < splits; ++z) {
+  int z = 0;
+  for (; z + 4 <= splits; z += 4) {
+    float4 p[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) p[u] = *reinterpret_cast<const float4*>(partial + (long)(z + u) * MN + i);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { s.x += p[u].x; s.y += p[u].y; s.z += p[u].z; s.w += p[u].w; }
+  }
+  for (; z < splits; ++z) {
     const float4 p = *reinterpret_cast<const float4*>(partial + (long)z * MN + i);
     s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
   }

@@ -212,8 +212,19 @@ __global__ void wgrad_patch_finish_kernel(const float* __restrict__ partial, int
   const int tile = cb * (Cout / 64) + kb;
   const int col = (2 - s9) * 64 + kl;
   const size_t off = r < 2 ? (size_t)(r * 64 + cl) * 192 + col : (size_t)128 * 192 + (size_t)cl * 192 + col;
+  // independent loads, issued several at a time; the additions stay in split order
   float sum = 0.f;
-  for (int z = 0; z < splits; ++z) sum += partial[((size_t)z * tiles + tile) * kPartialFloats + off];
+  const float* src = partial + (size_t)tile * kPartialFloats + off;
+  const size_t stride = (size_t)tiles * kPartialFloats;
+  int z = 0;
+  for (; z + 8 <= splits; z += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = src[(size_t)(z + u) * stride];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) sum += v[u];
+  }
+  for (; z < splits; ++z) sum += src[(size_t)z * stride];
   dW[((size_t)k * 9 + r * 3 + s9) * Cin + c] = sum;
 }
 
