@@ -91,6 +91,23 @@ cudaError_t softmax_xent(const float* logits, const int32_t* labels, float* prob
 // fp32 -> T copy (weights), and the dgrad filter: wt_t[c][r][s][k] = w[k][2-r][2-s][c].
 template <typename T>
 cudaError_t convert_f32(const float* src, T* dst, size_t n, cudaStream_t st);
+// Where the filters of layers 2..16 sit: in the flat fp32 parameter buffer (w_off) and in the three
+// bf16 copy buffers (copy_off, the same in each); first[l] = number of 32 x 32 tiles (per tap, of the
+// [Cout][Cin] matrix) before layer l, total = all tiles.  Cin and Cout are multiples of 32.
+struct FilterCopyTable {
+  int layers;
+  long total;
+  long first[16];
+  long w_off[16];
+  long copy_off[16];
+  int Cin[16], Cout[16];
+};
+// Rebuilds, from the fp32 master, the rotated filters of the input gradients ([Cin][3][3][Cout], rotated
+// by 180 degrees), the tap-major filters [9][Cout][Cin] and the rotated tap-major filters [9][Cin][Cout]
+// of every layer in the table, all bf16, in one launch.
+cudaError_t refresh_filter_copies(const float* params, bf16* dgrad_w, bf16* tap_fwd, bf16* tap_bwd,
+                                  const FilterCopyTable& tab, cudaStream_t st);
+
 // params -= lr * grads (fp32 master, in place); params_t (the storage-type copy, or null when T is
 // float and the master is the copy) receives the rounded result in the same pass.
 template <typename T>

@@ -553,7 +553,14 @@ __global__ void sgd_update_kernel(float* __restrict__ p, const float* __restrict
     const float4 d = *reinterpret_cast<const float4*>(g + i);
     w.x = fmaf(-lr, d.x, w.x); w.y = fmaf(-lr, d.y, w.y); w.z = fmaf(-lr, d.z, w.z); w.w = fmaf(-lr, d.w, w.w);
     *reinterpret_cast<float4*>(p + i) = w;
-    if (pt) { pt[i] = from_f32<T>(w.x); pt[i + 1] = from_f32<T>(w.y); pt[i + 2] = from_f32<T>(w.z); pt[i + 3] = from_f32<T>(w.w); }
+    if (pt) {
+      if (sizeof(T) == 2) {  // four bf16 as one 8-byte store (i is a multiple of 4, the buffer 256-byte aligned)
+        __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+        *reinterpret_cast<uint2*>(pt + i) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+      } else {
+        pt[i] = from_f32<T>(w.x); pt[i + 1] = from_f32<T>(w.y); pt[i + 2] = from_f32<T>(w.z); pt[i + 3] = from_f32<T>(w.w);
+      }
+    }
   } else {
     for (size_t k = i; k < n; ++k) {
       const float w = fmaf(-lr, g[k], p[k]);
@@ -586,6 +593,51 @@ template <typename T>
 cudaError_t make_dgrad_filter(const float* w, T* wt_t, int Cin, int Cout, cudaStream_t st) {
   long total = (long)Cin * 9 * Cout;
   dgrad_filter_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w, wt_t, Cin, Cout);
+  return cudaGetLastError();
+}
+
+// All three bf16 copies of the filters of up to 15 layers in one pass over the fp32 master: for
+// w[k][tap][c] of a layer, the rotated filter of the input gradient [c][8 - tap][k], the tap-major
+// filter [tap][k][c] and the rotated tap-major filter [8 - tap][c][k].  Two of the three are
+// transposes of the [Cout][Cin] matrix of a tap: a block takes a 32 x 32 tile of it through shared
+// memory so that reads and all three writes are contiguous.  first[] counts tiles here.
+__global__ void refresh_filter_copies_kernel(const float* __restrict__ params, bf16* __restrict__ dgrad_w,
+                                             bf16* __restrict__ tap_fwd, bf16* __restrict__ tap_bwd,
+                                             FilterCopyTable tab) {
+  __shared__ float tile[32][33];
+  const long b = blockIdx.x;
+  int l = 0;
+  while (l + 1 < tab.layers && b >= tab.first[l + 1]) ++l;  // first[] is ascending
+  const int Cin = tab.Cin[l], Cout = tab.Cout[l];
+  long t = b - tab.first[l];
+  const int c_tiles = Cin / 32;
+  const int c0 = (int)(t % c_tiles) * 32; t /= c_tiles;
+  const int k_tiles = Cout / 32;
+  const int k0 = (int)(t % k_tiles) * 32;
+  const int tap = (int)(t / k_tiles);
+  const float* w = params + tab.w_off[l];
+  const size_t base = tab.copy_off[l];
+  const int tx = threadIdx.x, ty = threadIdx.y;  // 32 x 8
+#pragma unroll
+  for (int j = 0; j < 32; j += 8) {
+    const int k = k0 + ty + j, c = c0 + tx;
+    const float v = w[((size_t)k * 9 + tap) * Cin + c];
+    tile[ty + j][tx] = v;
+    tap_fwd[base + ((size_t)tap * Cout + k) * Cin + c] = __float2bfloat16_rn(v);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < 32; j += 8) {
+    const int c = c0 + ty + j, k = k0 + tx;
+    const bf16 v = __float2bfloat16_rn(tile[tx][ty + j]);
+    dgrad_w[base + ((size_t)c * 9 + (8 - tap)) * Cout + k] = v;
+    tap_bwd[base + ((size_t)(8 - tap) * Cin + c) * Cout + k] = v;
+  }
+}
+
+cudaError_t refresh_filter_copies(const float* params, bf16* dgrad_w, bf16* tap_fwd, bf16* tap_bwd,
+                                  const FilterCopyTable& tab, cudaStream_t st) {
+  refresh_filter_copies_kernel<<<(unsigned)tab.total, dim3(32, 8), 0, st>>>(params, dgrad_w, tap_fwd, tap_bwd, tab);
   return cudaGetLastError();
 }
 

@@ -453,6 +453,24 @@ void drop_graphs(vgg19 *n) {
 // gradients, tap-major filters, the padded first-layer filter), rebuilt from the fp32 master on `st`.
 int refresh_filter_copies(vgg19 *n, cudaStream_t st) {
   const bool h = n->cfg.dtype == VGG19_BF16;
+  if (h && n->tap_fwd && n->tap_bwd) {
+    // tensor-core configuration: all three bf16 copies of layers 2..16 in one launch
+    FilterCopyTable tab{};
+    tab.layers = kConvLayers - 1;
+    long first = 0;
+    for (int l = 1; l < kConvLayers; ++l) {
+      const ConvLayer &c = n->conv[l];
+      tab.first[l - 1] = first;
+      tab.w_off[l - 1] = (long)c.w_off;
+      tab.copy_off[l - 1] = (long)c.dgrad_off;
+      tab.Cin[l - 1] = c.Cin; tab.Cout[l - 1] = c.Cout;
+      first += 9L * (c.Cin / 32) * (c.Cout / 32);
+    }
+    tab.total = first;
+    CUDA_TRY(n, vgg::refresh_filter_copies(n->params, (bf16 *)n->dgrad_w, n->tap_fwd, n->tap_bwd, tab, st));
+    if (n->w8) CUDA_TRY(n, tc_make_first_filter(n->params + n->conv[0].w_off, n->w8, st));
+    return VGG19_OK;
+  }
   for (int l = 1; l < kConvLayers; ++l) {
     const ConvLayer &c = n->conv[l];
     if (h)
