@@ -13,10 +13,14 @@ implicit-GEMM convolution on CTA pairs, timed per layer with CUDA events), the
 achieved bandwidth of the largest memory-bound kernel (`hbm_bound`), and the
 fp64 CPU checker timed on a bounded sample (`cpu_baseline`).
 
-With N > 1 (torchrun) every rank runs the same batch-100 pass on its own GPU:
-the path shards over the batch with no collective in the forward pass, so the
-aggregate is N * 100 images per step over the slowest rank's time; the training
-step adds its one exchange, an all-reduce of the gradients.
+With N > 1 every rank runs the same batch-100 pass on its own GPU: the path
+shards over the batch with no collective in the forward pass, so the aggregate
+is N * 100 images per step over the slowest rank's time; the training step adds
+its one exchange, an all-reduce of the gradients.  Under torchrun the ranks are
+the launcher's; a plain `python bench.py --gpus N` (no WORLD_SIZE in the
+environment) starts N ranks itself through torch.distributed.run.
+`--backend gloo --dry` runs only the multi-rank plumbing (rendezvous, barrier,
+max over ranks, gradient averaging, aggregation) on CPU ranks, for tests.
 
 --impl reference times the CPU checker itself (rank 0 only).
 """
@@ -75,8 +79,9 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def stop(self, t_begin=None, t_end=None):
-        """Summary of the samples taken between the two wall-clock times (all samples if none fall inside)."""
+    def stop(self, t_begin=None, t_end=None, extra_window=None):
+        """Summary of the samples taken between the two wall-clock times (all samples if none fall inside);
+        with extra_window=(t0, t1) also {"extra": summary of the samples inside that second window}."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -101,12 +106,61 @@ class ClockSampler:
                 continue
         self.file.close()
         os.unlink(self.file.name)
-        inside = [r for r in rows if t_begin is not None and t_begin <= r[0] <= t_end]
-        use = inside if inside else rows
-        reasons = sorted({n for r in use for n in r[3]})
-        return {"sm_mhz": statistics.median(r[1] for r in use) if use else None,
-                "sm_max_mhz": max(r[2] for r in use) if use else None,
-                "samples": len(use), "window": "timed region" if inside else "whole run", "reasons": reasons}
+        def summary(t0, t1, label):
+            inside = [r for r in rows if t0 is not None and t0 <= r[0] <= t1]
+            use = inside if inside else rows
+            reasons = sorted({n for r in use for n in r[3]})
+            return {"sm_mhz": statistics.median(r[1] for r in use) if use else None,
+                    "sm_max_mhz": max(r[2] for r in use) if use else None,
+                    "samples": len(use), "window": label if inside else "whole run", "reasons": reasons}
+        out = summary(t_begin, t_end, "timed region")
+        if extra_window:
+            out["extra"] = summary(extra_window[0], extra_window[1], "sustained region")
+        return out
+
+
+TRAFFIC_PROFILE = os.path.join("profiles", "conv3x3_pair_tc_kernel_256_layer6_b48_full.txt")
+TRAFFIC_SOURCES = ("tc_conv_pair.cu", "tc_common.cuh")
+
+
+def kernel_source_digest():
+    """sha256 over the source files of the dominant kernel: the ncu summary records the digest it was
+    captured with, so that counters of an older kernel are not passed off as the current one's."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in TRAFFIC_SOURCES:
+        with open(os.path.join(ROOT, "paper_1810_09868_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def dominant_kernel_traffic():
+    """(bytes per batch-100 launch or None, note): dram__bytes_read.sum + dram__bytes_write.sum of the
+    dominant kernel, read from its ncu summary under profiles/ (a layer-6 launch captured at the batch the
+    file states) and scaled by the pixel count; None when the summary is missing, unreadable, or was
+    captured with other kernel sources than the ones now in the tree."""
+    import re
+    path = os.path.join(ROOT, TRAFFIC_PROFILE)
+    try:
+        text = open(path).read()
+    except OSError:
+        return None, f"{TRAFFIC_PROFILE} missing"
+    unit = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    total = 0.0
+    for key in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+        m = re.search(r"^" + re.escape(key) + r"\s+([0-9.]+)\s+(\w+)", text, re.M)
+        if not m or m.group(2) not in unit:
+            return None, f"{key} not found in {TRAFFIC_PROFILE}"
+        total += float(m.group(1)) * unit[m.group(2)]
+    b = re.search(r"^capture batch:\s*(\d+)", text, re.M)
+    d = re.search(r"^kernel source digest:\s*(\w+)", text, re.M)
+    if not b or not d:
+        return None, f"{TRAFFIC_PROFILE} states no capture batch / source digest"
+    if d.group(1) != kernel_source_digest():
+        return None, "the kernel's sources changed since the counters in " + TRAFFIC_PROFILE + " were taken"
+    batch = int(b.group(1))
+    return total * BATCH / batch, (f"ncu DRAM bytes of the layer-6 launch at batch {batch} from {TRAFFIC_PROFILE}, scaled by "
+                                   f"the pixel count to batch {BATCH} (traffic is proportional to pixels; the filter is 1.2 MB)")
 
 
 def slowest_rank_ms(ms, world, device="cpu"):
@@ -212,6 +266,67 @@ def time_conv_layers(pkg, net, torch, stream, reps=5):
     return out
 
 
+def time_conv_layers_backward(pkg, net, torch, stream, images, reps=5):
+    """Per-layer CUDA-event timing of the two backward kernels of every convolution at batch 100, on the
+    activations a training pass left in the workspace: the input gradient (with the ReLU mask of the layer
+    below where the pass applies it there) and the filter + bias gradient (with its finishing kernel).
+    The upstream gradient is synthetic: N(0, 1e-3) with half of the entries zero, like a ReLU-masked one.
+    Returns [(layer, dgrad_ms or None, wgrad_ms, flop)]."""
+    out = []
+    n_max = BATCH * 224 * 224 * 64
+    dz_all = torch.randn(n_max, dtype=torch.float32, device=net.device).mul_(1e-3)
+    dz_all.mul_((torch.rand(n_max, device=net.device) < 0.5).float())
+    dz_all = dz_all.to(torch.bfloat16)
+    dx_all = torch.empty(n_max, dtype=torch.bfloat16, device=net.device)
+    for l, (s, ci, co) in enumerate(CONV):
+        if l == 0:
+            x, pooled_input = images, False
+        else:
+            x = net.saved_tensor(BATCH, pkg.VGG19_MODE_BACKWARD, l - 1)
+            pooled_input = x.shape[1] != s
+            if pooled_input:
+                x = net.saved_tensor(BATCH, pkg.VGG19_MODE_BACKWARD, {1: 16, 3: 17, 7: 18, 11: 19, 15: 20}[l - 1])
+        dz = dz_all[:BATCH * s * s * co].view(BATCH, s, s, co)
+        dx = dx_all[:BATCH * s * s * ci].view(BATCH, s, s, ci)
+        dw = torch.empty(co * 9 * ci, dtype=torch.float32, device=net.device)
+        db = torch.empty(co, dtype=torch.float32, device=net.device)
+        mask = None if pooled_input else x  # after a pool the pass masks in the scatter step instead
+        calls = {"wgrad": lambda: pkg.vgg19_conv_layer_backward_ex(net.handle, l + 1, x, dz, BATCH, dw, db, None, None, stream)}
+        if l > 0:
+            calls["dgrad"] = lambda: pkg.vgg19_conv_layer_backward_ex(net.handle, l + 1, None, dz, BATCH, None, None, dx, mask, stream)
+        ms = {}
+        for name, fn in calls.items():
+            with torch.cuda.stream(stream):
+                for _ in range(2):
+                    fn()
+                evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+                for a, b in evs:
+                    a.record(stream)
+                    fn()
+                    b.record(stream)
+            stream.synchronize()
+            ms[name] = sum(a.elapsed_time(b) for a, b in evs) / reps
+        out.append((l + 1, ms.get("dgrad"), ms["wgrad"], 2.0 * BATCH * s * s * co * 9 * ci))
+    return out
+
+
+def forward_roofline_ms(pk):
+    """Kernel-by-kernel roofline of the forward pass at batch 100: sum over its steps of
+    max(flop / tensor peak, bytes / copy bandwidth), with each activation written once and read once
+    (pooled where the pool is fused), the image read once, weights read once."""
+    tf, bw = pk["bf16_tflops"] * 1e12, pk["hbm_gbs"] * 1e9
+    pool_after = {1, 3, 7, 11, 15}
+    total = 0.0
+    for l, (s, ci, co) in enumerate(CONV):
+        flop = 2.0 * BATCH * s * s * co * 9 * ci
+        out_px = BATCH * s * s // (4 if l in pool_after else 1)
+        byts = 2.0 * (BATCH * s * s * ci + out_px * co + 9 * ci * co)
+        total += max(flop / tf, byts / bw)
+    for i, o in ((25088, 4096), (4096, 4096), (4096, 1000)):
+        total += max(2.0 * BATCH * i * o / tf, 2.0 * (i * o + BATCH * (i + o)) / bw)
+    return total * 1e3
+
+
 def time_first_layer(pkg, net, torch, stream, x, reps=5):
     """conv1_1 (3 -> 64 channels), the pass's largest memory-bound kernel: CUDA-event time of the layer
     (channel-padding copy + convolution) and the algorithmic bytes it has to move: the 3-channel image in,
@@ -246,11 +361,17 @@ def run_native(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+        if rank == 0:
+            print(f"bench: {world} ranks, one GPU each, NCCL communicator of size {dist.get_world_size()}", file=sys.stderr)
 
     params = si.vgg19_params(H, W, seed=0, bf16_exact=True)
     images = si.images(BATCH, H, W, seed=1, bf16_exact=True)
     labels = si.labels(BATCH, seed=2)
-    net = pkg.Net(H, W, BATCH, pkg.VGG19_BF16, params=params, host_io=True, device=f"cuda:{local}")
+    # the training-step workspace (backward pass + gradient buffer) also covers the forward pass and its
+    # two host-staging slots
+    net = pkg.Net(H, W, BATCH, pkg.VGG19_BF16, params=params, mode=pkg.VGG19_MODE_TRAIN, device=f"cuda:{local}")
+    assert net.workspace.numel() >= (pkg.vgg19_workspace_bytes(net.handle, BATCH, pkg.VGG19_MODE_FORWARD)
+                                     + pkg.vgg19_io_bytes(net.handle, BATCH, pkg.VGG19_MODE_FORWARD))
     x = torch.from_numpy(images).to(dev).to(torch.bfloat16)
     y = torch.from_numpy(labels).to(dev)
     logits = torch.empty(BATCH, 1000, dtype=torch.float32, device=dev)
@@ -284,10 +405,25 @@ def run_native(args):
     fwd = lambda: pkg.vgg19_forward(net.handle, x, BATCH, logits, None, stream)
     bwd = lambda: pkg.vgg19_backward(net.handle, x, y, BATCH, grads, loss, None, stream)
 
+    side = torch.cuda.Stream(device=dev)
+    dense_off, _ = pkg.vgg19_param_info(net.handle, 32)
+    dense_ready = torch.cuda.Event()
+    dense_ready.record(stream)  # creates the handle the library records into
+
     def train():
-        # forward + backward, the gradient all-reduce over the ranks (N > 1), one SGD step
+        if world == 1:
+            # one GPU: forward, loss, backward and the update of every parameter copy as ONE recorded graph
+            pkg.vgg19_train_step(net.handle, x, y, BATCH, TRAIN_LR, loss, stream)
+            return
+        # several GPUs: the backward pass signals `dense_ready` once the dense layers' gradients (86 % of
+        # the buffer) are final; their all-reduce runs on a side stream beside the convolution layers'
+        # backward pass, the convolution gradients are exchanged when the pass ends, then one SGD step
         pkg.vgg19_backward(net.handle, x, y, BATCH, grads, loss, None, stream)
-        average_gradients(grads, world)
+        with torch.cuda.stream(side):
+            side.wait_event(dense_ready)
+            average_gradients(grads[dense_off:], world)
+        average_gradients(grads[:dense_off], world)
+        stream.wait_stream(side)
         pkg.vgg19_sgd_step(net.handle, grads, TRAIN_LR, stream)
 
     sampler = ClockSampler(local) if rank == 0 else None
@@ -300,10 +436,20 @@ def run_native(args):
     bwd_steps = max(3, args.steps // 2)
     bwd_ms = timed(bwd, bwd_steps, max(3, args.warmup))
     t_end = time.time()
-    clocks = sampler.stop(t_begin, t_end) if sampler else None
     net.sync_status(stream)
+    # sustained: back-to-back forward passes for about args.sustained_s seconds (the power cap settles the
+    # SM clock within the first second), timed as one region
+    sustained_steps = max(args.steps, int(args.sustained_s * 1e3 / (fwd_ms / args.steps)))
+    t_sus0 = time.time()
+    sustained_ms = timed(fwd, sustained_steps, 0)
+    t_sus1 = time.time()
+    net.sync_status(stream)
+    clocks = sampler.stop(t_begin, t_end, extra_window=(t_sus0, t_sus1)) if sampler else None
+    sustained_clocks = clocks.pop("extra", None) if clocks else None
 
     # training step last: it moves the weights (by a learning rate small enough to keep them sane)
+    if world > 1:
+        pkg.vgg19_set_dense_grads_event(net.handle, dense_ready)
     train_steps = max(3, args.steps // 2)
     train_ms = timed(train, train_steps, 3)
     net.sync_status(stream)
@@ -342,6 +488,7 @@ def run_native(args):
     stream.synchronize()
     layers = time_conv_layers(pkg, net, torch, stream)
     first_ms, first_bytes = time_first_layer(pkg, net, torch, stream, x)
+    bwd_layers = time_conv_layers_backward(pkg, net, torch, stream, x)
     # dominant kernel: conv3x3_pair_tc_kernel<256>, the 12 launches of layers 5..16 (60 % of the pass)
     dom = [t for t in layers if t[0] >= 5]
     conv_ms = sum(ms for _, ms, _, _ in dom)
@@ -352,9 +499,33 @@ def run_native(args):
     peak = pk["bf16_tflops"]
     per_layer = {f"conv{l}": {"ms": round(ms, 4), "tflops": round(f / (ms * 1e-3) / 1e12, 1), "path": path}
                  for l, ms, f, path in layers}
-    # dram__bytes_read+write of one launch of this kernel on layer 6 (56x56, 256->256), captured with
-    # ncu at batch 48 (113.5 MB) and scaled by the pixel count to the batch-100 launch timed here
-    traffic = 113.47e6 * BATCH / 48
+    traffic, traffic_note = dominant_kernel_traffic()
+    traffic_per_launch = None if traffic is None else traffic  # the layer-6 launch; one of the 12 timed here
+    # backward kernels per layer, and every tensor-bound kernel below 60 % of the bf16 peak
+    per_layer_bwd, below = {}, []
+    for l, dg, wg, f in bwd_layers:
+        row = {"wgrad_ms": round(wg, 4)}
+        if l == 1:
+            # filter gradient of the 3-channel layer: bound by reading dz (642 MB) and the image
+            byts = BATCH * H * W * (64 + 3) * 2
+            row["wgrad_gbs"] = round(byts / (wg * 1e-3) / 1e9, 1)
+            row["wgrad_frac_of_hbm"] = round(byts / (wg * 1e-3) / 1e9 / pk["hbm_gbs"], 3)
+        else:
+            row["wgrad_tflops"] = round(f / (wg * 1e-3) / 1e12, 1)
+            row["wgrad_frac"] = round(f / (wg * 1e-3) / 1e12 / peak, 3)
+            row["dgrad_ms"] = round(dg, 4)
+            row["dgrad_tflops"] = round(f / (dg * 1e-3) / 1e12, 1)
+            row["dgrad_frac"] = round(f / (dg * 1e-3) / 1e12 / peak, 3)
+            for kind in ("wgrad", "dgrad"):
+                if row[kind + "_frac"] < 0.6:
+                    below.append(f"conv{l} {kind} {row[kind + '_frac']:.2f}")
+        per_layer_bwd[f"conv{l}"] = row
+    for l, ms, f, path in layers:
+        if f / (ms * 1e-3) / 1e12 / peak < 0.6:
+            below.append(f"conv{l} fwd {f / (ms * 1e-3) / 1e12 / peak:.2f}")
+    bwd_conv_ms = sum((dg or 0.0) + wg for _, dg, wg, _ in bwd_layers)
+    bwd_conv_flop = sum(f * (2 if l > 1 else 0) for l, _, _, f in bwd_layers)
+    roof_ms = forward_roofline_ms(pk)
 
     n_fwd = pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_FORWARD)
     cpu_rate, cpu_dt = oracle_forward_rate(args.cpu_images)
@@ -375,23 +546,41 @@ def run_native(args):
         "gpu_launches": n_fwd * args.steps,
         "fwd_tflops_per_gpu": fwd_tflops,
         "fwd_frac_of_bf16_peak": fwd_tflops / peak,
+        "fwd_frac_of_roofline": roof_ms / (fwd_ms / args.steps),
+        "fwd_roofline_ms": roof_ms,
+        "sustained": {"value": aggregate_images_per_s(world, BATCH, sustained_steps, sustained_ms), "unit": "images/s",
+                      "steps": sustained_steps, "seconds": sustained_ms * 1e-3, "ms_per_step": sustained_ms / sustained_steps,
+                      "tflops_per_gpu": BATCH * sustained_steps / (sustained_ms * 1e-3) * FWD_FLOP_PER_IMAGE / 1e12,
+                      "frac_of_sustained_bf16_peak": BATCH * sustained_steps / (sustained_ms * 1e-3) * FWD_FLOP_PER_IMAGE / 1e12
+                                                     / pk["bf16_tflops_sustained"],
+                      "clocks": sustained_clocks},
         "fwd_bwd": {"value": world * BATCH * bwd_steps / (bwd_ms * 1e-3), "unit": "images/s", "steps": bwd_steps,
                     "ms_per_step": bwd_ms / bwd_steps,
                     "launches_per_step": pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_BACKWARD)},
         "train_step": {"value": world * BATCH * train_steps / (train_ms * 1e-3), "unit": "images/s", "steps": train_steps,
                        "ms_per_step": train_ms / train_steps, "lr": TRAIN_LR,
-                       "what": "forward + backward + " + ("NCCL all-reduce of the 143.7 M fp32 gradients + " if world > 1 else "")
-                               + "SGD update of the fp32 master, bf16 and filter copies"},
+                       "what": ("vgg19_train_step: forward + backward + SGD update of the fp32 master, bf16 and filter "
+                                "copies as one CUDA graph" if world == 1 else
+                                "vgg19_backward + NCCL all-reduce of the dense gradients (494 MB) on a side stream from "
+                                "the point the pass signals them final, of the convolution gradients (80 MB) at its "
+                                "end + vgg19_sgd_step"),
+                       "launches_per_step": pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_TRAIN) if world == 1 else None},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "traffic": traffic,
+                     "frac": achieved / peak, "traffic": traffic_per_launch,
                      "kernel": "conv3x3_pair_tc_kernel<256>: 3x3 convolution forward as a tcgen05 cta_group::2 implicit "
                                "GEMM on CTA pairs, layers 5..16 (12 launches per pass), algorithmic flops / summed launch time",
-                     "traffic_note": "DRAM bytes of the layer-6 launch (algorithmic: 160.6 MB in + 160.6 MB out "
-                                     "+ 1.2 MB filter at batch 100); the output is still in L2 when the launch ends",
+                     "traffic_note": traffic_note + "; algorithmic bytes of that launch: 160.6 MB in + 160.6 MB out + 1.2 MB "
+                                     "filter (the output is partly still in L2 when the launch ends)",
                      "peak_source": f"{pk['source']} burst bf16 GEMM (kernel timed alone per layer)",
                      "all_conv_layers_2_16": {"tflops": all_flop / (all_ms * 1e-3) / 1e12,
                                               "frac": all_flop / (all_ms * 1e-3) / 1e12 / peak},
-                     "per_layer": per_layer},
+                     "per_layer": per_layer,
+                     "per_layer_bwd": per_layer_bwd,
+                     "bwd_conv_kernels": {"ms": bwd_conv_ms, "tflops": bwd_conv_flop / (bwd_conv_ms * 1e-3) / 1e12,
+                                          "note": "input- and filter-gradient kernels of layers 1..16, each timed alone"},
+                     "below_60pct_of_bf16_peak": below,
+                     "hbm_bound_not_listed_above": "conv1 fwd and wgrad (3 input channels) and the dense layers at batch "
+                                                   "100 are bound by HBM, see hbm_bound and per_layer_bwd.conv1"},
         "hbm_bound": {"kernel": "conv1_1 forward (pad_to8_kernel + conv3x3_c8_tc_kernel): 3-channel image in, 64-channel activation out",
                       "ms": round(first_ms, 4), "achieved": first_bytes / (first_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
                       "unit": "GB/s", "frac": first_bytes / (first_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
@@ -401,6 +590,46 @@ def run_native(args):
         "context": {"paper_tpuv2_core_s_per_batch100": 0.23, "paper_xeon_4114_flux_cpu_s_per_batch100": 52.4},
     }
     print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def spawn_ranks(args):
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script, one per GPU, through
+    torch.distributed.run on 127.0.0.1 and hand their exit status back."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ)
+    if args.backend == "nccl":
+        # the communicator's size and transport show in NCCL's own start-up lines (stderr)
+        env.setdefault("NCCL_DEBUG", "INFO")
+        env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
+def run_dry(args):
+    """The multi-rank plumbing of run_native without a GPU: rendezvous, barrier, max over ranks of a
+    per-rank duration, gradient averaging, whole-job aggregation.  Each rank pretends its pass took
+    (10 + rank) ms per step and that its gradient is the constant rank + 1."""
+    import torch
+    import torch.distributed as dist
+    if args.backend != "gloo":
+        raise SystemExit("--dry runs on CPU ranks: use --backend gloo")
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms = slowest_rank_ms((10.0 + rank) * args.steps, world)
+    g = average_gradients(torch.full((8,), float(rank + 1)), world)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "dry": True, "n_gpus": world, "steps": args.steps,
+                          "value": aggregate_images_per_s(world, BATCH, args.steps, ms), "unit": "images/s",
+                          "ms_per_step": ms / args.steps, "mean_gradient": float(g[0]), "scaling": "weak"}))
     if world > 1:
         dist.destroy_process_group()
 
@@ -441,6 +670,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--cpu-images", type=int, default=24, help="images the CPU checker is timed on")
+    ap.add_argument("--sustained-s", type=float, default=2.5, help="seconds of back-to-back passes for the sustained figure")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"])
+    ap.add_argument("--dry", action="store_true", help="multi-rank plumbing only, on CPU ranks (needs --backend gloo)")
     ap.add_argument("--profile-layer", type=int, default=0, help="run only this conv layer (1..16) a few times and exit")
     ap.add_argument("--profile-batch", type=int, default=16)
     ap.add_argument("--profile-kind", default="fwd", choices=["fwd", "bwd"])
@@ -451,6 +683,10 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
+    elif args.dry:
+        run_dry(args)
     else:
         run_native(args)
 

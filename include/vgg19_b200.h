@@ -57,7 +57,11 @@ enum {
   VGG19_FLAG_NO_CTA_PAIRS = 4     /* one CTA per tile everywhere: no two-CTA (cta_group::2) kernels */
 };
 
-typedef enum { VGG19_MODE_FORWARD = 0, VGG19_MODE_BACKWARD = 1 } vgg19_mode;
+typedef enum {
+  VGG19_MODE_FORWARD = 0,  /* vgg19_forward */
+  VGG19_MODE_BACKWARD = 1, /* vgg19_backward */
+  VGG19_MODE_TRAIN = 2     /* vgg19_train_step(s): the backward workspace plus a gradient buffer */
+} vgg19_mode;
 
 typedef struct {
   int32_t height;    /* input height, multiple of 32 */
@@ -127,6 +131,42 @@ int vgg19_backward(vgg19_t *net, const void *images, const int32_t *labels, int3
  * same stream see the new parameters.  Graphs recorded earlier stay valid. */
 int vgg19_sgd_step(vgg19_t *net, const float *grads, float lr, void *stream);
 
+/* The training step as ONE device program: forward + loss + backward on a
+ * batch and the gradient-descent update of every parameter (fp32 master, bf16
+ * copy, the rotated / tap-major / padded filter copies), recorded as a single
+ * CUDA graph - the paper's claim for its own system is that the forward pass,
+ * the backward pass and the training loop fuse into one executable
+ * (introduction and conclusion).  The gradient never leaves the workspace,
+ * which must hold vgg19_workspace_bytes(net, batch, VGG19_MODE_TRAIN).
+ * images / labels: device, as for vgg19_backward.  loss: device fp32 scalar
+ * (the loss BEFORE the update) or NULL.  lr may change from call to call
+ * without a new recording (the update kernels read it from device memory).
+ * For one GPU only: with several, the gradients must be averaged between the
+ * two halves - use vgg19_backward, the exchange, vgg19_sgd_step. */
+int vgg19_train_step(vgg19_t *net, const void *images, const int32_t *labels, int32_t batch, float lr,
+                     float *loss, void *stream);
+
+/* `steps` (1..64) training steps on `steps` resident batches as one graph:
+ * images [steps][batch][H][W][3], labels [steps][batch], losses (or NULL)
+ * device fp32 [steps]; step k trains on batch k with the parameters step k-1
+ * left.  The counterpart of compiling the training LOOP, not just its body. */
+int vgg19_train_steps(vgg19_t *net, const void *images, const int32_t *labels, int32_t batch, int32_t steps,
+                      float lr, float *losses, void *stream);
+
+/* Overlap point for data-parallel training.  In the flat gradient buffer the
+ * three dense layers come last (from the offset vgg19_param_info(net, 32)
+ * reports; 123.6 M of the 143.7 M elements at 224x224) and the backward pass
+ * finishes them first, before any convolution layer's gradient.  With an
+ * event set here (a cudaEvent_t the caller owns; NULL clears it), every later
+ * vgg19_backward records it on its stream at that point - inside the recorded
+ * graph too - so that a caller can start the all-reduce of the dense
+ * gradients on another stream (cudaStreamWaitEvent) while the convolution
+ * layers' backward pass, most of the pass's time, still runs, and exchange the
+ * convolution gradients when the pass ends.  The paper lists distributed
+ * primitives as future work (section 8); the exchange itself stays with the
+ * caller.  Setting or clearing the event discards recorded graphs. */
+int vgg19_set_dense_grads_event(vgg19_t *net, void *cuda_event);
+
 /* HOST-buffer convenience wrappers: copy images (and labels) to the device,
  * run the pass, copy the results back and wait for the stream.  The bound
  * workspace must hold vgg19_workspace_bytes(net, batch, mode) +
@@ -147,7 +187,11 @@ int vgg19_backward_host(vgg19_t *net, const void *host_images, const int32_t *ho
  * the executable of section 7.2.  host_images must stay untouched, and the
  * results are not in host_logits / host_probs, until `stream` has been waited
  * for (vgg19_sync_status); with more than two calls in flight the library orders
- * the reuse of a slot itself.  stream must not be the legacy default stream.
+ * the reuse of a slot itself; a call whose batch differs from the previous
+ * call's, or that follows a pass made through another entry point, uploads
+ * only after the work already enqueued on `stream` (the staging slots move
+ * with the batch).  Keep all calls in flight on one handle on one stream.
+ * stream must not be the legacy default stream.
  * Needs the same workspace as vgg19_forward_host (vgg19_io_bytes counts both slots). */
 int vgg19_forward_host_async(vgg19_t *net, const void *host_images, int32_t batch, float *host_logits,
                              float *host_probs, void *stream);
@@ -166,6 +210,16 @@ int vgg19_conv_layer_forward(vgg19_t *net, int32_t layer, const void *x, int32_t
  * NULL) dx in the config's dtype [batch][h][w][Cin] (section 7.3). */
 int vgg19_conv_layer_backward(vgg19_t *net, int32_t layer, const void *x, const void *dz,
                               int32_t batch, float *dw, float *db, void *dx, void *stream);
+
+/* The same with the two halves separable and the ReLU of the layer below
+ * folded in, as the whole pass runs them (section 7.3: the `select`s that
+ * follow each input-gradient convolution).  dw and db may both be NULL (input
+ * gradient only; x is then unused and may be NULL), or dx may be NULL (filter
+ * and bias gradient only).  relu_mask (or NULL): [batch][h][w][Cin] in the
+ * config's dtype, the stored output of the layer below; dx is set to zero
+ * wherever relu_mask is not positive. */
+int vgg19_conv_layer_backward_ex(vgg19_t *net, int32_t layer, const void *x, const void *dz, int32_t batch,
+                                 float *dw, float *db, void *dx, const void *relu_mask, void *stream);
 
 /* Where a pass at `batch` in `mode` leaves the activations it stores, as a
  * byte offset into the bound workspace, so that a caller can inspect the
@@ -191,7 +245,8 @@ int vgg19_saved_tensor(const vgg19_t *net, int32_t batch, int32_t mode, int32_t 
  * provide a workspace, because both need cudaMalloc.  This function needs
  * neither: it takes no handle, and the split-K scratch its kernel uses is a
  * fixed array of VGG19_STATIC_SCRATCH_BYTES compiled into the library (every
- * GPU that loads the library carries that array until the process exits).  It
+ * GPU on which the library's code is loaded carries that array until the
+ * process exits; see below for when that happens).  It
  * calls no cudaMalloc / cudaFree and no allocating library routine.
  *
  *   x  : device, [batch][height][width][cin]   layer input
@@ -207,6 +262,14 @@ int vgg19_saved_tensor(const vgg19_t *net, int32_t batch, int32_t mode, int32_t 
  *
  * The first call on each device looks up the array's device address (that
  * device must be current); make that first call outside any stream capture.
+ * With CUDA's default lazy module loading that first call is also when the
+ * driver places the array, and the kernels' code, on the device: a process
+ * that is about to hand the GPU's memory to someone else should make one call
+ * per device at start-up, before the memory is claimed (or run with
+ * CUDA_MODULE_LOADING=EAGER, which places everything when the library loads);
+ * from the second call on, free device memory is unchanged by a call.  If the
+ * lookup fails (for instance because the device is already full) the call and
+ * every later one on that device return VGG19_ERR_CUDA.
  * All calls share the one array and it keeps whatever the last call left in
  * it; the kernels never rely on its previous contents.  Two calls that overlap
  * on the GPU (different streams) race on it: keep calls on one stream, or
@@ -216,8 +279,22 @@ int vgg19_conv_wgrad_static(const void *x, const void *dz, int32_t batch, int32_
                             int32_t cin, int32_t cout, int32_t dtype, float *dw, float *db,
                             size_t *needed_bytes, void *stream);
 
-/* Wait for the stream and report any device-side error recorded so far. */
+/* Wait for the stream and report any device-side error recorded so far:
+ * VGG19_ERR_DEVICE_TIMEOUT when a bounded wait inside a kernel ran out,
+ * VGG19_ERR_ARG when a label outside [0,1000) reached the loss (the label is
+ * never used as an index; that pass's loss is NaN).  The record is cleared,
+ * and the handle stays usable. */
 int vgg19_sync_status(vgg19_t *net, void *stream);
+
+/* Diagnostic for the error path above.  Every wait inside the kernels (on a
+ * copy, on the tensor cores, on a free buffer) is bounded; when one runs out
+ * the kernel records a code, lets what it has in flight finish and returns.
+ * This call enqueues one tiny kernel whose wait is certain to run out - a
+ * barrier in shared memory on which nothing arrives, limit about a millisecond,
+ * no copy engine or tensor memory involved - so that a caller (or a test) can
+ * see the whole chain: the next vgg19_sync_status returns
+ * VGG19_ERR_DEVICE_TIMEOUT, and passes enqueued afterwards run normally. */
+int vgg19_selftest_wait_timeout(vgg19_t *net, void *stream);
 
 /* Number of kernel launches (graph nodes) one forward / backward call makes. */
 int vgg19_launch_count(const vgg19_t *net, int32_t mode, int32_t *n_kernels);

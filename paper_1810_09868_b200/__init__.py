@@ -59,6 +59,11 @@ class Net:
         """parameters <- parameters - lr * grads, on the device, with every derived filter copy rebuilt."""
         binding.vgg19_sgd_step(self.handle, grads, lr, stream or self._torch.cuda.current_stream(self.device))
 
+    def train_step(self, images, labels, lr, loss=None, stream=None):
+        """Forward + backward + update as one recorded device program (workspace of VGG19_MODE_TRAIN)."""
+        stream = stream or self._torch.cuda.current_stream(self.device)
+        binding.vgg19_train_step(self.handle, images, labels, images.shape[0], lr, loss, stream)
+
     def saved_tensor(self, batch, mode, index):
         """View of a stored activation inside the workspace (no copy)."""
         off, dims = binding.vgg19_saved_tensor(self.handle, batch, mode, index)

@@ -16,13 +16,14 @@ VGG19_ERR_ARG, VGG19_ERR_SHAPE, VGG19_ERR_WORKSPACE = -1, -2, -3
 VGG19_ERR_CUDA, VGG19_ERR_DEVICE_TIMEOUT, VGG19_ERR_UNSUPPORTED_ARCH = -4, -5, -6
 VGG19_FP32, VGG19_BF16 = 0, 1
 VGG19_FLAG_NO_GRAPH, VGG19_FLAG_NO_TENSOR_CORES, VGG19_FLAG_NO_CTA_PAIRS = 1, 2, 4
-VGG19_MODE_FORWARD, VGG19_MODE_BACKWARD = 0, 1
+VGG19_MODE_FORWARD, VGG19_MODE_BACKWARD, VGG19_MODE_TRAIN = 0, 1, 2
 
 EXPORTS = (
     "vgg19_create", "vgg19_create_from_params", "vgg19_destroy", "vgg19_param_count", "vgg19_param_info",
     "vgg19_get_params", "vgg19_set_params", "vgg19_workspace_bytes", "vgg19_bind_workspace",
-    "vgg19_forward", "vgg19_backward", "vgg19_sgd_step", "vgg19_io_bytes", "vgg19_forward_host", "vgg19_forward_host_async", "vgg19_backward_host",
-    "vgg19_conv_layer_forward", "vgg19_conv_layer_backward", "vgg19_saved_tensor", "vgg19_conv_wgrad_static", "vgg19_sync_status", "vgg19_launch_count",
+    "vgg19_forward", "vgg19_backward", "vgg19_sgd_step", "vgg19_train_step", "vgg19_train_steps",
+    "vgg19_set_dense_grads_event", "vgg19_io_bytes", "vgg19_forward_host", "vgg19_forward_host_async", "vgg19_backward_host",
+    "vgg19_conv_layer_forward", "vgg19_conv_layer_backward", "vgg19_conv_layer_backward_ex", "vgg19_saved_tensor", "vgg19_conv_wgrad_static", "vgg19_sync_status", "vgg19_selftest_wait_timeout", "vgg19_launch_count",
     "vgg19_describe", "vgg19_last_error",
 )
 
@@ -70,15 +71,20 @@ def load():
         "vgg19_forward": ([vp, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_backward": ([vp, vp, vp, i32, vp, vp, vp, vp], ctypes.c_int),
         "vgg19_sgd_step": ([vp, vp, ctypes.c_float, vp], ctypes.c_int),
+        "vgg19_train_step": ([vp, vp, vp, i32, ctypes.c_float, vp, vp], ctypes.c_int),
+        "vgg19_train_steps": ([vp, vp, vp, i32, i32, ctypes.c_float, vp, vp], ctypes.c_int),
+        "vgg19_set_dense_grads_event": ([vp, vp], ctypes.c_int),
         "vgg19_io_bytes": ([vp, i32, i32], sz),
         "vgg19_forward_host": ([vp, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_forward_host_async": ([vp, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_backward_host": ([vp, vp, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_forward": ([vp, i32, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_backward": ([vp, i32, vp, vp, i32, vp, vp, vp, vp], ctypes.c_int),
+        "vgg19_conv_layer_backward_ex": ([vp, i32, vp, vp, i32, vp, vp, vp, vp, vp], ctypes.c_int),
         "vgg19_saved_tensor": ([vp, i32, i32, i32, ctypes.POINTER(sz), ctypes.POINTER(ctypes.c_int64)], ctypes.c_int),
         "vgg19_conv_wgrad_static": ([vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, ctypes.POINTER(sz), vp], ctypes.c_int),
         "vgg19_sync_status": ([vp, vp], ctypes.c_int),
+        "vgg19_selftest_wait_timeout": ([vp, vp], ctypes.c_int),
         "vgg19_launch_count": ([vp, i32, ctypes.POINTER(i32)], ctypes.c_int),
         "vgg19_describe": ([vp, ctypes.c_char_p, sz], ctypes.c_int),
         "vgg19_last_error": ([vp], ctypes.c_char_p),
@@ -159,6 +165,22 @@ def vgg19_sgd_step(net, grads, lr, stream=None):
     return _check(net, load().vgg19_sgd_step(net, _ptr(grads), float(lr), _stream(stream)))
 
 
+def vgg19_train_step(net, images, labels, batch, lr, loss=None, stream=None):
+    return _check(net, load().vgg19_train_step(net, _ptr(images), _ptr(labels), batch, float(lr), _ptr(loss), _stream(stream)))
+
+
+def vgg19_train_steps(net, images, labels, batch, steps, lr, losses=None, stream=None):
+    return _check(net, load().vgg19_train_steps(net, _ptr(images), _ptr(labels), batch, steps, float(lr), _ptr(losses),
+                                                 _stream(stream)))
+
+
+def vgg19_set_dense_grads_event(net, event):
+    """event: a torch.cuda.Event that has been recorded at least once (so that its handle exists), a raw
+    cudaEvent_t as an integer, or None."""
+    h = None if event is None else (event if isinstance(event, int) else event.cuda_event)
+    return _check(net, load().vgg19_set_dense_grads_event(net, h))
+
+
 def vgg19_workspace_bytes(net, batch, mode):
     return load().vgg19_workspace_bytes(net, batch, mode)
 
@@ -205,6 +227,11 @@ def vgg19_conv_layer_backward(net, layer, x, dz, batch, dw, db, dx=None, stream=
                                                          _ptr(dx), _stream(stream)))
 
 
+def vgg19_conv_layer_backward_ex(net, layer, x, dz, batch, dw=None, db=None, dx=None, relu_mask=None, stream=None):
+    return _check(net, load().vgg19_conv_layer_backward_ex(net, layer, _ptr(x), _ptr(dz), batch, _ptr(dw), _ptr(db),
+                                                            _ptr(dx), _ptr(relu_mask), _stream(stream)))
+
+
 def vgg19_saved_tensor(net, batch, mode, index):
     off = ctypes.c_size_t()
     dims = (ctypes.c_int64 * 4)()
@@ -225,6 +252,10 @@ def vgg19_conv_wgrad_static(x, dz, batch, height, width, cin, cout, dtype, dw, d
 
 def vgg19_sync_status(net, stream=None):
     return _check(net, load().vgg19_sync_status(net, _stream(stream)))
+
+
+def vgg19_selftest_wait_timeout(net, stream=None):
+    return _check(net, load().vgg19_selftest_wait_timeout(net, _stream(stream)))
 
 
 def vgg19_launch_count(net, mode):

@@ -26,6 +26,8 @@ enum DeviceError : int {
   kDevTimeoutStageFree = 2, // producer waited too long for a free stage
   kDevTimeoutAccum = 3,     // epilogue waited too long for the accumulator
   kDevTimeoutTmemFree = 4,  // MMA issuer waited too long for a drained accumulator
+  kDevTimeoutTest = 5,      // the self-test kernel's wait on a barrier nobody arrives on
+  kDevBadLabel = 64,        // a label outside [0, classes): not a timeout, reported as a bad argument
 };
 
 // ---- CUDA-core kernels (simt_kernels.cu) ---------------------------------
@@ -84,9 +86,12 @@ cudaError_t simt_dense_dw(const T* dY, const T* X, float* dW, float* db, int M, 
 
 // Row-wise softmax of fp32 logits (probs may be null), and for the backward
 // pass the per-row loss and dlogits = (p - onehot(label)) / rows, stored as T.
+// A label outside [0, classes) is never dereferenced: the row's loss becomes NaN and kDevBadLabel is
+// recorded in dev_error (when given).
 template <typename T>
 cudaError_t softmax_xent(const float* logits, const int32_t* labels, float* probs, T* dlogits,
-                         float* row_loss, float* loss, int rows, int classes, cudaStream_t st);
+                         float* row_loss, float* loss, int rows, int classes, cudaStream_t st,
+                         int* dev_error = nullptr);
 
 // fp32 -> T copy (weights), and the dgrad filter: wt_t[c][r][s][k] = w[k][2-r][2-s][c].
 template <typename T>
@@ -109,9 +114,12 @@ cudaError_t refresh_filter_copies(const float* params, bf16* dgrad_w, bf16* tap_
                                   const FilterCopyTable& tab, cudaStream_t st);
 
 // params -= lr * grads (fp32 master, in place); params_t (the storage-type copy, or null when T is
-// float and the master is the copy) receives the rounded result in the same pass.
+// float and the master is the copy) receives the rounded result in the same pass.  With lr_dev the
+// rate is read from that device scalar instead of `lr` (a recorded graph keeps working when it changes).
 template <typename T>
-cudaError_t sgd_update(float* params, const float* grads, T* params_t, float lr, size_t n, cudaStream_t st);
+cudaError_t sgd_update(float* params, const float* grads, T* params_t, float lr, size_t n, cudaStream_t st,
+                       const float* lr_dev = nullptr);
+cudaError_t set_scalar(float* dst, float v, cudaStream_t st);
 template <typename T>
 cudaError_t make_dgrad_filter(const float* w, T* wt_t, int Cin, int Cout, cudaStream_t st);
 

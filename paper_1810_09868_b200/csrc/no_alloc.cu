@@ -3,6 +3,8 @@
 // fixed array inside this library instead of a caller-provided workspace.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "../../include/vgg19_b200.h"
 #include "common.cuh"
 
@@ -14,7 +16,8 @@ namespace {
 static __device__ __align__(256) float g_static_scratch[VGG19_STATIC_SCRATCH_BYTES / sizeof(float)];
 
 constexpr int kMaxDevices = 64;
-float* g_scratch_ptr[kMaxDevices];  // zero-initialised: not looked up yet
+float* g_scratch_ptr[kMaxDevices];     // written once per device, under g_lookup_once
+std::once_flag g_lookup_once[kMaxDevices];
 
 }  // namespace
 
@@ -31,13 +34,14 @@ extern "C" int vgg19_conv_wgrad_static(const void* x, const void* dz, int32_t ba
   if (need > VGG19_STATIC_SCRATCH_BYTES) return VGG19_ERR_WORKSPACE;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VGG19_ERR_CUDA;
-  if (!g_scratch_ptr[dev]) {
-    // first call on this device: resolve the array's device address (the device is current)
+  // First call on this device: resolve the array's device address (the device is current).  One host
+  // thread does the lookup, any others calling at the same moment wait for it.  With lazy module
+  // loading (the CUDA default) this lookup is also what makes the driver place the array on the device.
+  std::call_once(g_lookup_once[dev], [dev] {
     float* p = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_scratch) != cudaSuccess || !p)
-      return VGG19_ERR_CUDA;
-    g_scratch_ptr[dev] = p;
-  }
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_scratch) == cudaSuccess) g_scratch_ptr[dev] = p;
+  });
+  if (!g_scratch_ptr[dev]) return VGG19_ERR_CUDA;
   // Nothing in the scratch has to start at zero: every partial sum the second
   // pass reads is written by the first pass of the same call.
   cudaStream_t st = static_cast<cudaStream_t>(stream);

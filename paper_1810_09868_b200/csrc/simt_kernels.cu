@@ -489,7 +489,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 template <typename T>
 __global__ void softmax_xent_kernel(const float* logits, const int32_t* labels, float* probs,
-                                    T* dlogits, float* row_loss, int rows, int classes) {
+                                    T* dlogits, float* row_loss, int rows, int classes, int* dev_error) {
   int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
   int lane = threadIdx.x % 32;
   if (row >= rows) return;
@@ -502,13 +502,19 @@ __global__ void softmax_xent_kernel(const float* logits, const int32_t* labels, 
   s = warp_sum(s);
   float inv = 1.f / s;
   int label = labels ? labels[row] : -1;
+  const bool bad_label = labels && (unsigned)label >= (unsigned)classes;
+  if (bad_label) {  // never index with it: no one-hot term, a NaN loss, and a code for the host
+    label = -1;
+    if (lane == 0 && dev_error) atomicCAS(dev_error, 0, (int)kDevBadLabel);
+  }
   float scale = 1.f / (float)rows;
   for (int j = lane; j < classes; j += 32) {
     float p = expf(l[j] - m) * inv;
     if (probs) probs[(long)row * classes + j] = p;
     if (dlogits) dlogits[(long)row * classes + j] = from_f32<T>((p - (j == label ? 1.f : 0.f)) * scale);
   }
-  if (row_loss && label >= 0 && lane == 0) row_loss[row] = (m + logf(s)) - l[label];
+  if (row_loss && lane == 0 && (label >= 0 || bad_label))
+    row_loss[row] = bad_label ? __int_as_float(0x7fc00000) : (m + logf(s)) - l[label];
 }
 
 __global__ void mean_loss_kernel(const float* row_loss, float* loss, int rows) {
@@ -520,10 +526,10 @@ __global__ void mean_loss_kernel(const float* row_loss, float* loss, int rows) {
 
 template <typename T>
 cudaError_t softmax_xent(const float* logits, const int32_t* labels, float* probs, T* dlogits,
-                         float* row_loss, float* loss, int rows, int classes, cudaStream_t st) {
+                         float* row_loss, float* loss, int rows, int classes, cudaStream_t st, int* dev_error) {
   const int warps = 4;
   softmax_xent_kernel<T><<<(rows + warps - 1) / warps, warps * 32, 0, st>>>(
-      logits, labels, probs, dlogits, row_loss, rows, classes);
+      logits, labels, probs, dlogits, row_loss, rows, classes, dev_error);
   if (loss && row_loss) mean_loss_kernel<<<1, 32, 0, st>>>(row_loss, loss, rows);
   return cudaGetLastError();
 }
@@ -546,7 +552,8 @@ cudaError_t convert_f32(const float* src, T* dst, size_t n, cudaStream_t st) {
 // (four elements per thread where the count allows; the tail one at a time).
 template <typename T>
 __global__ void sgd_update_kernel(float* __restrict__ p, const float* __restrict__ g, T* __restrict__ pt, float lr,
-                                  size_t n) {
+                                  const float* __restrict__ lr_dev, size_t n) {
+  if (lr_dev) lr = *lr_dev;  // the rate of a recorded training step lives in device memory
   const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i + 3 < n) {
     float4 w = *reinterpret_cast<float4*>(p + i);
@@ -571,8 +578,15 @@ __global__ void sgd_update_kernel(float* __restrict__ p, const float* __restrict
 }
 
 template <typename T>
-cudaError_t sgd_update(float* params, const float* grads, T* params_t, float lr, size_t n, cudaStream_t st) {
-  sgd_update_kernel<T><<<(unsigned)((n / 4 + 256) / 256), 256, 0, st>>>(params, grads, params_t, lr, n);
+cudaError_t sgd_update(float* params, const float* grads, T* params_t, float lr, size_t n, cudaStream_t st,
+                       const float* lr_dev) {
+  sgd_update_kernel<T><<<(unsigned)((n / 4 + 256) / 256), 256, 0, st>>>(params, grads, params_t, lr, lr_dev, n);
+  return cudaGetLastError();
+}
+
+__global__ void set_scalar_kernel(float* dst, float v) { *dst = v; }
+cudaError_t set_scalar(float* dst, float v, cudaStream_t st) {
+  set_scalar_kernel<<<1, 1, 0, st>>>(dst, v);
   return cudaGetLastError();
 }
 
@@ -658,9 +672,10 @@ cudaError_t refresh_filter_copies(const float* params, bf16* dgrad_w, bf16* tap_
   template cudaError_t simt_bias_grad<T>(const T*, float*, float*, long, int, cudaStream_t);           \
   template cudaError_t simt_dense_db<T>(const T*, float*, int, int, cudaStream_t);                    \
   template cudaError_t softmax_xent<T>(const float*, const int32_t*, float*, T*, float*, float*,     \
-                                       int, int, cudaStream_t);                                      \
+                                       int, int, cudaStream_t, int*);                                \
   template cudaError_t convert_f32<T>(const float*, T*, size_t, cudaStream_t);                       \
-  template cudaError_t sgd_update<T>(float*, const float*, T*, float, size_t, cudaStream_t);         \
+  template cudaError_t sgd_update<T>(float*, const float*, T*, float, size_t, cudaStream_t,          \
+                                     const float*);                                                  \
   template cudaError_t make_dgrad_filter<T>(const float*, T*, int, int, cudaStream_t);
 
 INSTANTIATE(float)

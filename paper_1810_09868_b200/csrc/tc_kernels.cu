@@ -472,4 +472,26 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
   }
 }
 
+namespace {
+__global__ void wait_selftest_kernel(int* dev_error, long long limit_cycles) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    tc::mbar_init(tc::smem_u32(&bar), 1);
+    tc::mbar_fence_init();
+  }
+  __syncthreads();
+  // phase 0 of a freshly initialised barrier completes only when its one expected arrival comes; none does
+  if (threadIdx.x == 0)
+    tc::mbar_wait(tc::smem_u32(&bar), 0, &abort_flag, dev_error, kDevTimeoutTest, limit_cycles);
+  __syncthreads();
+}
+}  // namespace
+
+cudaError_t tc_wait_selftest(int* dev_error, long long limit_cycles, cudaStream_t st) {
+  wait_selftest_kernel<<<1, 32, 0, st>>>(dev_error, limit_cycles);
+  return cudaGetLastError();
+}
+
 }  // namespace vgg

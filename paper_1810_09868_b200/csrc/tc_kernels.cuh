@@ -91,4 +91,10 @@ size_t tc_first_wgrad_scratch_elems(ConvShape s);
 cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* db, float* partial, ConvShape s, int* dev_error,
                            cudaStream_t st);
 
+// Self-test of the bounded-wait plumbing: one CTA of 32 threads initialises an mbarrier in shared
+// memory on which nothing ever arrives and waits for it with a limit of `limit_cycles` SM cycles; the
+// wait runs out, kDevTimeoutTest lands in dev_error and the kernel returns normally.  No TMA, no
+// tensor memory, nothing in flight when it gives up.
+cudaError_t tc_wait_selftest(int* dev_error, long long limit_cycles, cudaStream_t st);
+
 }  // namespace vgg

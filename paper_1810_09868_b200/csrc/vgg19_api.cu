@@ -69,7 +69,8 @@ struct vgg19 {
   void *ws = nullptr;
   size_t ws_bytes = 0;
   std::vector<GraphEntry> graphs;
-  int launches[2] = {0, 0};
+  int launches[3] = {0, 0, 0};
+  cudaEvent_t dense_grads_event = nullptr;  // caller's; recorded once the dense layers' gradients are final
   std::string err;
   bool use_tc = false;
   bool use_pair = false;  // two-CTA kernels where a layer's shape takes them
@@ -79,6 +80,9 @@ struct vgg19 {
   cudaEvent_t ev_uploaded[2] = {nullptr, nullptr}, ev_consumed[2] = {nullptr, nullptr};
   bool slot_used[2] = {false, false};
   unsigned next_slot = 0;
+  int async_batch = 0;        // batch of the last vgg19_forward_host_async call (0: none yet)
+  bool other_pass = false;    // a pass went through another entry point since that call
+  cudaEvent_t ev_order = nullptr;
 };
 
 namespace {
@@ -114,6 +118,7 @@ struct Plan {
   size_t x8;                // image copied to 8 channels (bf16 tensor-core path of layer 1)
   bool valid = true;
   size_t row_loss, loss;
+  size_t grads, lr;         // training step: the gradient buffer and the learning rate (a device scalar)
   size_t total;
   size_t io_images, io_labels, io_logits, io_probs, io_grads, io_loss, io_total;
 };
@@ -166,6 +171,8 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
   if (conv_fwd_partial > dense_partial) dense_partial = conv_fwd_partial;
   if (mode == VGG19_MODE_FORWARD) p.partial = take(dense_partial * 4);
   if (dense_partial > max_partial) max_partial = dense_partial;
+  const bool train = mode == VGG19_MODE_TRAIN;
+  if (train) mode = VGG19_MODE_BACKWARD;
   if (mode == VGG19_MODE_BACKWARD) {
     p.dl = take((size_t)B * kClasses * n->elt);
     p.dz2 = take((size_t)B * 4096 * n->elt);
@@ -177,6 +184,10 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
     p.partial = take(max_partial * 4);
     p.row_loss = take((size_t)B * 4);
     p.loss = take(256);
+  }
+  if (train) {
+    p.grads = take(n->n_params * 4);
+    p.lr = take(256);
   }
   p.total = off;
   size_t io = off;
@@ -200,6 +211,7 @@ struct PassArgs {
   const int32_t *labels;
   float *logits, *probs, *grads, *loss;
   int batch;
+  int steps = 1;  // training mode: batches taken in turn by one recorded graph
 };
 
 template <typename T>
@@ -261,7 +273,9 @@ struct Pass {
                      const T *mask) {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
-    if (first_tc_ok(l, s)) {
+    if (!dW) {
+      // input gradient only (per-layer entry point)
+    } else if (first_tc_ok(l, s)) {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       ok(tc_first_wgrad((const bf16 *)buf(p.x8), (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st), 2);
     } else if (n->use_tc && tc_wgrad_patch_supported(s)) {
@@ -343,12 +357,21 @@ struct Pass {
     float *g = a.grads;
     const FcLayer *f = n->fc;
     ok(softmax_xent<T>(logits, a.labels, a.probs, buf(p.dl), fbuf(p.row_loss), loss, B, kClasses,
-                       st), 2);
+                       st, n->dev_error), 2);
     const T *flat = buf(p.pooled[4]);
     // dense 3, 2, 1: filter gradient, then input gradient masked by the ReLU below
     dense_backward(f[2], buf(p.a2), buf(p.dl), B, g + f[2].w_off, g + f[2].b_off, buf(p.dz2), buf(p.a2));
     dense_backward(f[1], buf(p.a1), buf(p.dz2), B, g + f[1].w_off, g + f[1].b_off, buf(p.dz1), buf(p.a1));
     dense_backward(f[0], flat, buf(p.dz1), B, g + f[0].w_off, g + f[0].b_off, buf(p.dflat), nullptr);
+    if (n->dense_grads_event && err == cudaSuccess) {
+      // the dense layers' gradients (the tail of the flat buffer, 86 % of it at 224x224) are final here:
+      // a caller's exchange of them can run beside the convolution layers' backward pass.  Inside a
+      // capture the record becomes a node of the graph that signals the caller's (external) event.
+      cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+      cudaStreamIsCapturing(st, &cs);
+      err = cudaEventRecordWithFlags(n->dense_grads_event, st,
+                                     cs == cudaStreamCaptureStatusActive ? cudaEventRecordExternal : cudaEventRecordDefault);
+    }
     // convolutions 16..1.  `dz` is the gradient at layer l's pre-activation.
     T *dz = buf(p.dza), *other = buf(p.dzb);
     {
@@ -387,15 +410,35 @@ int check_batch(vgg19 *n, int batch, int mode, size_t extra) {
   return VGG19_OK;
 }
 
+int refresh_filter_copies(vgg19 *n, cudaStream_t st);
+
 template <typename T>
 int enqueue(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st, int *launches) {
   Pass<T> pass{n, make_plan(n, a.batch, mode), st};
   if (mode == VGG19_MODE_FORWARD) {
     pass.keep_activations = false;
     pass.forward(a);
-  } else {
+  } else if (mode == VGG19_MODE_BACKWARD) {
     pass.forward_tail_split = false;
     pass.backward(a);
+  } else {
+    // training steps: a.steps times [forward + backward on the next batch, parameter update], the
+    // gradient staying in the workspace; images / labels / loss advance by one batch per step
+    pass.forward_tail_split = false;
+    const size_t img_stride = (size_t)a.batch * n->cfg.height * n->cfg.width * 3 * n->elt;
+    for (int k = 0; k < a.steps && pass.err == cudaSuccess; ++k) {
+      PassArgs b = a;
+      b.images = static_cast<const char *>(a.images) + (size_t)k * img_stride;
+      b.labels = a.labels + (size_t)k * a.batch;
+      b.loss = a.loss ? a.loss + k : nullptr;
+      b.grads = pass.fbuf(pass.p.grads);
+      pass.backward(b);
+      pass.ok(sgd_update<T>(n->params, b.grads, n->cfg.dtype == VGG19_BF16 ? (T *)n->params_t : (T *)nullptr, 0.f,
+                            n->n_params, st, pass.fbuf(pass.p.lr)), 1);
+      int rc = refresh_filter_copies(n, st);
+      if (rc != VGG19_OK) return rc;
+      pass.launches += n->use_tc ? 2 : 0;
+    }
   }
   if (launches) *launches = pass.launches;
   n->launches[mode] = pass.launches;
@@ -413,9 +456,11 @@ int enqueue_any(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st, int *lau
 // else record it first.  The legacy default stream cannot be captured, so work
 // given to it is enqueued directly.
 int run_pass(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st) {
+  n->other_pass = true;  // vgg19_forward_host_async clears this again for its own passes
   if ((n->cfg.flags & VGG19_FLAG_NO_GRAPH) || st == nullptr || st == cudaStreamLegacy)
     return enqueue_any(n, mode, a, st, nullptr);
-  const void *key[6] = {a.images, a.labels, a.logits, a.probs, a.grads, a.loss};
+  const void *key[6] = {a.images, a.labels, a.logits, a.probs, mode == VGG19_MODE_TRAIN ? (const void *)(intptr_t)a.steps : a.grads,
+                        a.loss};
   for (auto &g : n->graphs)
     if (g.mode == mode && g.batch == a.batch && !memcmp(g.p, key, sizeof key)) {
       CUDA_TRY(n, cudaGraphLaunch(g.exec, st));
@@ -603,6 +648,7 @@ void vgg19_destroy(vgg19_t *n) {
     if (n->ev_uploaded[i]) cudaEventDestroy(n->ev_uploaded[i]);
     if (n->ev_consumed[i]) cudaEventDestroy(n->ev_consumed[i]);
   }
+  if (n->ev_order) cudaEventDestroy(n->ev_order);
   delete n;
 }
 
@@ -659,8 +705,35 @@ int vgg19_sgd_step(vgg19_t *n, const float *grads, float lr, void *stream) {
   return refresh_filter_copies(n, st);
 }
 
+int vgg19_train_steps(vgg19_t *n, const void *images, const int32_t *labels, int32_t batch, int32_t steps, float lr,
+                      float *losses, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!images || !labels || steps < 1 || steps > 64 || !(lr == lr))
+    return fail(n, VGG19_ERR_ARG, "null images / labels, steps outside [1, 64] or NaN learning rate");
+  int rc = check_batch(n, batch, VGG19_MODE_TRAIN, 0);
+  if (rc != VGG19_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Plan p = make_plan(n, batch, VGG19_MODE_TRAIN);
+  // the rate is a device scalar the recorded update kernels read, so one graph serves every rate
+  CUDA_TRY(n, set_scalar(reinterpret_cast<float *>(static_cast<char *>(n->ws) + p.lr), lr, st));
+  PassArgs a{images, labels, nullptr, nullptr, nullptr, losses, batch, steps};
+  return run_pass(n, VGG19_MODE_TRAIN, a, st);
+}
+
+int vgg19_train_step(vgg19_t *n, const void *images, const int32_t *labels, int32_t batch, float lr, float *loss,
+                     void *stream) {
+  return vgg19_train_steps(n, images, labels, batch, 1, lr, loss, stream);
+}
+
+int vgg19_set_dense_grads_event(vgg19_t *n, void *cuda_event) {
+  if (!n) return VGG19_ERR_ARG;
+  drop_graphs(n);  // recorded passes signal the event they were recorded with
+  n->dense_grads_event = static_cast<cudaEvent_t>(cuda_event);
+  return VGG19_OK;
+}
+
 size_t vgg19_workspace_bytes(const vgg19_t *n, int32_t batch, int32_t mode) {
-  if (!n || batch < 1 || batch > n->cfg.batch_max || (mode != 0 && mode != 1)) return 0;
+  if (!n || batch < 1 || batch > n->cfg.batch_max || mode < 0 || mode > 2) return 0;
   return make_plan(n, batch, mode).total;
 }
 
@@ -742,8 +815,18 @@ int vgg19_forward_host_async(vgg19_t *n, const void *host_images, int32_t batch,
       CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_uploaded[i], cudaEventDisableTiming));
       CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_consumed[i], cudaEventDisableTiming));
     }
+    CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_order, cudaEventDisableTiming));
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The staging slots sit behind the work area of a pass at THIS batch.  A pass enqueued earlier at
+  // another batch (or through another entry point) has a work area of another size, which may cover
+  // this call's slots: the early upload would then overwrite activations that pass is still using.
+  // In that case the upload waits for everything enqueued on `stream` so far instead of for the
+  // slot's last reader only.
+  if (n->async_batch != batch || n->other_pass) {
+    CUDA_TRY(n, cudaEventRecord(n->ev_order, st));
+    CUDA_TRY(n, cudaStreamWaitEvent(n->copy_stream, n->ev_order, 0));
+  }
   const unsigned slot = n->next_slot++ & 1u;
   char *base = static_cast<char *>(n->ws) + (size_t)slot * p.io_total;
   size_t img_bytes = (size_t)batch * n->cfg.height * n->cfg.width * 3 * n->elt;
@@ -763,6 +846,8 @@ int vgg19_forward_host_async(vgg19_t *n, const void *host_images, int32_t batch,
   if (host_probs) CUDA_TRY(n, cudaMemcpyAsync(host_probs, probs, out_bytes, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(n, cudaEventRecord(n->ev_consumed[slot], st));
   n->slot_used[slot] = true;
+  n->async_batch = batch;
+  n->other_pass = false;
   return VGG19_OK;
 }
 
@@ -801,6 +886,7 @@ int vgg19_conv_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t b
     // pooling after any layer is well defined; only the fused schedule is per-layer
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  n->other_pass = true;
   cudaError_t e;
   Plan plan{};
   plan.valid = false;  // without a bound workspace the layer runs on kernels that need no scratch
@@ -821,33 +907,42 @@ int vgg19_conv_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t b
   return VGG19_OK;
 }
 
-int vgg19_conv_layer_backward(vgg19_t *n, int32_t layer, const void *x, const void *dz,
-                              int32_t batch, float *dw, float *db, void *dx, void *stream) {
+int vgg19_conv_layer_backward_ex(vgg19_t *n, int32_t layer, const void *x, const void *dz, int32_t batch,
+                                 float *dw, float *db, void *dx, const void *relu_mask, void *stream) {
   if (!n) return VGG19_ERR_ARG;
-  if (layer < 1 || layer > kConvLayers || !x || !dz || !dw || !db || batch < 1)
+  if (layer < 1 || layer > kConvLayers || !dz || batch < 1 || (!dw != !db) || (dw && !x) || (!dw && !dx))
     return fail(n, VGG19_ERR_ARG, "bad layer (%d), batch (%d) or null tensor", layer, batch);
   if (dx && layer == 1) return fail(n, VGG19_ERR_ARG, "layer 1 has no input gradient");
+  if (relu_mask && !dx) return fail(n, VGG19_ERR_ARG, "relu_mask without dx");
   int rc = check_batch(n, batch, VGG19_MODE_BACKWARD, 0);
   if (rc != VGG19_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  n->other_pass = true;
   Plan p = make_plan(n, batch, VGG19_MODE_BACKWARD);
   cudaError_t e;
   if (n->cfg.dtype == VGG19_BF16) {
     Pass<bf16> ps{n, p, st};
-    ps.conv_backward(layer - 1, (const bf16 *)x, (const bf16 *)dz, batch, dw, db, (bf16 *)dx, nullptr);
+    ps.conv_backward(layer - 1, (const bf16 *)x, (const bf16 *)dz, batch, dw, db, (bf16 *)dx, (const bf16 *)relu_mask);
     e = ps.err;
   } else {
     Pass<float> ps{n, p, st};
-    ps.conv_backward(layer - 1, (const float *)x, (const float *)dz, batch, dw, db, (float *)dx, nullptr);
+    ps.conv_backward(layer - 1, (const float *)x, (const float *)dz, batch, dw, db, (float *)dx, (const float *)relu_mask);
     e = ps.err;
   }
   if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
   return VGG19_OK;
 }
 
+int vgg19_conv_layer_backward(vgg19_t *n, int32_t layer, const void *x, const void *dz,
+                              int32_t batch, float *dw, float *db, void *dx, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!x || !dw || !db) return fail(n, VGG19_ERR_ARG, "bad layer (%d), batch (%d) or null tensor", layer, batch);
+  return vgg19_conv_layer_backward_ex(n, layer, x, dz, batch, dw, db, dx, nullptr, stream);
+}
+
 int vgg19_saved_tensor(const vgg19_t *n, int32_t batch, int32_t mode, int32_t index,
                        size_t *offset_bytes, int64_t dims[4]) {
-  if (!n || !offset_bytes || !dims || batch < 1 || batch > n->cfg.batch_max || (mode != 0 && mode != 1) ||
+  if (!n || !offset_bytes || !dims || batch < 1 || batch > n->cfg.batch_max || mode < 0 || mode > 2 ||
       index < 0 || index > 22)
     return VGG19_ERR_ARG;
   Plan p = make_plan(n, batch, mode);
@@ -875,13 +970,22 @@ int vgg19_sync_status(vgg19_t *n, void *stream) {
   CUDA_TRY(n, cudaMemcpy(&code, n->dev_error, sizeof code, cudaMemcpyDeviceToHost));
   if (code != 0) {
     cudaMemset(n->dev_error, 0, 256);
+    if (code == kDevBadLabel)
+      return fail(n, VGG19_ERR_ARG, "a label outside [0, %d) reached the loss (its row's loss is NaN)", kClasses);
     return fail(n, VGG19_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (code %d)", code);
   }
   return VGG19_OK;
 }
 
+int vgg19_selftest_wait_timeout(vgg19_t *n, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  // a millisecond or two of SM clock: long enough to be a real wait, short enough for a test
+  CUDA_TRY(n, tc_wait_selftest(n->dev_error, 2000000ll, static_cast<cudaStream_t>(stream)));
+  return VGG19_OK;
+}
+
 int vgg19_launch_count(const vgg19_t *n, int32_t mode, int32_t *n_kernels) {
-  if (!n || !n_kernels || (mode != 0 && mode != 1)) return VGG19_ERR_ARG;
+  if (!n || !n_kernels || mode < 0 || mode > 2) return VGG19_ERR_ARG;
   *n_kernels = n->launches[mode];
   return VGG19_OK;
 }

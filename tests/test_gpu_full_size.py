@@ -2,17 +2,19 @@
 batch 100, in the launch configuration bench.py times (one CUDA graph per
 pass, tensor-core kernels).
 
-The fp64 CPU checker needs ~2 s per image forward and ~4 s forward+backward,
-so at batch 100 it is applied to sampled images; the rest of the batch is
-covered by properties that hold at any size:
-  * an image's logits do not depend on which batch it sits in (bit for bit:
-    the per-pixel accumulation order does not depend on the batch; the last
-    few images of the batch, whose tiles are cut along K to fill the last
-    round of CTAs, agree to fp32 rounding order instead);
-  * the batch-100 gradient is the mean of the gradients of its ten batch-10
-    chunks (the loss is a mean over images);
-and the gradient of a sampled chunk is checked against the checker's backward
-pass at the forward state the device stored.
+The fp64 CPU checker runs on the whole batch (about a third of a second per
+image forward and a second and a half backward on a 16-core host):
+  * forward: the logits of all 100 images against the checker's, per image,
+    with the strict and the near-tie-aware top-1 agreement counted over all
+    100; and an image's logits do not depend on which batch it sits in (bit
+    for bit: the per-pixel accumulation order does not depend on the batch;
+    the last few images of the batch, whose tiles are cut along K to fill the
+    last round of CTAs, agree to fp32 rounding order instead);
+  * backward: the batch-100 gradient against the checker's backward pass over
+    all 100 images at the forward state the device stored for that very pass
+    (read back chunk by chunk from the workspace, tail images included); the
+    decisions taken on that state against the checker's own on sampled images;
+    the batch-100 gradient is the mean of its ten batch-10 chunk gradients.
 Tolerances as in test_gpu_parity.py: 2e-2 relative L2 (bf16 storage, fp32 sums).
 """
 import numpy as np
@@ -21,7 +23,7 @@ import torch
 
 import oracle
 import seeded_inputs as si
-from test_gpu_parity import check_bf16_backward, rel_l2
+from test_gpu_parity import check_bf16_backward, check_decisions, free_running_cosines, rel_l2, FREE_COSINE_MIN
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -60,8 +62,7 @@ def test_config3_forward_batch1(full):
     ref_s = oracle.vgg19_forward(p64, images[:1], storage="bf16")
     got = logits.cpu().numpy()
     assert rel_l2(got, ref) <= 2e-2 and rel_l2(got, ref_s) <= 2e-2
-    bound = 2e-2 * np.sqrt(np.mean(ref ** 2))
-    assert top1_agrees(got[0], ref[0], bound)
+    assert int(np.argmax(got[0])) == int(np.argmax(ref[0]))
     pr = probs.cpu().numpy()
     assert abs(pr.sum() - 1.0) < 1e-4
     # the softmax of logits this large amplifies a logit error of d into a relative error of ~d
@@ -70,7 +71,7 @@ def test_config3_forward_batch1(full):
     print(f"config 3: logits rel-L2 {rel_l2(got, ref):.2e} (unrounded checker), {rel_l2(got, ref_s):.2e} (bf16 storage)")
 
 
-def test_config4_forward_batch100(full):
+def test_config4_forward_batch100_every_image(full):
     p, net, params, images, labels, x, y = full
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
@@ -79,13 +80,35 @@ def test_config4_forward_batch100(full):
     got = logits.cpu().numpy()
     assert np.isfinite(got).all()
     p64 = params.astype(np.float64)
-    sample = [0, 37, 63, 99]
-    ref = oracle.vgg19_forward(p64, images[sample])
+    ref = np.concatenate([oracle.vgg19_forward(p64, images[i:i + 10]) for i in range(0, B, 10)])
+    errs = np.array([rel_l2(got[i], ref[i]) for i in range(B)])
+    assert errs.max() <= 2e-2, (int(errs.argmax()), float(errs.max()))
+    assert rel_l2(got, ref) <= 2e-2
+    # top-1.  These are random weights on noise images: the logits of an image are nearly tied (the
+    # checker's margin between its best two classes is often below the 2e-2 error bound on a logit), so
+    # the arg-max of several images is decided by rounding.  Counted three ways: strict agreement with
+    # the fp64 checker; agreement when a differing arg-max is excused by a checker margin between the
+    # two candidates below twice the 2e-2 bound on a logit (both answers are then correct) - this is
+    # the reading under which the 99 % bar is asserted; and, as the yardstick for the strict count, how
+    # often the checker's own bf16-storage model agrees strictly with its fp64 self.
     bound = 2e-2 * np.sqrt(np.mean(ref ** 2))
-    agree = 0
-    for row, i in enumerate(sample):
-        assert rel_l2(got[i], ref[row]) <= 2e-2, i
-        agree += top1_agrees(got[i], ref[row], bound)
+    ref_s = np.concatenate([oracle.vgg19_forward(p64, images[i:i + 10], storage="bf16") for i in range(0, B, 10)])
+    strict = sum(int(np.argmax(got[i])) == int(np.argmax(ref[i])) for i in range(B))
+    excused = sum(top1_agrees(got[i], ref[i], bound) for i in range(B))
+    model_strict = sum(int(np.argmax(ref_s[i])) == int(np.argmax(ref[i])) for i in range(B))
+    vs_model = sum(int(np.argmax(got[i])) == int(np.argmax(ref_s[i])) for i in range(B))
+    margins = [float(abs(ref[i][int(np.argmax(ref[i]))] - ref[i][int(np.argmax(got[i]))]) / bound)
+               for i in range(B) if int(np.argmax(got[i])) != int(np.argmax(ref[i]))]
+    print(f"config 4: all {B} images, logits rel-L2 worst {errs.max():.2e} median {np.median(errs):.2e}; top-1 strict "
+          f"{strict}/{B} (the checker's bf16-storage model against its fp64 self: {model_strict}/{B}; device against "
+          f"that model: {vs_model}/{B}), near-ties excused {excused}/{B}; checker margins of the strict "
+          f"disagreements, in units of the logit error bound: {[round(m, 2) for m in margins]}")
+    assert excused >= 99
+    assert strict >= 90 and strict >= model_strict - 3
+    assert rel_l2(got, ref_s) <= 2e-2
+    # an image's result does not depend on the batch it sits in
+    worst_tail = 0.0
+    for i in range(B):
         with torch.cuda.stream(s):
             single = net.forward(x[i:i + 1], stream=s).clone()
         net.sync_status(s)
@@ -97,13 +120,32 @@ def test_config4_forward_batch100(full):
             # Each bf16 store then turns a last-bit difference into a whole bf16 ulp for some elements,
             # so after eight such layers the two results differ like two bf16 implementations do
             # (both are within 2e-2 of the checker, asserted above): bar 1e-2.
-            assert rel_l2(single[0].cpu().numpy(), got[i]) <= 1e-2, i
-    assert agree == len(sample)
-    print(f"config 4: sampled images {sample}, worst logits rel-L2 "
-          f"{max(rel_l2(got[i], ref[r]) for r, i in enumerate(sample)):.2e}, top-1 agreement {agree}/{len(sample)}")
+            e = rel_l2(single[0].cpu().numpy(), got[i])
+            worst_tail = max(worst_tail, e)
+            assert e <= 1e-2, i
+    print(f"config 4: batch-1 logits equal the batch-100 ones bit for bit for images 0..89, tail images within {worst_tail:.2e}")
 
 
-def test_config5_backward_batch100(full):
+def stored_state_chunk(p, net, images, logits, lo, hi):
+    """The checker's (logits, saved) for images lo..hi-1 of the batch-100 pass, from what the device stored."""
+    steps = oracle.vgg19_steps()
+    outs, ci, pi, fi = [], 0, 0, 0
+    for st in steps:
+        if st[0] == "conv":
+            idx = ci; ci += 1
+        elif st[0] == "pool":
+            idx = 16 + pi; pi += 1
+        else:
+            idx = 21 + fi; fi += 1
+        if idx <= 22:
+            t = net.saved_tensor(B, p.VGG19_MODE_BACKWARD, idx)[lo:hi].float().cpu().numpy().astype(np.float64)
+            outs.append(t.reshape(hi - lo, 4096) if idx >= 21 else t)
+        else:
+            outs.append(np.asarray(logits[lo:hi], dtype=np.float64))
+    return oracle.state_from_outputs(steps, images[lo:hi], outs)
+
+
+def test_config5_backward_batch100_every_image(full):
     p, net, params, images, labels, x, y = full
     s = torch.cuda.Stream()
     grads = torch.empty(net.n_params, dtype=torch.float32, device=DEV)
@@ -113,6 +155,42 @@ def test_config5_backward_batch100(full):
         net.backward(x, y, grads=grads, loss=loss, logits=logits, stream=s)
     net.sync_status(s)
     assert torch.isfinite(grads).all()
+    got_logits = logits.cpu().numpy()
+    # the checker differentiates the network, image chunk by image chunk, at the forward state this very
+    # batch-100 pass stored (tail images included), and the chunk gradients add up to the batch gradient
+    steps = oracle.vgg19_steps()
+    p64 = params.astype(np.float64)
+    o_grads = np.zeros(p64.size)
+    o_loss = 0.0
+    decisions_checked = []
+    for lo in range(0, B, 4):
+        state = stored_state_chunk(p, net, images, got_logits, lo, lo + 4)
+        if lo in (0, 48, 96):
+            # sampled chunks (start, middle, tail): the device's decisions against the checker's own, and
+            # its stored activations against the checker's
+            o_logits, o_saved = oracle.forward(steps, p64, images[lo:lo + 4], keep=True, storage="bf16")
+            assert rel_l2(got_logits[lo:lo + 4], o_logits) <= 2e-2
+            for sd, so in zip(state[1], o_saved):
+                if sd[0] in ("conv", "fc"):
+                    assert rel_l2(sd[2], so[2]) <= 2e-2, (lo, sd[0])
+            decisions_checked.append(check_decisions(state[1], o_saved))
+        l, _, _ = oracle.backward(steps, p64, images[lo:lo + 4], labels[lo:lo + 4], n_total=B, grads=o_grads,
+                                  storage="bf16", state=state)
+        o_loss += l
+    assert abs(float(loss) - o_loss) <= 1e-3 * abs(o_loss)
+    g = grads.cpu().numpy()
+    worst = 0.0
+    for off, dims in net.param_slices():
+        n = int(np.prod(dims))
+        e = rel_l2(g[off:off + n], o_grads[off:off + n])
+        worst = max(worst, e)
+        assert e <= 2e-2, (dims, e)
+    rows = [r for d in decisions_checked for r in d]
+    print(f"config 5: batch-100 gradient against the checker over all {B} images at the stored state, worst tensor "
+          f"{worst:.2e}; loss {float(loss):.5f} vs {o_loss:.5f}; decisions on images 0-3, 48-51, 96-99: masks differ <= "
+          f"{max(f for k, f, _ in rows if k != 'pool'):.2e}, pools <= {max(f for k, f, _ in rows if k == 'pool'):.2e}, "
+          f"worst near-tie {max(w for _, _, w in rows):.2e} of rms")
+    del o_grads
     # property: mean of the ten batch-10 chunk gradients
     mean = torch.zeros_like(grads)
     mean_loss = 0.0
@@ -133,10 +211,13 @@ def test_config5_backward_batch100(full):
         worst = max(worst, e)
         assert e <= 2e-2, (dims, e)
     print(f"config 5: batch-100 gradient vs mean of batch-10 chunk gradients, worst tensor {worst:.2e}")
-    # sampled chunk against the checker at the stored forward state
-    n_s = 2
-    lg = torch.empty(n_s, 1000, dtype=torch.float32, device=DEV)
+    # free-running: the device's gradient of a batch of 8 (the first and the last four images) against the
+    # checker's own pass on them, each side at its own forward state: direction of every tensor
+    pick = [0, 1, 2, 3, 96, 97, 98, 99]
     with torch.cuda.stream(s):
-        net.backward(x[:n_s], y[:n_s], grads=g10, loss=l10, logits=lg, stream=s)
+        net.backward(x[pick].contiguous(), y[pick].contiguous(), grads=g10, loss=l10, stream=s)
     net.sync_status(s)
-    check_bf16_backward(net, params, images[:n_s], labels[:n_s], lg.cpu().numpy(), g10.cpu().numpy(), float(l10))
+    _, own, _ = oracle.vgg19_backward(p64, images[pick], labels[pick], chunk=4, storage="bf16")
+    cos = free_running_cosines(net, g10.cpu().numpy(), own)
+    print(f"config 5: free-running gradient of 8 images, smallest per-tensor cosine {min(cos):.4f}")
+    assert min(cos) >= FREE_COSINE_MIN, cos

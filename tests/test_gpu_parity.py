@@ -11,8 +11,13 @@ activations read back from the workspace).  The ReLU masks and pool
 arg-maxima are integer decisions made on those stored values; an
 implementation whose forward arithmetic differs by one part in 10^7 flips
 enough near-zero pre-activations to move every gradient tensor by 5-25%, so
-gradients are compared where they are unique: given the decisions.  The
-unsynchronised difference is printed for information.
+gradients are compared where they are unique: given the decisions
+(tests/test_oracle_bf16_sensitivity.py reproduces that measurement with the
+checker alone).  What that comparison cannot see is asserted separately: the
+fraction of decisions on which the device's stored state and the checker's own
+forward pass differ is small and every differing one is a near-tie, and the
+free-running gradient (each side at its own forward state) keeps the direction
+of every tensor (cosine >= 0.90).
 """
 import numpy as np
 import pytest
@@ -72,8 +77,77 @@ def device_state(net, B, images, logits):
     return oracle.state_from_outputs(steps, images, outs)
 
 
+def pool_argmax(x):
+    """Arg-max (0..3, scan order (0,0),(0,1),(1,0),(1,1), first maximum wins) and the four candidates
+    of every 2x2 window of an NHWC tensor."""
+    N, Hh, Ww, C = x.shape
+    w = x.reshape(N, Hh // 2, 2, Ww // 2, 2, C).transpose(0, 1, 3, 5, 2, 4).reshape(N, Hh // 2, Ww // 2, C, 4)
+    return np.argmax(w, axis=-1), w
+
+
+def decision_agreement(d_saved, o_saved):
+    """How far the integer decisions of the backward pass (ReLU masks, pool arg-maxima) taken on the
+    device's stored forward state are from those the checker takes on its own bf16-storage forward
+    pass.  Per step: (kind, fraction of decisions that differ, worst near-tie measure), where the
+    near-tie measure of a differing decision is the size of the value that decided it relative to the
+    layer's rms: the activation itself for a mask, the checker's margin between the two candidate
+    positions for a pooling window.  A correct forward pass differs only on near-ties."""
+    out = []
+    for sd, so in zip(d_saved, o_saved):
+        if sd[0] in ("conv", "fc"):
+            if sd[0] == "fc" and not sd[4]:
+                continue
+            yd, yo = sd[2], so[2]
+            rms = float(np.sqrt(np.mean(yo ** 2))) + 1e-300
+            differ = (yd > 0) != (yo > 0)
+            frac = float(differ.mean())
+            worst = float(np.maximum(yd, yo)[differ].max() / rms) if differ.any() else 0.0
+            out.append((sd[0] + "-relu", frac, worst))
+        else:
+            ad, _ = pool_argmax(sd[1])
+            ao, wo = pool_argmax(so[1])
+            live = wo.max(axis=-1) > 0  # a window of zeros passes no gradient through the ReLU below
+            differ = (ad != ao) & live
+            frac = float(differ.sum() / max(int(live.sum()), 1))
+            rms = float(np.sqrt(np.mean(so[1] ** 2))) + 1e-300
+            margin = wo.max(axis=-1) - np.take_along_axis(wo, ad[..., None], axis=-1)[..., 0]
+            worst = float(margin[differ].max() / rms) if differ.any() else 0.0
+            out.append(("pool", frac, worst))
+    return out
+
+
+# Bounds on the decisions that may differ between the device's forward state and the checker's own.
+# Measured at 224x224 on twelve images of the batch-100 pass: at most 0.27 % of a layer's ReLU masks and
+# 2.7 % of its live pooling windows (bf16 keeps 8 significant bits, so neighbouring positive activations
+# tie or sit one ulp apart often), every one of them a near-tie: the deciding value at most 6 % of the
+# layer's rms, while the activations agree to 2e-2 in L2.
+MASK_DIFFER_MAX, POOL_DIFFER_MAX, NEAR_TIE_MAX = 0.02, 0.06, 0.25
+# Free-running comparison (each side differentiates at its own forward state): direction only.  The
+# checker against itself under a 1e-7 weight perturbation keeps 0.978 (32x32); the device against the
+# checker measured 0.945 on the least aligned tensor (the first layer's filter, 224x224, 8 images).
+FREE_COSINE_MIN = 0.90
+
+
+def check_decisions(d_saved, o_saved):
+    rows = decision_agreement(d_saved, o_saved)
+    for kind, frac, worst in rows:
+        assert frac <= (POOL_DIFFER_MAX if kind == "pool" else MASK_DIFFER_MAX), rows
+        assert worst <= NEAR_TIE_MAX, rows
+    return rows
+
+
+def free_running_cosines(net, grads, o_grads):
+    cos = []
+    for off, dims in net.param_slices():
+        n = int(np.prod(dims))
+        a, b = np.asarray(grads[off:off + n], dtype=np.float64), o_grads[off:off + n]
+        cos.append(float(a @ b / max(np.linalg.norm(a) * np.linalg.norm(b), 1e-300)))
+    return cos
+
+
 def check_bf16_backward(net, params, images, labels, logits, grads, loss, tol=2e-2):
-    """Forward parity on logits and stored activations; backward parity at the stored state."""
+    """Forward parity on logits and stored activations; the decisions taken on the stored state against
+    the checker's own; backward parity at the stored state; direction of the free-running gradient."""
     B = images.shape[0]
     steps = oracle.vgg19_steps()
     p64 = params.astype(np.float64)
@@ -87,13 +161,18 @@ def check_bf16_backward(net, params, images, labels, logits, grads, loss, tol=2e
         if sd[0] in ("conv", "fc") and sd[2].shape == so[2].shape:
             worst_act = max(worst_act, rel_l2(sd[2], so[2]))
     assert worst_act <= tol
+    decisions = check_decisions(d_saved, o_saved)
     o_loss, o_grads, _ = oracle.backward(steps, p64, images, labels, storage="bf16", state=(d_logits, d_saved))
     assert abs(loss - o_loss) <= 1e-3 * abs(o_loss)
     worst = check_grads(net, grads, o_grads, tol)
-    _, free_grads, _ = oracle.backward(steps, p64, images, labels, storage="bf16")
+    _, free_grads, _ = oracle.backward(steps, p64, images, labels, storage="bf16", state=(o_logits, o_saved))
+    cos = free_running_cosines(net, grads, free_grads)
+    assert min(cos) >= FREE_COSINE_MIN, cos
     print(f"bf16 {images.shape[1]}x{images.shape[2]} B={B}: logits {e_logits:.2e}, worst activation {worst_act:.2e}, "
-          f"worst gradient tensor at the stored state {worst:.2e}, whole-gradient difference to the checker's own "
-          f"forward state {rel_l2(grads, free_grads):.2e}")
+          f"decisions differing: masks <= {max(f for k, f, _ in decisions if k != 'pool'):.2e}, pools <= "
+          f"{max(f for k, f, _ in decisions if k == 'pool'):.2e}, worst near-tie {max(w for _, _, w in decisions):.2e} of rms; "
+          f"worst gradient tensor at the stored state {worst:.2e}; free-running: whole-gradient difference "
+          f"{rel_l2(grads, free_grads):.2e}, smallest per-tensor cosine {min(cos):.4f}")
     return worst
 
 
@@ -311,3 +390,183 @@ def test_async_host_entry_point_matches_the_blocking_one():
         assert torch.equal(g, w)
     assert not torch.equal(want[0], want[1])
     net.close()
+
+
+def test_async_host_entry_point_with_changing_batch_sizes():
+    """The staging slots of vgg19_forward_host_async sit behind the work area of a pass at the call's own
+    batch, so a smaller batch right after a larger one (the ragged last batch of a serving loop) would
+    upload into memory the larger pass is still using unless the library orders the two.  Alternating
+    batch 4 and batch 1 must give the blocking call's logits bit for bit."""
+    p = pkg()
+    params, _, _ = make_inputs(64, 64, 4, True)
+    net = p.Net(64, 64, 4, p.VGG19_BF16, params=params, mode=p.VGG19_MODE_FORWARD, host_io=True)
+    stream = torch.cuda.Stream()
+    sizes = [4, 1, 4, 1, 1, 4, 2, 4]
+    batches = [torch.from_numpy(si.images(b, 64, 64, seed=30 + i, bf16_exact=True)).to(torch.bfloat16).pin_memory()
+               for i, b in enumerate(sizes)]
+    want = []
+    for x, b in zip(batches, sizes):
+        out = torch.empty(b, 1000, dtype=torch.float32).pin_memory()
+        p.vgg19_forward_host(net.handle, x, b, out, None, stream)
+        want.append(out.clone())
+    for _ in range(3):
+        got = [torch.full((b, 1000), float("nan"), dtype=torch.float32).pin_memory() for b in sizes]
+        for x, b, out in zip(batches, sizes, got):
+            p.vgg19_forward_host_async(net.handle, x, b, out, None, stream)
+        net.sync_status(stream)
+        for g, w in zip(got, want):
+            assert torch.equal(g, w)
+    net.close()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
+    """Every wait inside the tensor-core kernels is bounded; one that runs out records a code and the
+    kernel returns.  The library's self-test kernel waits (about a millisecond) on a barrier nothing
+    arrives on: vgg19_sync_status must report VGG19_ERR_DEVICE_TIMEOUT once, clear the record, and the
+    next pass on the same handle must give the result it gave before."""
+    p = pkg()
+    params, images, _ = make_inputs(32, 32, 2, True)
+    net = p.Net(32, 32, 2, p.VGG19_BF16, params=params, mode=p.VGG19_MODE_FORWARD)
+    x = torch.from_numpy(images).to(DEV).to(torch.bfloat16)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        before = net.forward(x, stream=s).clone()
+    net.sync_status(s)
+    p.vgg19_selftest_wait_timeout(net.handle, s)
+    with pytest.raises(p.binding.Vgg19Error) as e:
+        net.sync_status(s)
+    assert e.value.code == p.VGG19_ERR_DEVICE_TIMEOUT
+    net.sync_status(s)  # the record was cleared
+    with torch.cuda.stream(s):
+        after = net.forward(x, stream=s).clone()
+    net.sync_status(s)
+    assert torch.equal(before, after)
+    net.close()
+
+
+def test_a_label_out_of_range_is_reported_not_dereferenced():
+    p = pkg()
+    B = 3
+    params, images, labels = make_inputs(32, 32, B, True)
+    net = p.Net(32, 32, B, p.VGG19_BF16, params=params)
+    x = torch.from_numpy(images).to(DEV).to(torch.bfloat16)
+    for bad in (1000, -7, 2 ** 31 - 1):
+        y = torch.from_numpy(labels).to(DEV).clone()
+        y[1] = bad
+        grads, loss = net.backward(x, y)
+        with pytest.raises(p.binding.Vgg19Error) as e:
+            net.sync_status()
+        assert e.value.code == p.VGG19_ERR_ARG
+        assert torch.isnan(loss).all()
+    grads, loss = net.backward(x, torch.from_numpy(labels).to(DEV))
+    net.sync_status()
+    assert torch.isfinite(loss).all() and torch.isfinite(grads).all()
+    net.close()
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_train_steps_as_one_graph_match_backward_then_sgd_step(bf16):
+    """vgg19_train_steps (k training steps recorded as one CUDA graph: forward, loss, backward, parameter
+    update and filter-copy rebuild per step, the gradient staying in the workspace) against the same k
+    steps made of separate vgg19_backward + vgg19_sgd_step calls (bit for bit: same kernels, same order),
+    and the first step against the checker: loss and updated parameters w - lr * dL/dw at the stored
+    forward state."""
+    p = pkg()
+    B, K, lr = 2, 3, 0.02
+    dtype = p.VGG19_BF16 if bf16 else p.VGG19_FP32
+    params, _, _ = make_inputs(32, 32, B, bf16, bias_std=0.1)
+    images = si.images(K * B, 32, 32, seed=1, bf16_exact=bf16)
+    labels = si.labels(K * B, seed=2)
+    net = p.Net(32, 32, B, dtype, params=params, mode=p.VGG19_MODE_TRAIN)
+    x = torch.from_numpy(images).to(DEV).to(net.act_dtype)
+    y = torch.from_numpy(labels).to(DEV)
+    s = torch.cuda.Stream()
+    # reference sequence on the same handle: separate calls
+    ref_losses, first_grads, first_logits = [], None, None
+    for k in range(K):
+        logits = torch.empty(B, 1000, dtype=torch.float32, device=DEV)
+        with torch.cuda.stream(s):
+            grads, loss = net.backward(x[k * B:(k + 1) * B], y[k * B:(k + 1) * B], logits=logits, stream=s)
+            if k == 0:
+                net.sync_status(s)
+                first_grads, first_logits = grads.cpu().numpy(), logits.cpu().numpy()
+                first_state = device_state(net, B, images[:B], first_logits) if bf16 else None
+            net.sgd_step(grads, lr, stream=s)
+        net.sync_status(s)
+        ref_losses.append(float(loss))
+    want = np.empty_like(params)
+    p.vgg19_get_params(net.handle, want)
+    # the same three steps as one graph, from the same starting point, twice (the second run replays the graph)
+    for run in range(2):
+        p.vgg19_set_params(net.handle, params)
+        losses = torch.full((K,), float("nan"), dtype=torch.float32, device=DEV)
+        p.vgg19_train_steps(net.handle, x, y, B, K, lr, losses, s)
+        net.sync_status(s)
+        got = np.empty_like(params)
+        p.vgg19_get_params(net.handle, got)
+        assert np.array_equal(got, want), run
+        assert losses.cpu().tolist() == ref_losses, run
+    assert p.vgg19_launch_count(net.handle, p.VGG19_MODE_TRAIN) >= K * (16 + 3 + 1)
+    # one step against the checker
+    p.vgg19_set_params(net.handle, params)
+    loss1 = torch.empty(1, dtype=torch.float32, device=DEV)
+    p.vgg19_train_step(net.handle, x[:B], y[:B], B, lr, loss1, s)
+    net.sync_status(s)
+    after = np.empty_like(params)
+    p.vgg19_get_params(net.handle, after)
+    steps = oracle.vgg19_steps()
+    p64 = params.astype(np.float64)
+    if bf16:
+        o_loss, o_grads, _ = oracle.backward(steps, p64, images[:B], labels[:B], storage="bf16", state=first_state)
+    else:
+        o_loss, o_grads, _ = oracle.backward(steps, p64, images[:B], labels[:B])
+    assert abs(float(loss1) - o_loss) <= 1e-3 * abs(o_loss)
+    o_after = oracle.sgd_step(p64, o_grads, lr)
+    # compare the step taken, not the parameters (which barely move): w_after - w_before
+    assert rel_l2(after.astype(np.float64) - p64, o_after - p64) <= (2e-2 if bf16 else 2e-4)
+    net.close()
+
+
+def test_dense_gradient_event_fires_inside_the_pass_and_changes_nothing():
+    """With vgg19_set_dense_grads_event the backward pass (as a recorded graph and enqueued directly) signals
+    the caller's event once the three dense layers' gradients are final: a side stream that waits for the
+    event and copies that part of the gradient buffer must get the final values, must be done before the
+    pass ends, and the gradients must equal those of a pass without the event."""
+    p = pkg()
+    B = 4
+    params, images, labels = make_inputs(64, 64, B, True)
+    x = torch.from_numpy(images).to(DEV).to(torch.bfloat16)
+    y = torch.from_numpy(labels).to(DEV)
+    for flags in (0, p.VGG19_FLAG_NO_GRAPH):
+        net = p.Net(64, 64, B, p.VGG19_BF16, params=params, flags=flags)
+        dense_off, _ = p.vgg19_param_info(net.handle, 32)
+        s, side = torch.cuda.Stream(), torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            plain, _ = net.backward(x, y, stream=s)
+            plain = plain.clone()
+        net.sync_status(s)
+        ev = torch.cuda.Event(enable_timing=False)
+        ev.record(s)  # creates the underlying event
+        p.vgg19_set_dense_grads_event(net.handle, ev)
+        grads = torch.zeros(net.n_params, dtype=torch.float32, device=DEV)
+        early = torch.zeros(net.n_params - dense_off, dtype=torch.float32, device=DEV)
+        done_side, done_pass = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start = torch.cuda.Event(enable_timing=True)
+        for rep in range(3):  # first call records the graph, later ones replay it
+            grads.zero_()
+            torch.cuda.synchronize()
+            with torch.cuda.stream(s):
+                start.record(s)
+                net.backward(x, y, grads=grads, stream=s)
+                done_pass.record(s)
+            with torch.cuda.stream(side):
+                side.wait_event(ev)
+                early.copy_(grads[dense_off:])
+                done_side.record(side)
+            torch.cuda.synchronize()
+            net.sync_status(s)
+            assert torch.equal(grads, plain)
+            assert torch.equal(early, plain[dense_off:]), "the dense gradients were not final when the event fired"
+            assert start.elapsed_time(done_side) < start.elapsed_time(done_pass), "the event did not fire before the pass ended"
+        p.vgg19_set_dense_grads_event(net.handle, None)
+        net.close()

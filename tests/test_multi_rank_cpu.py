@@ -64,7 +64,14 @@ def _grad_worker(rank, world, port, out):
     _, g, _ = oracle.backward(TINY, params, x[half], labels[half])
     t = torch.from_numpy(g.copy())
     bench.average_gradients(t, world)
-    out[rank] = oracle.sgd_step(params, t.numpy(), 0.1)
+    # the overlapped exchange of the training step averages the buffer in two buckets (the dense layers'
+    # gradients first, the convolution layers' at the end of the pass): same result as one all-reduce
+    t2 = torch.from_numpy(g.copy())
+    cut = t2.numel() // 3
+    bench.average_gradients(t2[cut:], world)
+    bench.average_gradients(t2[:cut], world)
+    assert torch.equal(t, t2)
+    out[rank] = oracle.sgd_step(params, t2.numpy(), 0.1)
     dist.barrier()
     dist.destroy_process_group()
 
@@ -86,3 +93,21 @@ def test_two_ranks_average_to_the_whole_batch_gradient():
     want = oracle.sgd_step(params, g_all, 0.1)
     assert np.array_equal(res[0], res[1])  # replicas stay identical
     assert np.allclose(res[0], want, rtol=1e-12, atol=1e-14)
+
+
+def test_bench_gpus_n_starts_n_ranks_by_itself():
+    """`python bench.py --gpus 2` with no launcher in the environment must start two ranks (here CPU ranks
+    over gloo, plumbing only) and report the whole job: n_gpus 2, the slowest rank's time, both batches."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--backend", "gloo", "--dry",
+                        "--steps", "4"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2
+    assert abs(out["ms_per_step"] - 11.0) < 1e-9          # rank 1 pretends 11 ms per step: the slowest rank's
+    assert abs(out["value"] - 2 * 100 / 11e-3) < 1e-6    # both ranks' batches count
+    assert abs(out["mean_gradient"] - 1.5) < 1e-12       # mean of the ranks' constant gradients 1 and 2

@@ -6,8 +6,11 @@ budget), so they can neither create a network handle nor supply a workspace.
 vgg19_conv_wgrad_static() serves them from a scratch array built into the
 library.  This test calls it through the C ABI twice in a row - the second
 call finds the scratch dirty from the first - and compares both results with
-the handle-based vgg19_conv_layer_backward on the same tensors, within the
-per-layer tolerance of the other convolution tests (relative L2 <= 1e-3).
+the handle-based vgg19_conv_layer_backward on the same tensors and with the
+fp64 CPU checker's filter gradient, within the per-layer tolerance of the other
+convolution tests (relative L2 <= 1e-3).  The second call must leave the
+amount of free device memory as it found it (the first call on a device is the
+one that may make the driver load the library's code and the scratch array).
 It also checks that a shape beyond the built-in scratch is refused.
 
 Collected last on purpose: a run that stops at the first failure has then
@@ -17,6 +20,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import seeded_inputs as si
 
 pytestmark = pytest.mark.gpu
@@ -48,12 +52,20 @@ def test_static_scratch_wgrad_matches_the_workspace_path_twice(dtype_name):
         p.vgg19_conv_layer_backward(net.handle, layer, x, dz, B, dw_ref, db_ref, None, stream)
         dw = torch.full_like(dw_ref, float("nan"))
         db = torch.full_like(db_ref, float("nan"))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         rc, need = p.vgg19_conv_wgrad_static(x, dz, B, S, S, Cin, Cout, dtype, dw, db, stream)
         assert rc == p.VGG19_OK and 0 < need <= p.VGG19_STATIC_SCRATCH_BYTES
         net.sync_status()
+        if call == 1:
+            assert torch.cuda.mem_get_info()[0] == free_before, "a call after the first changed free device memory"
         assert torch.isfinite(dw).all() and torch.isfinite(db).all()
         assert rel_l2(dw, dw_ref) <= 1e-3, call
         assert rel_l2(db, db_ref) <= 1e-3, call
+        o_dw, o_db = oracle.conv3x3_wgrad(x.float().cpu().numpy().astype(np.float64),
+                                          dz.float().cpu().numpy().astype(np.float64))
+        assert rel_l2(dw.cpu(), torch.from_numpy(o_dw)) <= 1e-3, call
+        assert rel_l2(db.cpu(), torch.from_numpy(o_db)) <= 1e-3, call
     net.close()
 
 
