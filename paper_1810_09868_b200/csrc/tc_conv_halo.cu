@@ -299,6 +299,20 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     uint32_t stage_sel = 0;  // which of the two staging tiles the next chunk uses
     const uint8_t* mask_srow = smem_raw + (mask_smem - smem_u32(smem_raw)) + row * 128;
     uint32_t mask_phase = 0;
+    bool mask_pending = false;  // issuer only: a mask copy is in flight or unread
+    // Input gradient: the ReLU mask (the layer below's output at the same pixels) of a 64-channel chunk
+    // arrives as one tiled box in the staging layout.  The issuer requests the NEXT chunk's box as soon
+    // as every thread has read the current one, so that the copy's latency hides behind the rest of
+    // the epilogue and the wait for the next accumulator.
+    auto request_mask = [&](int unit, int c64) {
+      if (unit >= total_units) return;
+      const int mt = unit_m_tile(unit), nt = unit % a.n_tiles;
+      const int tw = mt % a.tiles_w, t = mt / a.tiles_w;
+      mbar_expect_tx(mask_bar, T::OUT_BYTES);
+      tma_load_4d(mask_smem, &map_m, mask_bar, nt * BN + c64, tw * PW, (t % a.tiles_h) * PH, t / a.tiles_h);
+      mask_pending = true;
+    };
+    if (a.mask && issuer) request_mask(first_unit, 0);
     for (int unit = first_unit; unit < total_units; unit += unit_stride, ++local) {
       const int buf = local % NACC;
       const uint32_t use = (uint32_t)(local / NACC);
@@ -322,14 +336,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           if (issuer) tma_store_wait_read<1>();  // the store before last, which used this staging tile, has read it
           named_bar_sync(1, 128);
         }
-        // input gradient: the ReLU mask (the layer below's output at the same pixels) arrives as one
-        // tiled box in the staging layout; everyone finished reading the previous one before the
-        // barrier above
         bool mask_ready = false;
-        if (a.mask && issuer) {
-          mbar_expect_tx(mask_bar, T::OUT_BYTES);
-          tma_load_4d(mask_smem, &map_m, mask_bar, c_base + c64, tw * PW, th * PH, img);
-        }
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           const int cc = c64 + half * 32;
@@ -347,7 +354,7 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           }
           if (a.mask) {
             if (!mask_ready) {  // a failed wait leaves the tile unmasked; the error word says so
-              mask_ready = mbar_wait(mask_bar, mask_phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
+              mbar_wait(mask_bar, mask_phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
               mask_phase ^= 1;
               mask_ready = true;
             }
@@ -394,10 +401,14 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         }
         if (a.out) {
           fence_async_smem();
-          named_bar_sync(1, 128);
+          named_bar_sync(1, 128);  // the staging tile is complete, and everyone has read the mask tile
           if (issuer) {
             tma_store_4d(&map_y, out_smem + stage_sel * T::OUT_BYTES, c_base + c64, tw * PW, th * PH, img);
             tma_store_commit();
+            if (a.mask) {
+              mask_pending = false;
+              if (c64 + 64 < BN) request_mask(unit, c64 + 64); else request_mask(unit + unit_stride, 0);
+            }
           }
           stage_sel ^= 1;
         }
@@ -411,6 +422,11 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       } else {
         mbar_arrive(acc_empty(buf));
       }
+    }
+    if (issuer && mask_pending) {
+      // left early (a wait ran out) with a mask copy in flight: let it land before shared memory goes away
+      const unsigned long long t0 = global_timer_ns();
+      while (!mbar_try_wait(mask_bar, mask_phase) && global_timer_ns() - t0 < 100000000ull) {}
     }
     if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }

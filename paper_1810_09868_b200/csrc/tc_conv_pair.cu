@@ -36,9 +36,9 @@ struct PairTile {
   static constexpr int B_BYTES = (BN / 2) * BK * 2;  // this CTA's half of the filter slice
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int OUT_BYTES = BM * 64 * 2;      // staging tile of the TMA store
-  static constexpr int STAGES = (kSmemLimit - 4608 - OUT_BYTES) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608 - OUT_BYTES) / STAGE_BYTES;
+  static constexpr int STAGES = (kSmemLimit - 4608 - 2 * OUT_BYTES) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608 - 2 * OUT_BYTES) / STAGE_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;           // double-buffered accumulator
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + 1024 + 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_BYTES + 1024 + 256;  // staging tile + mask tile
 };
 
 struct PairArgs {
@@ -77,17 +77,19 @@ __device__ __forceinline__ Work get_work(int w, const PairArgs& a, int k_blocks)
 template <int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                       const __grid_constant__ CUtensorMap map_y, PairArgs a) {
+                       const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_m, PairArgs a) {
   using T = PairTile<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t out_smem = smem_base + T::STAGES * T::STAGE_BYTES;
-  const uint32_t bars = out_smem + T::OUT_BYTES;
+  const uint32_t mask_smem = out_smem + T::OUT_BYTES;  // ReLU-mask tile of the chunk being finished (input gradient)
+  const uint32_t bars = mask_smem + T::OUT_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };                       // used in the even CTA
   auto empty_bar = [&](int s) { return bars + 8u * (T::STAGES + s); };        // both CTAs
   auto acc_full_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + b); };       // both CTAs
   auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + 2 + b); };  // used in the even CTA
   const uint32_t drain_bar = bars + 8u * (2 * T::STAGES + 4);
+  const uint32_t mask_bar = bars + 8u * (2 * T::STAGES + 5);  // this CTA's own
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ __align__(16) float bias_s[512];
@@ -105,6 +107,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     for (int s = 0; s < T::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 2); }
     mbar_init(drain_bar, 1);
+    mbar_init(mask_bar, 1);
     mbar_fence_init();
     tma_prefetch_desc(&map_x);
     tma_prefetch_desc(&map_w);
@@ -211,6 +214,28 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     int local = 0;
     const bool issuer = threadIdx.x == 64;  // owns the TMA store groups
     uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
+    const uint8_t* mask_srow = smem_raw + (mask_smem - smem_u32(smem_raw)) + row * 128;
+    // Input gradient: the ReLU mask (the stored output of the layer below at the same pixels and
+    // channels) of a 128 x 64 chunk arrives by TMA in the staging tile's layout.  The issuer requests
+    // the NEXT chunk's tile as soon as every thread has read the current one, so the copy's latency
+    // hides behind the rest of the epilogue and the wait for the next accumulator.
+    uint32_t mask_phase = 0;
+    bool mask_pending = false;  // issuer only: a mask copy is in flight or unread
+    // first chunk (work item, 64-column block) at or after (w, c64) whose epilogue applies a mask here
+    auto request_mask = [&](int w, int c64) {
+      for (; w < total_work; w += n_pairs, c64 = 0) {
+        const Work wk = get_work(w, a, k_blocks);
+        if (wk.split >= 0) return;  // tail items (all that follow, too) are masked by the finishing kernel
+        const int mp = wk.tile / a.n_tiles, nt = wk.tile - mp * a.n_tiles;
+        const int mt = 2 * mp + (int)rank;
+        if ((long)mt * BM >= a.pixels) continue;
+        mbar_expect_tx(mask_bar, T::OUT_BYTES);
+        tma_load_2d(mask_smem, &map_m, mask_bar, nt * BN + c64, mt * BM);  // rows past the end read as zero
+        mask_pending = true;
+        return;
+      }
+    };
+    if (a.mask && issuer) request_mask(pair, 0);
     for (int w = pair; w < total_work; w += n_pairs, ++local) {
       const Work wk = get_work(w, a, k_blocks);
       const int buf = local & 1;
@@ -224,7 +249,6 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       const bool valid = pixel < a.pixels;
       const bool tile_valid = (long)m_tile * BM < a.pixels;
       const int c_base = n_tile * BN;
-      const bf16* mask_row = (a.mask && valid) ? a.mask + pixel * a.Cout + c_base : nullptr;
       if (wk.split >= 0) {
         // part of a tail tile's K range: raw sums, one row per thread, for the finishing kernel
         float* dst = a.partial + ((size_t)wk.split * a.tail_rows + (size_t)(pixel - a.tail_row0)) * a.Cout + c_base;
@@ -249,6 +273,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       for (int c64 = 0; c64 < BN && tile_valid; c64 += 64) {
         if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
         named_bar_sync(1, 128);
+        bool mask_ready = false;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           const int cc = c64 + half * 32;
@@ -264,11 +289,15 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
             packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
           }
-          if (mask_row) {
-            const uint4* mp = reinterpret_cast<const uint4*>(mask_row + cc);
+          if (a.mask) {
+            if (!mask_ready) {  // a failed wait leaves the chunk unmasked; the error word says so
+              mbar_wait(mask_bar, mask_phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
+              mask_phase ^= 1;
+              mask_ready = true;
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const uint4 m = __ldg(mp + q);
+              const uint4 m = *reinterpret_cast<const uint4*>(mask_srow + (((half * 4 + q) ^ (row & 7)) << 4));
               const uint32_t mw[4] = {m.x, m.y, m.z, m.w};
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
@@ -289,16 +318,25 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           }
         }
         fence_async_smem();
-        named_bar_sync(1, 128);
+        named_bar_sync(1, 128);  // the staging tile is complete, and everyone has read the mask tile
         if (issuer) {
           // rows past the end of the tensor (last tile) are clipped by the copy engine
           tma_store_2d(&map_y, out_smem, c_base + c64, m_tile * BM);
           tma_store_commit();
+          if (a.mask) {
+            mask_pending = false;
+            if (c64 + 64 < BN) request_mask(w, c64 + 64); else request_mask(w + n_pairs, 0);
+          }
         }
       }
       tc_fence_before();
       named_bar_sync(1, 128);
       if (issuer) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));  // one arrival per CTA of the pair
+    }
+    if (issuer && mask_pending) {
+      // left early (a wait ran out) with a mask copy in flight: let it land before shared memory goes away
+      const unsigned long long t0 = global_timer_ns();
+      while (!mbar_try_wait(mask_bar, mask_phase) && global_timer_ns() - t0 < 100000000ull) {}
     }
     if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }
@@ -403,10 +441,12 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
   if (!tc_conv3x3_pair_supported(s)) return cudaErrorInvalidValue;
   constexpr int BN = 256;
   using T = PairTile<BN>;
-  CUtensorMap mx, mw, my;
+  CUtensorMap mx, mw, my, mm;
   if (!make_im2col_map(&mx, in, s.N, s.H, s.W, s.Cin, BM)) return cudaErrorInvalidValue;
   if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, BN / 2)) return cudaErrorInvalidValue;
   if (!make_tiled_map_2d(&my, out, (uint64_t)s.N * s.H * s.W, (uint64_t)s.Cout, BM)) return cudaErrorInvalidValue;
+  mm = my;  // only read when there is a mask
+  if (mask && !make_tiled_map_2d(&mm, mask, (uint64_t)s.N * s.H * s.W, (uint64_t)s.Cout, BM)) return cudaErrorInvalidValue;
   PairArgs a;
   a.pixels = s.N * s.H * s.W;
   a.H = s.H; a.W = s.W;
@@ -441,7 +481,7 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
   }
   const int work = a.main_tiles + (tiles - a.main_tiles) * a.tail_splits;
   const int pairs = work < cap ? work : cap;
-  conv3x3_pair_tc_kernel<BN><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
+  conv3x3_pair_tc_kernel<BN><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
   e = cudaGetLastError();
   if (launches) *launches = 1;
   if (e != cudaSuccess || !a.partial) return e;

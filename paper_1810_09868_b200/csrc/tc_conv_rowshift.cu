@@ -235,6 +235,18 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
     const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(group * ACC_STRIDE);
     const bool pool_lane = lane < 16 && (j & 1) == 0 && col_ok;
     uint32_t use = 0;  // tiles this group has taken
+    bool mask_pending = false;  // issuer only: a mask copy is in flight or unread
+    // Input gradient: the group's mask tile (the layer below's output at the tile's pixels) by TMA.  The
+    // issuer requests the NEXT tile's as soon as the whole group has read the current one, so the copy's
+    // latency hides behind the store and the wait for the next accumulator.
+    auto request_mask = [&](int tile) {
+      if (tile >= a.tiles) return;
+      const int tw = tile % a.tiles_w, t = tile / a.tiles_w;
+      mbar_expect_tx(my_mask_bar, OUT_BYTES);
+      tma_load_4d(my_mask, &map_m, my_mask_bar, 0, tw * TW, (t % a.tiles_h) * TH, t / a.tiles_h);
+      mask_pending = true;
+    };
+    if (a.mask && issuer) request_mask(blockIdx.x + group * gridDim.x);
     for (int tile = blockIdx.x + group * gridDim.x; tile < a.tiles; tile += 2 * gridDim.x, ++use) {
       const bool got = mbar_wait(acc_full(group), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
       if (named_bar_or(bar_id, kGroupThreads, !got)) break;  // the group's warps leave together
@@ -247,14 +259,8 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
         if (issuer) tma_store_wait_read<0>();
         named_bar_sync(bar_id, kGroupThreads);
       }
-      if (a.mask) {
-        if (issuer) {
-          mbar_expect_tx(my_mask_bar, OUT_BYTES);
-          tma_load_4d(my_mask, &map_m, my_mask_bar, 0, w0, h0, img);
-        }
-        // a failed wait leaves the tile unmasked; the error word says so
-        mbar_wait(my_mask_bar, use & 1, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
-      }
+      // a failed wait leaves the tile unmasked; the error word says so
+      if (a.mask) mbar_wait(my_mask_bar, use & 1, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
       bf16* pool_row = a.pooled ? a.pooled + (((long)img * (a.H / 2) + (h0 + ph) / 2) * (a.W / 2) + (w0 + j) / 2) * 64
                                 : nullptr;
 #pragma unroll
@@ -324,12 +330,21 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
       mbar_arrive(acc_empty(group));
       if (a.out) {
         fence_async_smem();
-        named_bar_sync(bar_id, kGroupThreads);
+        named_bar_sync(bar_id, kGroupThreads);  // the staging tile is complete, and the group has read its mask tile
         if (issuer) {
           tma_store_4d(&map_y, out_smem + group * OUT_BYTES, 0, w0, h0, img);
           tma_store_commit();
+          if (a.mask) {
+            mask_pending = false;
+            request_mask(tile + 2 * gridDim.x);
+          }
         }
       }
+    }
+    if (issuer && mask_pending) {
+      // left early (a wait ran out) with a mask copy in flight: let it land before shared memory goes away
+      const unsigned long long t0 = global_timer_ns();
+      while (!mbar_try_wait(my_mask_bar, use & 1) && global_timer_ns() - t0 < 100000000ull) {}
     }
     if (issuer) tma_store_wait_all();  // shared memory must outlive the stores that read it
   }
