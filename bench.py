@@ -291,9 +291,9 @@ def time_conv_layers_backward(pkg, net, torch, stream, images, reps=5):
         dw = torch.empty(co * 9 * ci, dtype=torch.float32, device=net.device)
         db = torch.empty(co, dtype=torch.float32, device=net.device)
         mask = None if pooled_input else x  # after a pool the pass masks in the scatter step instead
-        calls = {"wgrad": lambda: pkg.vgg19_conv_layer_backward_ex(net.handle, l + 1, x, dz, BATCH, dw, db, None, None, stream)}
+        calls = {"wgrad": lambda: pkg.vgg19_conv_layer_backward_ex(net.handle, l + 1, x, dz, BATCH, dw, db, None, None, None, stream)}
         if l > 0:
-            calls["dgrad"] = lambda: pkg.vgg19_conv_layer_backward_ex(net.handle, l + 1, None, dz, BATCH, None, None, dx, mask, stream)
+            calls["dgrad"] = lambda: pkg.vgg19_conv_layer_backward_ex(net.handle, l + 1, None, dz, BATCH, None, None, dx, mask, None, stream)
         ms = {}
         for name, fn in calls.items():
             with torch.cuda.stream(stream):

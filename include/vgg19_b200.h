@@ -205,6 +205,15 @@ int vgg19_forward_host_async(vgg19_t *net, const void *host_images, int32_t batc
 int vgg19_conv_layer_forward(vgg19_t *net, int32_t layer, const void *x, int32_t batch,
                              void *y, void *pooled, void *stream);
 
+/* The same, also recording what the backward pass needs to know about the
+ * max-pool (the appendix table's `select-and-scatter`): pool_code (with pooled;
+ * or NULL), device uint8 [batch][h/2][w/2][Cout], receives for every window
+ * where its maximum sits - 0..3 for (0,0), (0,1), (1,0), (1,1), the first one
+ * on ties - or 4 when that maximum is not positive, i.e. when the ReLU before
+ * the pool passes no gradient to the window. */
+int vgg19_conv_layer_forward_ex(vgg19_t *net, int32_t layer, const void *x, int32_t batch, void *y, void *pooled,
+                                uint8_t *pool_code, void *stream);
+
 /* Gradients of that layer given dz = d(loss)/d(pre-activation) already
  * masked by the ReLU: dw fp32 [Cout][3][3][Cin], db fp32 [Cout], and (unless
  * NULL) dx in the config's dtype [batch][h][w][Cin] (section 7.3). */
@@ -217,9 +226,17 @@ int vgg19_conv_layer_backward(vgg19_t *net, int32_t layer, const void *x, const 
  * gradient only; x is then unused and may be NULL), or dx may be NULL (filter
  * and bias gradient only).  relu_mask (or NULL): [batch][h][w][Cin] in the
  * config's dtype, the stored output of the layer below; dx is set to zero
- * wherever relu_mask is not positive. */
+ * wherever relu_mask is not positive.  pool_code (or NULL; excludes
+ * relu_mask): for a layer whose input is a pooled tensor, the codes
+ * vgg19_conv_layer_forward_ex recorded for that pool, [batch][h][w][Cin]; dx
+ * is then the gradient at the output of the layer BELOW the pool,
+ * [batch][2h][2w][Cin]: every value of the input gradient goes to the window
+ * position its code names (nowhere for code 4), zeros elsewhere - pool scatter
+ * and ReLU mask in one, done in the input-gradient kernel's epilogue where the
+ * layer's shape allows. */
 int vgg19_conv_layer_backward_ex(vgg19_t *net, int32_t layer, const void *x, const void *dz, int32_t batch,
-                                 float *dw, float *db, void *dx, const void *relu_mask, void *stream);
+                                 float *dw, float *db, void *dx, const void *relu_mask, const uint8_t *pool_code,
+                                 void *stream);
 
 /* Where a pass at `batch` in `mode` leaves the activations it stores, as a
  * byte offset into the bound workspace, so that a caller can inspect the

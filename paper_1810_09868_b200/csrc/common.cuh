@@ -57,9 +57,17 @@ cudaError_t simt_bias_grad(const T* dz, float* db, float* partial, long P, int C
 template <typename T>
 cudaError_t simt_dense_db(const T* dY, float* db, int M, int Out, cudaStream_t st);
 
-// y = max over 2x2 windows (stride 2) of x, NHWC.
+// y = max over 2x2 windows (stride 2) of x, NHWC.  code (or null), one byte per element of y: where the
+// window's maximum sits, 0..3 in the order (0,0), (0,1), (1,0), (1,1), the first one on ties; 4 when the
+// maximum is not positive (the ReLU that produced x passes no gradient to this window).
 template <typename T>
-cudaError_t simt_maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st);
+cudaError_t simt_maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st, uint8_t* code = nullptr);
+
+// Pool scatter from the stored codes: dy[n][2i + a][2j + b][c] = dp[n][i][j][c] where code = 2a + b,
+// 0 elsewhere (and everywhere for code 4): select-and-scatter fused with the ReLU mask below it,
+// without reading the activation again.  H, W are the full-resolution sizes.
+template <typename T>
+cudaError_t simt_pool_scatter(const uint8_t* code, const T* dp, T* dy, int N, int H, int W, int C, cudaStream_t st);
 
 // dy[pos] = dp[window] where pos is the window's first maximum of y and
 // y[pos] > 0, else 0 (pool scatter fused with the ReLU mask of the layer that

@@ -264,8 +264,8 @@ union Pack8 {
   bf16 h[8];
 };
 
-__global__ void maxpool_fwd_bf16x8_kernel(const bf16* __restrict__ x, bf16* __restrict__ y, long total8, int H, int W,
-                                          int C8) {
+__global__ void maxpool_fwd_bf16x8_kernel(const bf16* __restrict__ x, bf16* __restrict__ y, uint8_t* __restrict__ code,
+                                          long total8, int H, int W, int C8) {
   long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total8) return;
   int Wo = W / 2, Ho = H / 2;
@@ -278,6 +278,50 @@ __global__ void maxpool_fwd_bf16x8_kernel(const bf16* __restrict__ x, bf16* __re
 #pragma unroll
   for (int e = 0; e < 4; ++e) r.h2[e] = __hmax2(__hmax2(a.h2[e], b.h2[e]), __hmax2(c.h2[e], d.h2[e]));
   reinterpret_cast<uint4*>(y)[i] = r.u;
+  if (code) {
+    // where the window's maximum sits (first one in the order (0,0), (0,1), (1,0), (1,1)), or 4 when
+    // it is not positive: all the backward pass needs to know about this window
+    uint32_t w[2] = {0u, 0u};
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float v[4] = {__bfloat162float(a.h[e]), __bfloat162float(b.h[e]), __bfloat162float(c.h[e]),
+                          __bfloat162float(d.h[e])};
+      float m = v[0];
+      uint32_t best = 0;
+#pragma unroll
+      for (int q = 1; q < 4; ++q)
+        if (v[q] > m) { m = v[q]; best = q; }
+      if (!(m > 0.f)) best = 4;
+      w[e >> 2] |= best << (8 * (e & 3));
+    }
+    reinterpret_cast<uint2*>(code)[i] = make_uint2(w[0], w[1]);
+  }
+}
+
+// dy[window position q] = dp[window] where q is the stored arg-max code, else 0 (code 4: nowhere)
+__global__ void pool_scatter_bf16x8_kernel(const uint8_t* __restrict__ code, const bf16* __restrict__ dp,
+                                           bf16* __restrict__ dy, long total8, int H, int W, int C8) {
+  long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total8) return;
+  int Wo = W / 2, Ho = H / 2;
+  int c8 = i % C8; long t = i / C8;
+  int j = t % Wo; t /= Wo;
+  int ii = t % Ho; long n = t / Ho;
+  const long base = ((n * H + 2 * ii) * W + 2 * j) * C8 + c8;
+  const long off[4] = {0, (long)C8, (long)W * C8, (long)W * C8 + C8};
+  Pack8 g, o[4];
+  g.u = __ldg(reinterpret_cast<const uint4*>(dp) + i);
+  const uint2 k = __ldg(reinterpret_cast<const uint2*>(code) + i);
+  const uint32_t kw[2] = {k.x, k.y};
+  const bf16 zero = __float2bfloat16_rn(0.f);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const uint32_t best = (kw[e >> 2] >> (8 * (e & 3))) & 0xFFu;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) o[q].h[e] = (uint32_t)q == best ? g.h[e] : zero;
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(dy)[base + off[q]] = o[q].u;
 }
 
 __global__ void maxpool_bwd_relu_bf16x8_kernel(const bf16* __restrict__ y, const bf16* __restrict__ dp,
@@ -367,7 +411,7 @@ cudaError_t simt_bias_grad(const T* dz, float* db, float* partial, long P, int C
 // ---- pooling ---------------------------------------------------------------
 
 template <typename T>
-__global__ void maxpool_fwd_kernel(const T* x, T* y, long total, int H, int W, int C) {
+__global__ void maxpool_fwd_kernel(const T* x, T* y, uint8_t* code, long total, int H, int W, int C) {
   long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   int Wo = W / 2, Ho = H / 2;
@@ -375,11 +419,30 @@ __global__ void maxpool_fwd_kernel(const T* x, T* y, long total, int H, int W, i
   int j = t % Wo; t /= Wo;
   int ii = t % Ho; long n = t / Ho;
   const T* p = x + ((n * H + 2 * ii) * W + 2 * j) * C + c;
-  float m = to_f32(p[0]);
-  m = fmaxf(m, to_f32(p[C]));
-  m = fmaxf(m, to_f32(p[(long)W * C]));
-  m = fmaxf(m, to_f32(p[(long)W * C + C]));
+  const float v[4] = {to_f32(p[0]), to_f32(p[C]), to_f32(p[(long)W * C]), to_f32(p[(long)W * C + C])};
+  float m = v[0];
+  int best = 0;
+#pragma unroll
+  for (int q = 1; q < 4; ++q)
+    if (v[q] > m) { m = v[q]; best = q; }
   y[i] = from_f32<T>(m);
+  if (code) code[i] = (uint8_t)(m > 0.f ? best : 4);
+}
+
+template <typename T>
+__global__ void pool_scatter_kernel(const uint8_t* code, const T* dp, T* dy, long total, int H, int W, int C) {
+  long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  int Wo = W / 2, Ho = H / 2;
+  int c = i % C; long t = i / C;
+  int j = t % Wo; t /= Wo;
+  int ii = t % Ho; long n = t / Ho;
+  long base = ((n * H + 2 * ii) * W + 2 * j) * C + c;
+  long off[4] = {0, (long)C, (long)W * C, (long)W * C + C};
+  const int best = code[i];
+  const T g = dp[i];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) dy[base + off[q]] = (q == best) ? g : from_f32<T>(0.f);
 }
 
 template <typename T>
@@ -405,14 +468,26 @@ __global__ void maxpool_bwd_relu_kernel(const T* y, const T* dp, T* dy, long tot
 }
 
 template <typename T>
-cudaError_t simt_maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st) {
+cudaError_t simt_maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st, uint8_t* code) {
   long total = (long)N * (H / 2) * (W / 2) * C;
   if (std::is_same<T, bf16>::value && C % 8 == 0) {
-    maxpool_fwd_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>((const bf16*)x, (bf16*)y, total / 8, H,
-                                                                                 W, C / 8);
+    maxpool_fwd_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>((const bf16*)x, (bf16*)y, code,
+                                                                                 total / 8, H, W, C / 8);
     return cudaGetLastError();
   }
-  maxpool_fwd_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(x, y, total, H, W, C);
+  maxpool_fwd_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(x, y, code, total, H, W, C);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t simt_pool_scatter(const uint8_t* code, const T* dp, T* dy, int N, int H, int W, int C, cudaStream_t st) {
+  long total = (long)N * (H / 2) * (W / 2) * C;
+  if (std::is_same<T, bf16>::value && C % 8 == 0) {
+    pool_scatter_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>(code, (const bf16*)dp, (bf16*)dy,
+                                                                                  total / 8, H, W, C / 8);
+    return cudaGetLastError();
+  }
+  pool_scatter_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(code, dp, dy, total, H, W, C);
   return cudaGetLastError();
 }
 
@@ -660,7 +735,9 @@ cudaError_t refresh_filter_copies(const float* params, bf16* dgrad_w, bf16* tap_
                                        bool, cudaStream_t);                                          \
   template cudaError_t simt_conv3x3_wgrad<T>(const T*, const T*, float*, float*, float*, ConvShape,  \
                                              cudaStream_t);                                          \
-  template cudaError_t simt_maxpool_fwd<T>(const T*, T*, int, int, int, int, cudaStream_t);          \
+  template cudaError_t simt_maxpool_fwd<T>(const T*, T*, int, int, int, int, cudaStream_t, uint8_t*); \
+  template cudaError_t simt_pool_scatter<T>(const uint8_t*, const T*, T*, int, int, int, int,        \
+                                            cudaStream_t);                                           \
   template cudaError_t simt_maxpool_bwd_relu<T>(const T*, const T*, T*, int, int, int, int,          \
                                                 cudaStream_t);                                       \
   template cudaError_t simt_dense_nt<T>(const T*, const T*, const float*, const T*, T*, float*, int, \

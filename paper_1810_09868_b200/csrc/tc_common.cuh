@@ -211,6 +211,61 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t addr, uint32_t (&v)[16]) 
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- 2x2 max-pool in an epilogue ----------------------------------------------
+// The four values of a window sit in four lanes: this one (top left), lane + dx (its right neighbour),
+// lane + dy (below), lane + dx + dy.  v[] holds WORDS bf16 pairs (2 * WORDS channels) of this lane's pixel
+// and comes back as the window's maxima (meaningful in the top-left lane).
+template <int WORDS>
+__device__ __forceinline__ void pool2x2(uint32_t (&v)[WORDS], int dx, int dy) {
+#pragma unroll
+  for (int i = 0; i < WORDS; ++i) {
+    __nv_bfloat162 m = *reinterpret_cast<__nv_bfloat162*>(&v[i]);
+    uint32_t o = __shfl_down_sync(0xffffffffu, v[i], dx);
+    m = __hmax2(m, *reinterpret_cast<__nv_bfloat162*>(&o));
+    uint32_t mb = *reinterpret_cast<uint32_t*>(&m);
+    o = __shfl_down_sync(0xffffffffu, mb, dy);
+    m = __hmax2(m, *reinterpret_cast<__nv_bfloat162*>(&o));
+    v[i] = *reinterpret_cast<uint32_t*>(&m);
+  }
+}
+// The same, also giving each channel's arg-max code, one byte per channel in codes[] (four channels per
+// word): 0..3 for the window positions (0,0), (0,1), (1,0), (1,1), the first maximum in that order on
+// ties, or 4 when the maximum is not positive.  All comparisons are two channels at a time; the lower
+// row's left-or-right decisions come up as one word of flag bits (WORDS <= 16).
+template <int WORDS>
+__device__ __forceinline__ void pool2x2_codes(uint32_t (&v)[WORDS], int dx, int dy, uint32_t (&codes)[WORDS / 2]) {
+  static_assert(WORDS <= 16 && WORDS % 2 == 0, "flag bits i and 16 + i per word");
+  uint32_t left[WORDS];  // per half 0xFFFF where the left value of this lane's row is >= the right one
+  uint32_t flags = 0;
+#pragma unroll
+  for (int i = 0; i < WORDS; ++i) {
+    const uint32_t right = __shfl_down_sync(0xffffffffu, v[i], dx);
+    const __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&v[i]), b = *reinterpret_cast<const __nv_bfloat162*>(&right);
+    left[i] = __hge2_mask(a, b);
+    const __nv_bfloat162 m = __hmax2(a, b);
+    v[i] = *reinterpret_cast<const uint32_t*>(&m);
+    flags |= (left[i] & 0x00010001u) << i;
+  }
+  const uint32_t flags_below = __shfl_down_sync(0xffffffffu, flags, dy);
+  const uint32_t zero2 = 0u;
+  uint32_t k16[WORDS];  // the code of each channel in its 16-bit half
+#pragma unroll
+  for (int i = 0; i < WORDS; ++i) {
+    const uint32_t below = __shfl_down_sync(0xffffffffu, v[i], dy);
+    const __nv_bfloat162 t = *reinterpret_cast<__nv_bfloat162*>(&v[i]), b = *reinterpret_cast<const __nv_bfloat162*>(&below);
+    const uint32_t top = __hge2_mask(t, b);  // the upper row holds the (first) maximum
+    const __nv_bfloat162 m = __hmax2(t, b);
+    v[i] = *reinterpret_cast<const uint32_t*>(&m);
+    const uint32_t left_below = ((flags_below >> i) & 0x00010001u) * 0xFFFFu;
+    const uint32_t is_left = (top & left[i]) | (~top & left_below);
+    uint32_t k = (~top & 0x00020002u) | (~is_left & 0x00010001u);
+    const uint32_t positive = __hgt2_mask(m, *reinterpret_cast<const __nv_bfloat162*>(&zero2));
+    k16[i] = (k & positive) | (~positive & 0x00040004u);
+  }
+#pragma unroll
+  for (int j = 0; j < WORDS / 2; ++j) codes[j] = __byte_perm(k16[2 * j], k16[2 * j + 1], 0x6420);
+}
+
 // ---- CTA pairs (cluster of two, tcgen05 cta_group::2) --------------------------
 // One MMA spans both CTAs of the pair: each supplies its own 128 rows of A and half of the B tile
 // from its own shared memory and holds its 128 accumulator rows in its own tensor memory.  The even
@@ -393,6 +448,10 @@ bool make_tiled_map_2d_c8(CUtensorMap* map, const void* base, uint64_t rows, uin
 bool make_filter_row_map(CUtensorMap* map, const void* base, int Cout, int Cin, uint32_t box_cout);
 // NHWC bf16 tensor, tiled box of box_h x box_w pixels x 64 channels, 128 B swizzle.
 bool make_patch_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, uint32_t box_w, uint32_t box_h);
+// One of the four 2x2 window positions (a, b) of an NHWC bf16 tensor [N][H][W][C] as a tensor of its
+// own: [N][H/2][W/2][C] whose pixel (h, w) is pixel (2h + a, 2w + b) of the tensor; box as above.
+bool make_window_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, int a, int b, uint32_t box_w,
+                     uint32_t box_h);
 // NHWC bf16 tensor read through a 3x3 / pad 1 window: box = `pixels` x 64 channels, 128 B swizzle.
 bool make_im2col_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, uint32_t pixels);
 // NHWC bf16 tensor with 8 channels, tiled box of box_h x box_w pixels x 8 channels, no swizzle.

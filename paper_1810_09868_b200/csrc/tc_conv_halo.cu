@@ -67,13 +67,22 @@ struct HaloArgs {
   const bf16* mask;
   bf16* out;     // full-resolution output, or null when only the pooled output is wanted
   bf16* pooled;  // 2x2 max-pooled output [N][H/2][W/2][Cout], or null
+  uint8_t* code; // with pooled: arg-max code of every window (see simt_maxpool_fwd), or null
+  // Pool scatter (input gradient of a layer whose input is a pooled tensor): each 64-channel chunk of the
+  // tile is stored four times, once per window position, into the full-resolution gradient of the layer
+  // below the pool, keeping a value only at the position its window's stored code names.
+  const uint8_t* scatter_code;  // [N][H][W][Cout] at this kernel's resolution, or null
   int* dev_error;
 };
 
-template <int BN, bool PAIR>
+// MODE 0: plain (output, mask, pooled output); 1: pooled output with arg-max codes; 2: pool scatter.
+// Compile-time so that the plain kernel carries none of the other two's registers and instructions.
+template <int BN, bool PAIR, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_m,
+                       const __grid_constant__ CUtensorMap map_s0, const __grid_constant__ CUtensorMap map_s1,
+                       const __grid_constant__ CUtensorMap map_s2, const __grid_constant__ CUtensorMap map_s3,
                        HaloArgs a) {
   using T = HaloTile<BN, PAIR>;
   constexpr int NA = kMaxPatchSlots, NB = 4;  // most slots a plan may use (barrier numbering)
@@ -330,12 +339,26 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       const bool pool_lane = (lane & 1) == 0 && (lane & 8) == 0;
       bf16* pool_row = a.pooled ? a.pooled + (((long)img * (a.H / 2) + h / 2) * (a.W / 2) + w / 2) * a.Cout + c_base
                                 : nullptr;
+      uint8_t* code_row = (MODE == 1 && a.code) ? a.code + (((long)img * (a.H / 2) + h / 2) * (a.W / 2) + w / 2) * a.Cout + c_base : nullptr;
+      const uint8_t* scode_row = (MODE == 2 && h < a.H) ? a.scatter_code + (((long)img * a.H + h) * a.W + w) * a.Cout + c_base
+                                                             : nullptr;
 #pragma unroll 1
       for (int c64 = 0; c64 < BN; c64 += 64) {
         if (a.out) {
           if (issuer) tma_store_wait_read<1>();  // the store before last, which used this staging tile, has read it
           named_bar_sync(1, 128);
         }
+        // pool scatter: this pixel's 64 code bytes, requested before the tensor-memory loads
+        uint4 sc[4];
+        if (MODE != 2) {
+        } else if (scode_row) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) sc[q] = __ldg(reinterpret_cast<const uint4*>(scode_row + c64) + q);
+        } else {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) sc[q] = make_uint4(0x04040404u, 0x04040404u, 0x04040404u, 0x04040404u);
+        }
+        uint32_t kept[32];  // pool scatter: the chunk's values (bf16 pairs) of this pixel
         bool mask_ready = false;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -372,6 +395,10 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
               }
             }
           }
+          if (MODE == 2) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) kept[half * 16 + i] = packed[i];
+          }
           if (a.out) {
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -381,21 +408,20 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             }
           }
           if (a.pooled) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              __nv_bfloat162 m = *reinterpret_cast<__nv_bfloat162*>(&packed[i]);
-              uint32_t o = __shfl_down_sync(0xffffffffu, packed[i], 1);
-              m = __hmax2(m, *reinterpret_cast<__nv_bfloat162*>(&o));
-              uint32_t mb = *reinterpret_cast<uint32_t*>(&m);
-              o = __shfl_down_sync(0xffffffffu, mb, 8);
-              m = __hmax2(m, *reinterpret_cast<__nv_bfloat162*>(&o));
-              packed[i] = *reinterpret_cast<uint32_t*>(&m);
-            }
+            // 2x2 window: columns w, w + 1 (next lane) of rows h, h + 1 (8 lanes on)
+            uint32_t codes[8];
+            if (MODE == 1) pool2x2_codes<16>(packed, 1, 8, codes);
+            else pool2x2<16>(packed, 1, 8);
             if (pool_lane) {
               uint4* pp = reinterpret_cast<uint4*>(pool_row + cc);
 #pragma unroll
               for (int q = 0; q < 4; ++q)
                 pp[q] = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+              if (code_row) {
+                uint4* kp = reinterpret_cast<uint4*>(code_row + cc);
+                kp[0] = make_uint4(codes[0], codes[1], codes[2], codes[3]);
+                kp[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
+              }
             }
           }
         }
@@ -411,6 +437,43 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             }
           }
           stage_sel ^= 1;
+        }
+        if (MODE == 2) {
+          // four rounds through the two staging tiles in turn, one per window position q = 2a + b: the value
+          // where the window's code names q, zero elsewhere; the store's tensor map addresses pixel
+          // (2h + a, 2w + b) of the full-resolution gradient for patch coordinate (h, w)
+          const uint32_t kw[16] = {sc[0].x, sc[0].y, sc[0].z, sc[0].w, sc[1].x, sc[1].y, sc[1].z, sc[1].w,
+                                   sc[2].x, sc[2].y, sc[2].z, sc[2].w, sc[3].x, sc[3].y, sc[3].z, sc[3].w};
+#pragma unroll 1
+          for (uint32_t q = 0; q < 4; ++q) {
+            if (issuer) tma_store_wait_read<1>();  // the store before last, which used this staging tile, has read it
+            named_bar_sync(1, 128);
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {  // 16-byte chunks: 8 channels, 8 code bytes (two words)
+              uint32_t o[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t k2 = kw[ch * 2 + (e >> 1)] >> (16 * (e & 1));  // codes of channels 2e, 2e + 1 of the chunk
+                uint32_t keep = 0;
+                if ((k2 & 0xFFu) == q) keep |= 0x0000FFFFu;
+                if (((k2 >> 8) & 0xFFu) == q) keep |= 0xFFFF0000u;
+                o[e] = kept[ch * 4 + e] & keep;
+              }
+              *reinterpret_cast<uint4*>(stage_row0 + stage_sel * T::OUT_BYTES + ((ch ^ (row & 7)) << 4)) =
+                  make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            fence_async_smem();
+            named_bar_sync(1, 128);
+            if (issuer) {
+              const uint32_t src = out_smem + stage_sel * T::OUT_BYTES;
+              if (q == 0) tma_store_4d(&map_s0, src, c_base + c64, tw * PW, th * PH, img);
+              else if (q == 1) tma_store_4d(&map_s1, src, c_base + c64, tw * PW, th * PH, img);
+              else if (q == 2) tma_store_4d(&map_s2, src, c_base + c64, tw * PW, th * PH, img);
+              else tma_store_4d(&map_s3, src, c_base + c64, tw * PW, th * PH, img);
+              tma_store_commit();
+            }
+            stage_sel ^= 1;
+          }
         }
       }
       tc_fence_before();
@@ -443,9 +506,9 @@ conv3x3_halo_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   }
 }
 
-template <int BN, bool PAIR>
+template <int BN, bool PAIR, int MODE>
 cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const CUtensorMap& mm,
-                        HaloArgs a, cudaStream_t st) {
+                        const CUtensorMap* ms, HaloArgs a, cudaStream_t st) {
   using T = HaloTile<BN, PAIR>;
   // plan the shared memory: keep the whole filter resident when it fits beside two or three patch slots
   // (then only the input patches cross the L2-to-SM path, which is what bounds these layers), else
@@ -470,7 +533,7 @@ cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
   const int smem = a.na * A_SLOT + a.b_region_bytes + fixed;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_halo_tc_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::kLimit);
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_halo_tc_kernel<BN, PAIR, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::kLimit);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -489,10 +552,10 @@ cudaError_t launch_halo(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, conv3x3_halo_tc_kernel<BN, PAIR>, mx, mw, my, mm, a);
+    return cudaLaunchKernelEx(&cfg, conv3x3_halo_tc_kernel<BN, PAIR, MODE>, mx, mw, my, mm, ms[0], ms[1], ms[2], ms[3], a);
   }
   const int tiles = a.m_tiles * a.n_tiles;
-  conv3x3_halo_tc_kernel<BN, PAIR><<<tiles < sms ? tiles : sms, kThreads, smem, st>>>(mx, mw, my, mm, a);
+  conv3x3_halo_tc_kernel<BN, PAIR, MODE><<<tiles < sms ? tiles : sms, kThreads, smem, st>>>(mx, mw, my, mm, ms[0], ms[1], ms[2], ms[3], a);
   return cudaGetLastError();
 }
 
@@ -536,8 +599,11 @@ bool tc_conv3x3_halo_supported_unpooled(ConvShape s) {
 }
 
 cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
-                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, bool pairs) {
-  if (!out && !pooled) return cudaErrorInvalidValue;
+                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, bool pairs, uint8_t* code,
+                            const uint8_t* scatter_code, bf16* scatter_out) {
+  if (!out && !pooled && !scatter_out) return cudaErrorInvalidValue;
+  if ((scatter_code == nullptr) != (scatter_out == nullptr) || (scatter_out && (out || pooled || mask))) return cudaErrorInvalidValue;
+  if (code && !pooled) return cudaErrorInvalidValue;
   if (!(pooled ? tc_conv3x3_halo_supported(s) : tc_conv3x3_halo_supported_unpooled(s))) return cudaErrorInvalidValue;
   const int BN = s.Cout % 128 == 0 ? 128 : 64;
   // CTA pairs take two tiles at a time.  They pay with 128 output channels, where one CTA's MMAs are
@@ -551,15 +617,26 @@ cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const floa
   CUtensorMap mm = mw;  // only read when there is a mask
   if (mask && !make_patch_map(&mm, mask, s.N, s.H, s.W, s.Cout, PW, PH)) return cudaErrorInvalidValue;
   if (mask && !out) return cudaErrorInvalidValue;
+  // pool scatter: four views of the full-resolution gradient [N][2H][2W][Cout], one per window position
+  CUtensorMap ms[4] = {mw, mw, mw, mw};
+  if (scatter_out)
+    for (int q = 0; q < 4; ++q)
+      if (!make_window_map(&ms[q], scatter_out, s.N, 2 * s.H, 2 * s.W, s.Cout, q >> 1, q & 1, PW, PH)) return cudaErrorInvalidValue;
   HaloArgs a;
+  a.code = code; a.scatter_code = scatter_code;
   a.N = s.N; a.H = s.H; a.W = s.W;
   a.cin_blocks = s.Cin / 64; a.Cin = s.Cin; a.Cout = s.Cout;
   a.tiles_w = s.W / PW; a.tiles_h = (s.H + PH - 1) / PH;
   a.m_tiles = s.N * a.tiles_w * a.tiles_h;
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0; a.bias = bias; a.mask = mask; a.out = out; a.pooled = pooled; a.dev_error = dev_error;
-  if (pair) return launch_halo<128, true>(mx, mw, my, mm, a, st);
-  return BN == 128 ? launch_halo<128, false>(mx, mw, my, mm, a, st) : launch_halo<64, false>(mx, mw, my, mm, a, st);
+  const int mode = scatter_out ? 2 : (code ? 1 : 0);
+#define HALO_LAUNCH(MODE)                                                                      \
+  (pair ? launch_halo<128, true, MODE>(mx, mw, my, mm, ms, a, st)                              \
+        : (BN == 128 ? launch_halo<128, false, MODE>(mx, mw, my, mm, ms, a, st)                \
+                     : launch_halo<64, false, MODE>(mx, mw, my, mm, ms, a, st)))
+  return mode == 2 ? HALO_LAUNCH(2) : (mode == 1 ? HALO_LAUNCH(1) : HALO_LAUNCH(0));
+#undef HALO_LAUNCH
 }
 
 }  // namespace vgg

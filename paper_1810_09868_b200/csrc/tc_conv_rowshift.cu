@@ -56,12 +56,22 @@ struct RowArgs {
   const bf16* mask;
   bf16* out;     // full-resolution output or null
   bf16* pooled;  // 2x2 max-pooled output or null
+  uint8_t* code; // with pooled: arg-max code of every window (see simt_maxpool_fwd), or null
+  // Pool scatter (input gradient of a layer whose input is a pooled tensor): instead of storing the tile,
+  // store it four times, once per window position, into the full-resolution gradient of the layer below
+  // the pool, keeping a value only at the position its window's stored code names.
+  const uint8_t* scatter_code;  // [N][H][W][64] at this kernel's resolution, or null
   int* dev_error;
 };
 
+// MODE 0: plain (output, mask, pooled output); 1: pooled output with arg-max codes; 2: pool scatter.
+// Compile-time so that the plain kernel carries none of the other two's registers and instructions.
+template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                            const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_m,
+                           const __grid_constant__ CUtensorMap map_s0, const __grid_constant__ CUtensorMap map_s1,
+                           const __grid_constant__ CUtensorMap map_s2, const __grid_constant__ CUtensorMap map_s3,
                            RowArgs a) {
   constexpr int NA = kMaxPatchSlots, NB = kMaxFilterSlots;
   extern __shared__ uint8_t smem_raw[];
@@ -263,6 +273,15 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
       if (a.mask) mbar_wait(my_mask_bar, use & 1, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
       bf16* pool_row = a.pooled ? a.pooled + (((long)img * (a.H / 2) + (h0 + ph) / 2) * (a.W / 2) + (w0 + j) / 2) * 64
                                 : nullptr;
+      uint8_t* code_row = (MODE == 1 && a.code) ? a.code + (((long)img * (a.H / 2) + (h0 + ph) / 2) * (a.W / 2) + (w0 + j) / 2) * 64
+                                 : nullptr;
+      // pool scatter: this thread's 32 code bytes, requested before the tensor-memory loads
+      uint4 sc[2];
+      if (MODE == 2 && col_ok) {
+        const uint4* cp = reinterpret_cast<const uint4*>(a.scatter_code + (((long)img * a.H + h0 + ph) * a.W + w0 + j) * 64 + c_first);
+        sc[0] = __ldg(cp); sc[1] = __ldg(cp + 1);
+      }
+      uint32_t kept[16];  // pool scatter: the tile's values (bf16 pairs) of this thread's 32 channels
 #pragma unroll
       for (int c16 = c_first; c16 < c_first + 32; c16 += 16) {
         uint32_t v0[16], v1[16], v2[16];
@@ -300,6 +319,10 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
             }
           }
         }
+        if (MODE == 2) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) kept[((c16 - c_first) >> 1) + i] = packed[i];
+        }
         if (a.out && col_ok) {
 #pragma unroll
           for (int q = 0; q < 2; ++q)
@@ -308,20 +331,14 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
         }
         if (a.pooled) {
           // 2x2 window: columns j, j + 1 (next lane) of rows ph, ph + 1 (16 lanes on)
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            __nv_bfloat162 m = *reinterpret_cast<__nv_bfloat162*>(&packed[i]);
-            uint32_t o = __shfl_down_sync(0xffffffffu, packed[i], 1);
-            m = __hmax2(m, *reinterpret_cast<__nv_bfloat162*>(&o));
-            uint32_t mb = *reinterpret_cast<uint32_t*>(&m);
-            o = __shfl_down_sync(0xffffffffu, mb, 16);
-            m = __hmax2(m, *reinterpret_cast<__nv_bfloat162*>(&o));
-            packed[i] = *reinterpret_cast<uint32_t*>(&m);
-          }
+          uint32_t codes[4];
+          if (MODE == 1) pool2x2_codes<8>(packed, 1, 16, codes);
+          else pool2x2<8>(packed, 1, 16);
           if (pool_lane) {
             uint4* pp = reinterpret_cast<uint4*>(pool_row + c16);
             pp[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
             pp[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+            if (code_row) *reinterpret_cast<uint4*>(code_row + c16) = make_uint4(codes[0], codes[1], codes[2], codes[3]);
           }
         }
       }
@@ -337,6 +354,42 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
           if (a.mask) {
             mask_pending = false;
             request_mask(tile + 2 * gridDim.x);
+          }
+        }
+      }
+      if (MODE == 2) {
+        // four rounds through the group's staging tile, one per window position q = 2a + b: the value where
+        // the window's code names q, zero elsewhere; the store's tensor map addresses pixel (2h + a, 2w + b)
+        // of the full-resolution gradient for tile coordinate (h, w)
+        const uint32_t kw[8] = {sc[0].x, sc[0].y, sc[0].z, sc[0].w, sc[1].x, sc[1].y, sc[1].z, sc[1].w};
+#pragma unroll 1
+        for (uint32_t q = 0; q < 4; ++q) {
+          if (issuer) tma_store_wait_read<0>();  // the previous round's store has read the staging tile
+          named_bar_sync(bar_id, kGroupThreads);
+          if (col_ok) {
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {  // 16-byte chunks: 8 channels, 8 code bytes (two words)
+              uint32_t o[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t k2 = kw[ch * 2 + (e >> 1)] >> (16 * (e & 1));  // the codes of channels 2e, 2e + 1 of this chunk
+                uint32_t keep = 0;
+                if ((k2 & 0xFFu) == q) keep |= 0x0000FFFFu;
+                if (((k2 >> 8) & 0xFFu) == q) keep |= 0xFFFF0000u;
+                o[e] = kept[ch * 4 + e] & keep;
+              }
+              *reinterpret_cast<uint4*>(stage_row + ((((c_first >> 3) + ch) ^ (rr & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+          }
+          fence_async_smem();
+          named_bar_sync(bar_id, kGroupThreads);
+          if (issuer) {
+            const uint32_t src = out_smem + group * OUT_BYTES;
+            if (q == 0) tma_store_4d(&map_s0, src, 0, w0, h0, img);
+            else if (q == 1) tma_store_4d(&map_s1, src, 0, w0, h0, img);
+            else if (q == 2) tma_store_4d(&map_s2, src, 0, w0, h0, img);
+            else tma_store_4d(&map_s3, src, 0, w0, h0, img);
+            tma_store_commit();
           }
         }
       }
@@ -366,9 +419,12 @@ bool tc_conv3x3_rowshift_supported(ConvShape s) {
 }
 
 cudaError_t tc_conv3x3_rowshift(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
-                                bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st) {
-  if (!out && !pooled) return cudaErrorInvalidValue;
+                                bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, uint8_t* code,
+                                const uint8_t* scatter_code, bf16* scatter_out) {
+  if (!out && !pooled && !scatter_out) return cudaErrorInvalidValue;
   if (mask && !out) return cudaErrorInvalidValue;
+  if ((scatter_code == nullptr) != (scatter_out == nullptr) || (scatter_out && (out || pooled || mask))) return cudaErrorInvalidValue;
+  if (code && !pooled) return cudaErrorInvalidValue;
   if (!tc_conv3x3_rowshift_supported(s)) return cudaErrorInvalidValue;
   CUtensorMap mx, mw;
   if (!make_patch_map(&mx, in, s.N, s.H, s.W, s.Cin, AW, IH)) return cudaErrorInvalidValue;
@@ -377,7 +433,14 @@ cudaError_t tc_conv3x3_rowshift(const bf16* in, const bf16* wt_tap_major, const 
   if (out && !make_patch_map(&my, out, s.N, s.H, s.W, s.Cout, TW, TH)) return cudaErrorInvalidValue;
   CUtensorMap mm = mw;  // only read when there is a mask
   if (mask && !make_patch_map(&mm, mask, s.N, s.H, s.W, s.Cout, TW, TH)) return cudaErrorInvalidValue;
+  // pool scatter: four views of the full-resolution gradient [N][2H][2W][64], one per window position
+  // (a, b): pixel (h, w) of the view is pixel (2h + a, 2w + b) of the tensor
+  CUtensorMap ms[4] = {mw, mw, mw, mw};
+  if (scatter_out)
+    for (int q = 0; q < 4; ++q)
+      if (!make_window_map(&ms[q], scatter_out, s.N, 2 * s.H, 2 * s.W, s.Cout, q >> 1, q & 1, TW, TH)) return cudaErrorInvalidValue;
   RowArgs a;
+  a.code = code; a.scatter_code = scatter_code;
   a.N = s.N; a.H = s.H; a.W = s.W;
   a.cin_blocks = s.Cin / 64;
   a.tiles_w = s.W / TW; a.tiles_h = s.H / TH;
@@ -401,14 +464,19 @@ cudaError_t tc_conv3x3_rowshift(const bf16* in, const bf16* wt_tap_major, const 
   const int smem = a.na * A_BYTES + a.b_region_bytes + fixed;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_rowshift_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLimit);
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_rowshift_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_rowshift_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_rowshift_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLimit);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  conv3x3_rowshift_tc_kernel<<<a.tiles < sms ? a.tiles : sms, kThreads, smem, st>>>(mx, mw, my, mm, a);
+  const int grid = a.tiles < sms ? a.tiles : sms;
+  if (scatter_out) conv3x3_rowshift_tc_kernel<2><<<grid, kThreads, smem, st>>>(mx, mw, my, mm, ms[0], ms[1], ms[2], ms[3], a);
+  else if (code) conv3x3_rowshift_tc_kernel<1><<<grid, kThreads, smem, st>>>(mx, mw, my, mm, ms[0], ms[1], ms[2], ms[3], a);
+  else conv3x3_rowshift_tc_kernel<0><<<grid, kThreads, smem, st>>>(mx, mw, my, mm, ms[0], ms[1], ms[2], ms[3], a);
   return cudaGetLastError();
 }
 

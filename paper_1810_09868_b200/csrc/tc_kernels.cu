@@ -96,6 +96,20 @@ bool make_patch_map(CUtensorMap* map, const void* base, int N, int H, int W, int
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_window_map(CUtensorMap* map, const void* base, int N, int H, int W, int C, int a, int b, uint32_t box_w,
+                     uint32_t box_h) {
+  const TensorMapApi& api = tensor_map_api();
+  if (!api.ok || (H & 1) || (W & 1)) return false;
+  const char* first = static_cast<const char*>(base) + ((size_t)a * W + b) * C * 2;
+  cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W / 2, (cuuint64_t)H / 2, (cuuint64_t)N};
+  cuuint64_t strides[3] = {(cuuint64_t)2 * C * 2, (cuuint64_t)2 * W * C * 2, (cuuint64_t)H * W * C * 2};
+  cuuint32_t box[4] = {64, box_w, box_h, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return api.encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<char*>(first), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_filter_row_map(CUtensorMap* map, const void* base, int Cout, int Cin, uint32_t box_cout) {
   const TensorMapApi& api = tensor_map_api();
   if (!api.ok) return false;

@@ -39,15 +39,22 @@ bool tc_conv3x3_halo_supported_unpooled(ConvShape s);  // shapes it takes when n
 cudaError_t tc_make_tap_major(const float* w, bf16* out, int Cin, int Cout, bool for_dgrad, cudaStream_t st);
 // pairs: work as CTA pairs (two tiles at a time, each CTA staging half of the filter's output channels)
 // when the tile count is even.
+// code (with pooled, or null): the arg-max code of every pooling window, as simt_maxpool_fwd writes it.
+// scatter_code + scatter_out (input gradient of a layer that reads a pooled tensor; out, pooled and mask
+// null): the result is not stored at its own resolution but scattered through the pool into
+// scatter_out [N][2H][2W][Cout], each value to the window position its code names (none for code 4) and
+// zeros to the other three: select-and-scatter and the ReLU mask below it, fused into this epilogue.
 cudaError_t tc_conv3x3_halo(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
-                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, bool pairs = true);
+                            bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st, bool pairs = true,
+                            uint8_t* code = nullptr, const uint8_t* scatter_code = nullptr, bf16* scatter_out = nullptr);
 
 // The same convolution for 64 output channels (tc_conv_rowshift.cu): the three taps of a filter row
 // share one 128 x 192 x 16 MMA, and the epilogue adds the three column-shifted partial sums.  Same
 // arguments as tc_conv3x3_halo; W must be a multiple of 14 and H of 8.
 bool tc_conv3x3_rowshift_supported(ConvShape s);
 cudaError_t tc_conv3x3_rowshift(const bf16* in, const bf16* wt_tap_major, const float* bias, const bf16* mask, bf16* out,
-                                bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
+                                bf16* pooled, ConvShape s, bool relu, int* dev_error, cudaStream_t st,
+                                uint8_t* code = nullptr, const uint8_t* scatter_code = nullptr, bf16* scatter_out = nullptr);
 
 // Filter gradient of the same convolution as a GEMM with M = Cout, N = 9*Cin,
 // K = pixels (both operands read transposed, x through the im2col window):

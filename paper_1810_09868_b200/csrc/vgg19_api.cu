@@ -110,6 +110,7 @@ int fail(vgg19 *n, int code, const char *fmt, ...) {
 struct Plan {
   size_t act[kConvLayers];  // y_l = relu(conv_l + b): [B][H][W][Cout]
   size_t pooled[5];         // outputs of the five pools
+  size_t code[5];           // backward: one byte per pooled element, where its window's maximum sits
   size_t a1, a2;            // dense activations [B][4096]
   size_t logits, probs;     // fp32 [B][1000] (used when the caller passes none)
   size_t dl, dz2, dz1, dflat;  // backward: dlogits, dense pre-activation grads, d(flatten)
@@ -174,6 +175,8 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
   const bool train = mode == VGG19_MODE_TRAIN;
   if (train) mode = VGG19_MODE_BACKWARD;
   if (mode == VGG19_MODE_BACKWARD) {
+    for (int l = 0, k = 0; l < kConvLayers; ++l)
+      if (n->conv[l].pool_after) p.code[k++] = take((size_t)B * (n->conv[l].H / 2) * (n->conv[l].W / 2) * n->conv[l].Cout);
     p.dl = take((size_t)B * kClasses * n->elt);
     p.dz2 = take((size_t)B * 4096 * n->elt);
     p.dz1 = take((size_t)B * 4096 * n->elt);
@@ -241,7 +244,8 @@ struct Pass {
 
   // y = relu(conv(x) + b), optionally pooled.  With need_y false the full-resolution output may be
   // left unwritten when the pool is fused into the convolution's epilogue.
-  void conv_forward(int l, const T *x, int B, T *y, T *pooled, bool need_y = true) {
+  // code (with pooled, or null): receives the arg-max code of every pooling window for the backward pass.
+  void conv_forward(int l, const T *x, int B, T *y, T *pooled, bool need_y = true, uint8_t *code = nullptr) {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
     if (first_tc_ok(l, s)) {
@@ -249,11 +253,13 @@ struct Pass {
       ok(tc_first_conv((const bf16 *)buf(p.x8), n->w8, n->params + c.b_off, (bf16 *)y, s, true, n->dev_error, st), 1);
     } else if (n->use_tc && tc_conv3x3_rowshift_supported(s)) {
       ok(tc_conv3x3_rowshift((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
-                             (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st), 1);
+                             (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st,
+                             pooled ? code : nullptr), 1);
       return;
     } else if (n->use_tc && tc_conv3x3_halo_supported(s)) {
       ok(tc_conv3x3_halo((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
-                         (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st, n->use_pair), 1);
+                         (need_y || !pooled) ? (bf16 *)y : nullptr, (bf16 *)pooled, s, true, n->dev_error, st, n->use_pair,
+                         pooled ? code : nullptr), 1);
       return;
     } else if (pair_ok(s)) {
       int k = 1;
@@ -265,12 +271,15 @@ struct Pass {
                     (bf16 *)y, s, true, n->dev_error, st), 1);
     else
       ok(simt_conv3x3<T>(x, wt(c.w_off), n->params + c.b_off, nullptr, y, s, true, st), 1);
-    if (pooled) ok(simt_maxpool_fwd<T>(y, pooled, B, c.H, c.W, c.Cout, st), 1);
+    if (pooled) ok(simt_maxpool_fwd<T>(y, pooled, B, c.H, c.W, c.Cout, st, code), 1);
   }
 
-  // dW, db from (x, dz); dx = dgrad(dz) [* (mask > 0)] unless dx is null
+  // dW, db from (x, dz); dx = dgrad(dz) [* (mask > 0)] unless dx is null.  With code and dx_full (the
+  // layer's input is a pooled tensor): dx_full [B][2H][2W][Cin] = dgrad(dz) scattered through the pool by
+  // the stored arg-max codes, in the input-gradient kernel's own epilogue where that kernel can, else
+  // by way of dx (then scratch for the pooled-resolution gradient) and a scatter kernel.
   void conv_backward(int l, const T *x, const T *dz, int B, float *dW, float *db, T *dx,
-                     const T *mask) {
+                     const T *mask, const uint8_t *code = nullptr, T *dx_full = nullptr) {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
     if (!dW) {
@@ -288,6 +297,15 @@ struct Pass {
     if (dx) {
       ConvShape t{B, c.H, c.W, c.Cout, c.Cin};  // a 3x3 correlation from Cout to Cin channels
       const T *wr = static_cast<const T *>(n->dgrad_w) + c.dgrad_off;
+      if (code && n->use_tc && tc_conv3x3_rowshift_supported(t)) {
+        ok(tc_conv3x3_rowshift((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, nullptr, nullptr, nullptr, t, false,
+                               n->dev_error, st, nullptr, code, (bf16 *)dx_full), 1);
+        return;
+      } else if (code && n->use_tc && tc_conv3x3_halo_supported_unpooled(t)) {
+        ok(tc_conv3x3_halo((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, nullptr, nullptr, nullptr, t, false,
+                           n->dev_error, st, n->use_pair, nullptr, code, (bf16 *)dx_full), 1);
+        return;
+      }
       if (n->use_tc && tc_conv3x3_rowshift_supported(t))
         ok(tc_conv3x3_rowshift((const bf16 *)dz, n->tap_bwd + c.dgrad_off, nullptr, (const bf16 *)mask, (bf16 *)dx, nullptr,
                                t, false, n->dev_error, st), 1);
@@ -304,6 +322,7 @@ struct Pass {
                       t, false, n->dev_error, st), 1);
       else
         ok(simt_conv3x3<T>(dz, wr, nullptr, mask, dx, t, false, st), 1);
+      if (code) ok(simt_pool_scatter<T>(code, dx, dx_full, B, 2 * c.H, 2 * c.W, c.Cin, st), 1);
     }
   }
 
@@ -336,8 +355,11 @@ struct Pass {
     int pi = 0;
     for (int l = 0; l < kConvLayers; ++l) {
       T *y = buf(p.act[l]);
-      T *pooled = n->conv[l].pool_after ? buf(p.pooled[pi++]) : nullptr;
-      conv_forward(l, x, B, y, pooled, keep_activations);
+      T *pooled = n->conv[l].pool_after ? buf(p.pooled[pi]) : nullptr;
+      // a pass that will run backward stores, with each pooled tensor, where every window's maximum sat
+      uint8_t *code = pooled && a.grads ? reinterpret_cast<uint8_t *>(static_cast<char *>(n->ws) + p.code[pi]) : nullptr;
+      if (pooled) ++pi;
+      conv_forward(l, x, B, y, pooled, keep_activations, code);
       x = pooled ? pooled : y;
     }
     float *logits = a.logits ? a.logits : fbuf(p.logits);
@@ -374,9 +396,10 @@ struct Pass {
     }
     // convolutions 16..1.  `dz` is the gradient at layer l's pre-activation.
     T *dz = buf(p.dza), *other = buf(p.dzb);
+    auto code_of = [&](int pool) { return reinterpret_cast<const uint8_t *>(static_cast<char *>(n->ws) + p.code[pool]); };
     {
       const ConvLayer &c = n->conv[15];
-      ok(simt_maxpool_bwd_relu<T>(buf(p.act[15]), buf(p.dflat), dz, B, c.H, c.W, c.Cout, st), 1);
+      ok(simt_pool_scatter<T>(code_of(4), buf(p.dflat), dz, B, c.H, c.W, c.Cout, st), 1);
     }
     for (int l = kConvLayers - 1; l >= 0; --l) {
       const ConvLayer &c = n->conv[l];
@@ -387,10 +410,7 @@ struct Pass {
       if (l == 0) {
         conv_backward(l, x, dz, B, dW, db, nullptr, nullptr);
       } else if (in_is_pool) {
-        const ConvLayer &below = n->conv[l - 1];
-        conv_backward(l, x, dz, B, dW, db, buf(p.dxlow), nullptr);
-        ok(simt_maxpool_bwd_relu<T>(buf(p.act[l - 1]), buf(p.dxlow), other, B, below.H, below.W,
-                                    below.Cout, st), 1);
+        conv_backward(l, x, dz, B, dW, db, buf(p.dxlow), nullptr, code_of(n->pool_idx[l - 1]), other);
       } else {
         conv_backward(l, x, dz, B, dW, db, other, buf(p.act[l - 1]));
       }
@@ -879,8 +899,13 @@ int vgg19_backward_host(vgg19_t *n, const void *host_images, const int32_t *host
 
 int vgg19_conv_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t batch, void *y,
                              void *pooled, void *stream) {
+  return vgg19_conv_layer_forward_ex(n, layer, x, batch, y, pooled, nullptr, stream);
+}
+
+int vgg19_conv_layer_forward_ex(vgg19_t *n, int32_t layer, const void *x, int32_t batch, void *y, void *pooled,
+                                uint8_t *pool_code, void *stream) {
   if (!n) return VGG19_ERR_ARG;
-  if (layer < 1 || layer > kConvLayers || !x || !y || batch < 1)
+  if (layer < 1 || layer > kConvLayers || !x || !y || batch < 1 || (pool_code && !pooled))
     return fail(n, VGG19_ERR_ARG, "bad layer (%d), batch (%d) or null tensor", layer, batch);
   if (pooled && !n->conv[layer - 1].pool_after) {
     // pooling after any layer is well defined; only the fused schedule is per-layer
@@ -896,11 +921,11 @@ int vgg19_conv_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t b
   }
   if (n->cfg.dtype == VGG19_BF16) {
     Pass<bf16> ps{n, plan, st};
-    ps.conv_forward(layer - 1, (const bf16 *)x, batch, (bf16 *)y, (bf16 *)pooled);
+    ps.conv_forward(layer - 1, (const bf16 *)x, batch, (bf16 *)y, (bf16 *)pooled, true, pool_code);
     e = ps.err;
   } else {
     Pass<float> ps{n, plan, st};
-    ps.conv_forward(layer - 1, (const float *)x, batch, (float *)y, (float *)pooled);
+    ps.conv_forward(layer - 1, (const float *)x, batch, (float *)y, (float *)pooled, true, pool_code);
     e = ps.err;
   }
   if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
@@ -908,12 +933,14 @@ int vgg19_conv_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t b
 }
 
 int vgg19_conv_layer_backward_ex(vgg19_t *n, int32_t layer, const void *x, const void *dz, int32_t batch,
-                                 float *dw, float *db, void *dx, const void *relu_mask, void *stream) {
+                                 float *dw, float *db, void *dx, const void *relu_mask, const uint8_t *pool_code,
+                                 void *stream) {
   if (!n) return VGG19_ERR_ARG;
   if (layer < 1 || layer > kConvLayers || !dz || batch < 1 || (!dw != !db) || (dw && !x) || (!dw && !dx))
     return fail(n, VGG19_ERR_ARG, "bad layer (%d), batch (%d) or null tensor", layer, batch);
   if (dx && layer == 1) return fail(n, VGG19_ERR_ARG, "layer 1 has no input gradient");
   if (relu_mask && !dx) return fail(n, VGG19_ERR_ARG, "relu_mask without dx");
+  if (pool_code && (!dx || relu_mask)) return fail(n, VGG19_ERR_ARG, "pool_code needs dx and excludes relu_mask");
   int rc = check_batch(n, batch, VGG19_MODE_BACKWARD, 0);
   if (rc != VGG19_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -922,11 +949,17 @@ int vgg19_conv_layer_backward_ex(vgg19_t *n, int32_t layer, const void *x, const
   cudaError_t e;
   if (n->cfg.dtype == VGG19_BF16) {
     Pass<bf16> ps{n, p, st};
-    ps.conv_backward(layer - 1, (const bf16 *)x, (const bf16 *)dz, batch, dw, db, (bf16 *)dx, (const bf16 *)relu_mask);
+    if (pool_code)
+      ps.conv_backward(layer - 1, (const bf16 *)x, (const bf16 *)dz, batch, dw, db, ps.buf(p.dxlow), nullptr, pool_code, (bf16 *)dx);
+    else
+      ps.conv_backward(layer - 1, (const bf16 *)x, (const bf16 *)dz, batch, dw, db, (bf16 *)dx, (const bf16 *)relu_mask);
     e = ps.err;
   } else {
     Pass<float> ps{n, p, st};
-    ps.conv_backward(layer - 1, (const float *)x, (const float *)dz, batch, dw, db, (float *)dx, (const float *)relu_mask);
+    if (pool_code)
+      ps.conv_backward(layer - 1, (const float *)x, (const float *)dz, batch, dw, db, ps.buf(p.dxlow), nullptr, pool_code, (float *)dx);
+    else
+      ps.conv_backward(layer - 1, (const float *)x, (const float *)dz, batch, dw, db, (float *)dx, (const float *)relu_mask);
     e = ps.err;
   }
   if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
@@ -937,7 +970,7 @@ int vgg19_conv_layer_backward(vgg19_t *n, int32_t layer, const void *x, const vo
                               int32_t batch, float *dw, float *db, void *dx, void *stream) {
   if (!n) return VGG19_ERR_ARG;
   if (!x || !dw || !db) return fail(n, VGG19_ERR_ARG, "bad layer (%d), batch (%d) or null tensor", layer, batch);
-  return vgg19_conv_layer_backward_ex(n, layer, x, dz, batch, dw, db, dx, nullptr, stream);
+  return vgg19_conv_layer_backward_ex(n, layer, x, dz, batch, dw, db, dx, nullptr, nullptr, stream);
 }
 
 int vgg19_saved_tensor(const vgg19_t *n, int32_t batch, int32_t mode, int32_t index,

@@ -129,3 +129,60 @@ def test_conv_layer_tail_round_batch100(layer, S, Cin, Cout):
     # against the single-CTA kernels over the whole batch: rare one-ulp rounding flips only
     assert rel_l2(y, outs[p.binding.VGG19_FLAG_NO_CTA_PAIRS][0]) <= 1e-3
     assert rel_l2(dx, outs[p.binding.VGG19_FLAG_NO_CTA_PAIRS][1]) <= 1e-3
+
+
+def expected_pool_codes(y):
+    """Arg-max code of every 2x2 window of an NHWC activation: 0..3 in the order (0,0), (0,1), (1,0), (1,1),
+    the first maximum on ties; 4 where the maximum is not positive."""
+    N, H, W, C = y.shape
+    w = y.reshape(N, H // 2, 2, W // 2, 2, C).transpose(0, 1, 3, 5, 2, 4).reshape(N, H // 2, W // 2, C, 4)
+    code = np.argmax(w, axis=-1).astype(np.uint8)
+    code[w.max(axis=-1) <= 0] = 4
+    return code
+
+
+# (layer that ends a block, the layer above the pool or None, H=W of the block-ending layer, its Cin, Cout)
+POOLS = [(2, 3, 224, 64, 64), (4, 5, 112, 128, 128), (8, 9, 56, 256, 256), (12, 13, 28, 512, 512), (16, None, 14, 512, 512)]
+
+
+@pytest.mark.parametrize("below,above,S,Cin,Cout", POOLS)
+def test_pool_codes_and_scatter_through_the_pool(net224, below, above, S, Cin, Cout):
+    """The block-ending layers record, with the pooled tensor, where each window's maximum sat; the input
+    gradient of the layer above the pool is scattered through the pool by those codes (in the kernel's own
+    epilogue at the 224x224 and 112x112 blocks).  Codes: against the arg-max of the stored activation.
+    Scatter: against the checker's max-pool backward and ReLU backward at that stored activation."""
+    p, net, params = net224
+    B = 3 if S <= 28 else 1
+    x = layer_input(below, B, S, Cin)
+    xd = torch.from_numpy(x).to(DEV).to(torch.bfloat16)
+    y = torch.empty((B, S, S, Cout), dtype=torch.bfloat16, device=DEV)
+    pooled = torch.empty((B, S // 2, S // 2, Cout), dtype=torch.bfloat16, device=DEV)
+    code = torch.full((B, S // 2, S // 2, Cout), 255, dtype=torch.uint8, device=DEV)
+    st = torch.cuda.current_stream()
+    p.vgg19_conv_layer_forward_ex(net.handle, below, xd, B, y, pooled, code, st)
+    net.sync_status()
+    y_host = y.float().cpu().numpy().astype(np.float64)
+    want = expected_pool_codes(y_host)
+    got = code.cpu().numpy()
+    assert np.array_equal(got, want), f"{(got != want).sum()} of {want.size} codes differ"
+    assert (want == 4).any() and all((want == q).any() for q in range(4))
+    assert np.array_equal(pooled.float().cpu().numpy(), oracle.maxpool2x2_fwd(y_host))
+    if above is None:
+        return
+    C2 = SHAPES_BY_LAYER[above][2]
+    dz = si.normal(B * (S // 2) ** 2 * C2, seed=400 + above, stddev=1e-3, bf16_exact=True).reshape(B, S // 2, S // 2, C2)
+    dz = dz * (si.uniform(dz.size, seed=500 + above).reshape(dz.shape) < 0.5)
+    dzd = torch.from_numpy(dz).to(DEV).to(torch.bfloat16)
+    dfull = torch.full((B, S, S, Cout), float("nan"), dtype=torch.bfloat16, device=DEV)
+    p.vgg19_conv_layer_backward_ex(net.handle, above, None, dzd, B, None, None, dfull, None, code, st)
+    net.sync_status()
+    Wt, _ = layer_params(p, net, params, above)
+    low = oracle.round_bf16(oracle.conv3x3_dgrad(dz, Wt))
+    ref = oracle.relu_bwd(y_host, oracle.maxpool2x2_bwd(y_host, low))
+    g = dfull.float().cpu().numpy()
+    assert np.isfinite(g).all()
+    assert np.array_equal(g != 0, ref != 0) or rel_l2(g, ref) <= 1e-3
+    assert rel_l2(g, ref) <= 1e-3
+
+
+SHAPES_BY_LAYER = {3: (112, 64, 128), 5: (56, 128, 256), 9: (28, 256, 512), 13: (14, 512, 512)}
