@@ -210,7 +210,10 @@ int vgg19_conv_layer_forward(vgg19_t *net, int32_t layer, const void *x, int32_t
  * or NULL), device uint8 [batch][h/2][w/2][Cout], receives for every window
  * where its maximum sits - 0..3 for (0,0), (0,1), (1,0), (1,1), the first one
  * on ties - or 4 when that maximum is not positive, i.e. when the ReLU before
- * the pool passes no gradient to the window. */
+ * the pool passes no gradient to the window.  y may be NULL (with pooled, and
+ * without pool_code) where the layer's kernel pools in its own epilogue, as a
+ * forward-only pass runs the block-ending layers: the full-resolution output
+ * is then never written; VGG19_ERR_ARG where it cannot. */
 int vgg19_conv_layer_forward_ex(vgg19_t *net, int32_t layer, const void *x, int32_t batch, void *y, void *pooled,
                                 uint8_t *pool_code, void *stream);
 

@@ -19,8 +19,8 @@
 // Roles and pipeline are those of the general convolution kernel: warp 0 TMA
 // producer, warp 1 MMA issuer and TMEM owner, then epilogue warps; double-buffered
 // accumulator; persistent CTAs; time-limited waits.  The main loop is five MMAs
-// per tile, so the epilogue sets the pace: two groups of eight epilogue warps take
-// alternate tiles (each group its own accumulator buffer, staging tile and named
+// per tile, so the epilogue sets the pace: three groups of eight epilogue warps take
+// tiles in turn (each group its own accumulator buffer, staging tile and named
 // barrier), so that one tile's chain of wait, tensor-memory load, conversion, staging
 // and store overlaps the next tile's; within a group two warps per TMEM lane quarter
 // each convert and store 32 of the 64 output channels of their rows.
@@ -39,9 +39,11 @@ constexpr int STAGES = 8;
 constexpr int W_TAP_BYTES = BN * 16;      // 64 output channels x 8 channels
 constexpr int W_BYTES = 10 * W_TAP_BYTES;
 constexpr int OUT_TILE_BYTES = BM * BN * 2;  // 16 KB staging tile for the TMA store, two of them
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_TILE_BYTES + W_BYTES + 1024 + 256;
-constexpr int kThreads = 576;  // producer, MMA issuer, two groups of eight epilogue warps
+constexpr int kGroups = 3;     // epilogue groups, each with its own accumulator buffer and staging tile
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + kGroups * OUT_TILE_BYTES + W_BYTES + 1024 + 256;
 constexpr int kGroupThreads = 256;
+constexpr int kThreads = 64 + kGroups * kGroupThreads;  // producer, MMA issuer, the groups of eight epilogue warps
+constexpr int kTmemCols = 256;  // kGroups accumulators of 64 columns, rounded up to a power of two
 
 constexpr int PW = 8, PH = 16, IW = PW + 2, IH = PH + 2;  // patch mode: output patch and input patch with halo
 constexpr int PATCH_BYTES = IW * IH * 16;                 // 2880
@@ -61,14 +63,14 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t out_smem = smem_base + STAGES * STAGE_BYTES;  // 1024-byte aligned (20 KB stages)
-  const uint32_t w_smem = out_smem + 2 * OUT_TILE_BYTES;
+  const uint32_t w_smem = out_smem + kGroups * OUT_TILE_BYTES;
   const uint32_t bars = w_smem + W_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto acc_full_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
-  auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
-  const uint32_t w_bar = bars + 8u * (2 * STAGES + 4);
-  const uint32_t drain_bar = bars + 8u * (2 * STAGES + 5);
+  auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * STAGES + kGroups + b); };
+  const uint32_t w_bar = bars + 8u * (2 * STAGES + 2 * kGroups);
+  const uint32_t drain_bar = bars + 8u * (2 * STAGES + 2 * kGroups + 1);
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ __align__(16) float bias_s[512];  // the layer's bias (zeros when it has none)
@@ -93,7 +95,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 256); }
+    for (int b = 0; b < kGroups; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), kGroupThreads); }
     mbar_init(w_bar, 1);
     mbar_init(drain_bar, 1);
     mbar_fence_init();
@@ -101,7 +103,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tma_prefetch_desc(&map_w);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+    tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -160,8 +162,8 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       int local = 0;
       bool ok = mbar_wait(w_bar, 0, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
       for (int tile = blockIdx.x; tile < a.m_tiles && ok; tile += gridDim.x, ++local) {
-        const int buf = local & 1;
-        const uint32_t use = (uint32_t)(local >> 1);
+        const int buf = local % kGroups;
+        const uint32_t use = (uint32_t)(local / kGroups);
         if (!mbar_wait(acc_empty_bar(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
         if (!mbar_wait(full_bar(stage), phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
         tc_fence_after();
@@ -189,7 +191,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       }
     }
   } else {
-    const int group = (warp - 2) >> 3;            // which of the two accumulator buffers / staging tiles
+    const int group = (warp - 2) >> 3;            // which of the accumulator buffers / staging tiles
     const int quarter = warp & 3;                 // the TMEM lane quarter this warp may read
     const int row = quarter * 32 + lane;
     const int cc = (((warp - 2) >> 2) & 1) * 32;  // this warp's 32 of the 64 output channels
@@ -197,7 +199,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const bool issuer = threadIdx.x == 64 + group * kGroupThreads;  // owns the group's store groups
     const uint32_t stage_out = out_smem + (uint32_t)group * OUT_TILE_BYTES;
     uint32_t use = 0;  // tiles this group has taken
-    for (int tile = blockIdx.x + group * gridDim.x; tile < a.m_tiles; tile += 2 * gridDim.x, ++use) {
+    for (int tile = blockIdx.x + group * gridDim.x; tile < a.m_tiles; tile += kGroups * gridDim.x, ++use) {
       const bool got = mbar_wait(acc_full_bar(group), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
       // the group's previous store must have read the staging tile before anyone refills it; the
       // barrier doubles as the vote that lets the group's warps leave together if any wait failed
@@ -254,7 +256,7 @@ conv3x3_c8_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 2 * BN);
+    tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 

@@ -51,6 +51,11 @@ struct PairArgs {
   int relu;
   const float* bias;
   const bf16* mask;
+  // Forward-only passes of a block-ending layer: the full-resolution output is not kept; every value
+  // goes straight into the 2x2 max-pooled tensor [N][H/2][W/2][Cout] (zeroed beforehand) with a
+  // vector max-reduction on global memory.  A window's four pixels may sit in different tiles and
+  // CTAs: the reduction needs no meeting point, and a maximum does not depend on the order.
+  bf16* pooled;
   int* dev_error;
   // Tail split.  The first main_tiles tiles are whole rounds of the resident pairs; the rest (fewer
   // than half a round) are each cut into tail_splits ranges of tail_kb K blocks so that the last
@@ -74,7 +79,12 @@ __device__ __forceinline__ Work get_work(int w, const PairArgs& a, int k_blocks)
   return Work{a.main_tiles + t, kb0, min(k_blocks, kb0 + a.tail_kb), z};
 }
 
-template <int BN>
+// pooled[row][0..7] = max(pooled[row][0..7], v): eight bf16 in one reduction (ReLU outputs: the tensor starts at zero)
+__device__ __forceinline__ void red_max_bf16x8(bf16* dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("red.global.max.noftz.v4.bf16x2 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+template <int BN, bool POOL>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_m, PairArgs a) {
@@ -249,6 +259,12 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       const bool valid = pixel < a.pixels;
       const bool tile_valid = (long)m_tile * BM < a.pixels;
       const int c_base = n_tile * BN;
+      bf16* pool_row = nullptr;
+      if (POOL && valid) {
+        const int pw = (int)(pixel % a.W), t = (int)(pixel / a.W);
+        const int ph = t % a.H, pn = t / a.H;
+        pool_row = a.pooled + (((long)pn * (a.H / 2) + ph / 2) * (a.W / 2) + pw / 2) * a.Cout + c_base;
+      }
       if (wk.split >= 0) {
         // part of a tail tile's K range: raw sums, one row per thread, for the finishing kernel
         float* dst = a.partial + ((size_t)wk.split * a.tail_rows + (size_t)(pixel - a.tail_row0)) * a.Cout + c_base;
@@ -271,8 +287,10 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       }
 #pragma unroll 1
       for (int c64 = 0; c64 < BN && tile_valid; c64 += 64) {
-        if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
-        named_bar_sync(1, 128);
+        if (!POOL) {
+          if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
+          named_bar_sync(1, 128);
+        }
         bool mask_ready = false;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -288,6 +306,14 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
             __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
             packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          if (POOL) {
+            if (pool_row) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                red_max_bf16x8(pool_row + cc + 8 * q, packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+            }
+            continue;
           }
           if (a.mask) {
             if (!mask_ready) {  // a failed wait leaves the chunk unmasked; the error word says so
@@ -317,6 +343,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                 make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
           }
         }
+        if (POOL) continue;
         fence_async_smem();
         named_bar_sync(1, 128);  // the staging tile is complete, and everyone has read the mask tile
         if (issuer) {
@@ -357,7 +384,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 // (out, mask already point at the first tail row); eight channels per thread, splits added in order.
 __global__ void pair_tail_finish_kernel(const float* __restrict__ partial, int splits, long elems, int Cout,
                                         const float* __restrict__ bias, int relu, const bf16* __restrict__ mask,
-                                        bf16* __restrict__ out) {
+                                        bf16* __restrict__ out, bf16* __restrict__ pooled, long row0, int H, int W) {
   const long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 8;
   if (i >= elems) return;
   float x[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -389,16 +416,25 @@ __global__ void pair_tail_finish_kernel(const float* __restrict__ partial, int s
       packed[e] &= keep;
     }
   }
+  if (pooled) {
+    // forward-only pass of a block-ending layer: straight into the pooled tensor (see PairArgs::pooled)
+    const long pixel = row0 + i / Cout;
+    const int pw = (int)(pixel % W), t = (int)(pixel / W);
+    const int ph = t % H, pn = t / H;
+    red_max_bf16x8(pooled + (((long)pn * (H / 2) + ph / 2) * (W / 2) + pw / 2) * Cout + c, packed[0], packed[1], packed[2],
+                   packed[3]);
+    return;
+  }
   *reinterpret_cast<uint4*>(out + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
 }
 
 // CTA pairs of this kernel that can be resident at once (one pair per two SMs at most)
-template <int BN>
+template <int BN, bool POOL>
 cudaError_t resident_pairs(int* out) {
   using T = PairTile<BN>;
   static int max_pairs = 0;
   if (!max_pairs) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_pair_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_pair_tc_kernel<BN, POOL>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
@@ -412,7 +448,7 @@ cudaError_t resident_pairs(int* out) {
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr; cfg.numAttrs = 1;
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, conv3x3_pair_tc_kernel<BN>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, conv3x3_pair_tc_kernel<BN, POOL>, &cfg);
     if (e != cudaSuccess || n < 1) { cudaGetLastError(); n = sms / 2; }
     max_pairs = n < sms / 2 ? n : sms / 2;
     if (max_pairs < 1) max_pairs = 1;
@@ -436,15 +472,18 @@ size_t tc_conv3x3_pair_scratch_elems(ConvShape s) {
 }
 
 cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, const bf16* mask, bf16* out, ConvShape s,
-                            bool relu, int* dev_error, cudaStream_t st, float* partial, int* launches) {
+                            bool relu, int* dev_error, cudaStream_t st, float* partial, int* launches, bf16* pooled) {
   if (launches) *launches = 0;
   if (!tc_conv3x3_pair_supported(s)) return cudaErrorInvalidValue;
+  if (pooled && (mask || !relu || (s.H & 1) || (s.W & 1))) return cudaErrorInvalidValue;  // maxima of ReLU outputs only
+  if (!pooled && !out) return cudaErrorInvalidValue;
   constexpr int BN = 256;
   using T = PairTile<BN>;
   CUtensorMap mx, mw, my, mm;
   if (!make_im2col_map(&mx, in, s.N, s.H, s.W, s.Cin, BM)) return cudaErrorInvalidValue;
   if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, BN / 2)) return cudaErrorInvalidValue;
-  if (!make_tiled_map_2d(&my, out, (uint64_t)s.N * s.H * s.W, (uint64_t)s.Cout, BM)) return cudaErrorInvalidValue;
+  my = mw;  // only read when there is a full-resolution output
+  if (!pooled && !make_tiled_map_2d(&my, out, (uint64_t)s.N * s.H * s.W, (uint64_t)s.Cout, BM)) return cudaErrorInvalidValue;
   mm = my;  // only read when there is a mask
   if (mask && !make_tiled_map_2d(&mm, mask, (uint64_t)s.N * s.H * s.W, (uint64_t)s.Cout, BM)) return cudaErrorInvalidValue;
   PairArgs a;
@@ -455,10 +494,14 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
   a.m_pairs = (a.pixels + 2 * BM - 1) / (2 * BM);
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0;
-  a.bias = bias; a.mask = mask; a.dev_error = dev_error;
+  a.bias = bias; a.mask = mask; a.dev_error = dev_error; a.pooled = pooled;
   int cap = 0;
-  cudaError_t e = resident_pairs<BN>(&cap);
+  cudaError_t e = pooled ? resident_pairs<BN, true>(&cap) : resident_pairs<BN, false>(&cap);
   if (e != cudaSuccess) return e;
+  if (pooled) {
+    e = cudaMemsetAsync(pooled, 0, (size_t)s.N * (s.H / 2) * (s.W / 2) * s.Cout * sizeof(bf16), st);
+    if (e != cudaSuccess) return e;
+  }
   const int tiles = a.m_pairs * a.n_tiles, k_blocks = 9 * a.cin_blocks;
   a.main_tiles = tiles; a.tail_splits = 1; a.tail_kb = k_blocks; a.tail_row0 = 0; a.tail_rows = 0; a.partial = nullptr;
   // Whole rounds of `cap` tiles, then a tail of fewer than half a round: cut each tail tile's K range
@@ -481,14 +524,16 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
   }
   const int work = a.main_tiles + (tiles - a.main_tiles) * a.tail_splits;
   const int pairs = work < cap ? work : cap;
-  conv3x3_pair_tc_kernel<BN><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
+  if (pooled) conv3x3_pair_tc_kernel<BN, true><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
+  else conv3x3_pair_tc_kernel<BN, false><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
   e = cudaGetLastError();
   if (launches) *launches = 1;
   if (e != cudaSuccess || !a.partial) return e;
   const long elems = (long)a.tail_rows * a.Cout;
   const size_t row_off = (size_t)a.tail_row0 * a.Cout;
   pair_tail_finish_kernel<<<(unsigned)((elems / 8 + 255) / 256), 256, 0, st>>>(
-      partial, a.tail_splits, elems, a.Cout, bias, a.relu, mask ? mask + row_off : nullptr, out + row_off);
+      partial, a.tail_splits, elems, a.Cout, bias, a.relu, mask ? mask + row_off : nullptr, pooled ? nullptr : out + row_off,
+      pooled, (long)a.tail_row0, s.H, s.W);
   if (launches) *launches = 2;
   return cudaGetLastError();
 }

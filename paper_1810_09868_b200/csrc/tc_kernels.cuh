@@ -27,7 +27,7 @@ bool tc_conv3x3_pair_supported(ConvShape s);
 size_t tc_conv3x3_pair_scratch_elems(ConvShape s);
 cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, const bf16* mask,
                             bf16* out, ConvShape s, bool relu, int* dev_error, cudaStream_t st,
-                            float* partial = nullptr, int* launches = nullptr);
+                            float* partial = nullptr, int* launches = nullptr, bf16* pooled = nullptr);
 
 // The same convolution with the input patch (plus halo) kept in shared memory
 // for all nine taps (tc_conv_halo.cu): the large-image, few-channel layers.

@@ -242,6 +242,14 @@ struct Pass {
     return l == 0 && n->use_tc && p.valid && tc_first_conv_supported(s);
   }
 
+  // whether layer l's forward kernel can leave out the full-resolution output and write only the pooled one
+  bool pools_in_epilogue(int l, int B) const {
+    const ConvLayer &c = n->conv[l];
+    ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
+    if (!n->use_tc || first_tc_ok(l, s) || l == 0) return false;
+    return tc_conv3x3_rowshift_supported(s) || tc_conv3x3_halo_supported(s) || (pair_ok(s) && c.H % 2 == 0 && c.W % 2 == 0);
+  }
+
   // y = relu(conv(x) + b), optionally pooled.  With need_y false the full-resolution output may be
   // left unwritten when the pool is fused into the convolution's epilogue.
   // code (with pooled, or null): receives the arg-max code of every pooling window for the backward pass.
@@ -262,10 +270,14 @@ struct Pass {
                          pooled ? code : nullptr), 1);
       return;
     } else if (pair_ok(s)) {
+      // a block-ending layer whose own output nobody reads again pools in its epilogue
+      const bool pool_only = pooled && !need_y && !code && c.H % 2 == 0 && c.W % 2 == 0;
       int k = 1;
       ok(tc_conv3x3_pair((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
-                         (bf16 *)y, s, true, n->dev_error, st, p.valid && forward_tail_split ? fbuf(p.partial) : nullptr, &k), 0);
-      launches += k;
+                         (bf16 *)y, s, true, n->dev_error, st, p.valid && forward_tail_split ? fbuf(p.partial) : nullptr, &k,
+                         pool_only ? (bf16 *)pooled : nullptr), 0);
+      launches += k + (pool_only ? 1 : 0);
+      if (pool_only) return;
     } else if (tc_conv_ok(s))
       ok(tc_conv3x3((const bf16 *)x, (const bf16 *)wt(c.w_off), n->params + c.b_off, nullptr,
                     (bf16 *)y, s, true, n->dev_error, st), 1);
@@ -905,7 +917,7 @@ int vgg19_conv_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t b
 int vgg19_conv_layer_forward_ex(vgg19_t *n, int32_t layer, const void *x, int32_t batch, void *y, void *pooled,
                                 uint8_t *pool_code, void *stream) {
   if (!n) return VGG19_ERR_ARG;
-  if (layer < 1 || layer > kConvLayers || !x || !y || batch < 1 || (pool_code && !pooled))
+  if (layer < 1 || layer > kConvLayers || !x || (!y && !pooled) || batch < 1 || (pool_code && (!pooled || !y)))
     return fail(n, VGG19_ERR_ARG, "bad layer (%d), batch (%d) or null tensor", layer, batch);
   if (pooled && !n->conv[layer - 1].pool_after) {
     // pooling after any layer is well defined; only the fused schedule is per-layer
@@ -921,11 +933,14 @@ int vgg19_conv_layer_forward_ex(vgg19_t *n, int32_t layer, const void *x, int32_
   }
   if (n->cfg.dtype == VGG19_BF16) {
     Pass<bf16> ps{n, plan, st};
-    ps.conv_forward(layer - 1, (const bf16 *)x, batch, (bf16 *)y, (bf16 *)pooled, true, pool_code);
+    if (!y && !ps.pools_in_epilogue(layer - 1, batch))
+      return fail(n, VGG19_ERR_ARG, "layer %d at this size has no pooled-only kernel: y must not be null", layer);
+    ps.conv_forward(layer - 1, (const bf16 *)x, batch, (bf16 *)y, (bf16 *)pooled, y != nullptr, pool_code);
     e = ps.err;
   } else {
     Pass<float> ps{n, plan, st};
-    ps.conv_forward(layer - 1, (const float *)x, batch, (float *)y, (float *)pooled, true, pool_code);
+    if (!y) return fail(n, VGG19_ERR_ARG, "the fp32 configuration has no pooled-only kernel: y must not be null");
+    ps.conv_forward(layer - 1, (const float *)x, batch, (float *)y, (float *)pooled, y != nullptr, pool_code);
     e = ps.err;
   }
   if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));

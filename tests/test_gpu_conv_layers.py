@@ -186,3 +186,28 @@ def test_pool_codes_and_scatter_through_the_pool(net224, below, above, S, Cin, C
 
 
 SHAPES_BY_LAYER = {3: (112, 64, 128), 5: (56, 128, 256), 9: (28, 256, 512), 13: (14, 512, 512)}
+
+
+@pytest.mark.parametrize("layer,S,Cin,Cout", [(2, 224, 64, 64), (4, 112, 128, 128), (8, 56, 256, 256), (12, 28, 512, 512),
+                                              (16, 14, 512, 512)])
+def test_block_ending_layers_pool_in_their_epilogue(net224, layer, S, Cin, Cout):
+    """Forward-only passes never write the full-resolution output of a block-ending layer: the pooled tensor
+    comes out of the convolution's own epilogue (shuffles inside a patch tile at 224x224 and 112x112, a
+    max-reduction on global memory at 56x56 and below).  It must equal, bit for bit, the 2x2 max-pool of the
+    full-resolution output the same layer writes when asked for it."""
+    p, net, params = net224
+    B = 3
+    x = layer_input(layer, B, S, Cin)
+    xd = torch.from_numpy(x).to(DEV).to(torch.bfloat16)
+    y = torch.empty((B, S, S, Cout), dtype=torch.bfloat16, device=DEV)
+    st = torch.cuda.current_stream()
+    p.vgg19_conv_layer_forward(net.handle, layer, xd, B, y, None, st)
+    for rep in range(2):
+        pooled = torch.full((B, S // 2, S // 2, Cout), float("nan"), dtype=torch.bfloat16, device=DEV)
+        p.vgg19_conv_layer_forward_ex(net.handle, layer, xd, B, None, pooled, None, st)
+        net.sync_status()
+        want = torch.nn.functional.max_pool2d(y.float().permute(0, 3, 1, 2), 2).permute(0, 2, 3, 1)
+        assert torch.equal(pooled.float(), want), rep
+    Wt, b = layer_params(p, net, params, layer)
+    ref = oracle.maxpool2x2_fwd(oracle.round_bf16(oracle.relu_fwd(oracle.conv3x3_fwd(x[:1], Wt, b))))
+    assert rel_l2(pooled[:1].float().cpu().numpy(), ref) <= 1e-3
