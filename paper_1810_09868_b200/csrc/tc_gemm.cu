@@ -59,6 +59,11 @@ struct GemmArgs {
   int* dev_error;
   float* db_partial; // column sums of A at db_partial[((split * n_tiles) + n_tile) * M + m], or null
   int tma_store;     // fp32 output (partial or out_f, no bias / ReLU / mask) leaves through staging tiles and map_c
+  // Gradient-descent step folded into the epilogue (tma_store path, no split): the tile is a weight
+  // gradient that is never stored; out_f / map_c address the fp32 master weights, which become
+  // w - lr * D, and sgd_copy receives their bf16 rounding.  lr is read from device memory.
+  bf16* sgd_copy;
+  const float* sgd_lr;
 };
 constexpr int kStoreStagingBytes = 2 * BM * 128;  // two tiles of 128 rows x 32 fp32
 
@@ -300,11 +305,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const bool issuer = threadIdx.x == 64;
       const int row = quarter * 32 + lane;
       const int row0 = (g.partial ? (int)blockIdx.y * g.M : 0) + m0;
+      // folded update: this thread's 32 master weights of the next chunk are requested one chunk ahead
+      const bool fold = g.sgd_copy != nullptr;
+      const float lr = fold ? __ldg(g.sgd_lr) : 0.f;
+      const long w_row = (long)m * g.ldc + n0;
+      float4 w_next[8];
+      auto fetch = [&](int cc) {
+        if (row_ok && n0 + cc < g.N) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) w_next[q] = __ldg(reinterpret_cast<const float4*>(g.out_f + w_row + cc) + q);
+        }
+      };
+      if (fold) fetch(0);
 #pragma unroll 1
       for (int cc = 0; cc < BN; cc += 32) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)cc, v);
         tmem_ld_wait();
+        if (fold) {
+          float4 w[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) w[q] = w_next[q];
+          if (cc + 32 < BN) fetch(cc + 32);
+          if (row_ok && n0 + cc < g.N) {
+            uint32_t h[16];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float a0 = fmaf(-lr, __uint_as_float(v[4 * q]), w[q].x), a1 = fmaf(-lr, __uint_as_float(v[4 * q + 1]), w[q].y);
+              const float a2 = fmaf(-lr, __uint_as_float(v[4 * q + 2]), w[q].z), a3 = fmaf(-lr, __uint_as_float(v[4 * q + 3]), w[q].w);
+              v[4 * q] = __float_as_uint(a0); v[4 * q + 1] = __float_as_uint(a1);
+              v[4 * q + 2] = __float_as_uint(a2); v[4 * q + 3] = __float_as_uint(a3);
+              __nv_bfloat162 lo = __floats2bfloat162_rn(a0, a1), hi = __floats2bfloat162_rn(a2, a3);
+              h[2 * q] = *reinterpret_cast<uint32_t*>(&lo); h[2 * q + 1] = *reinterpret_cast<uint32_t*>(&hi);
+            }
+            uint4* hp = reinterpret_cast<uint4*>(g.sgd_copy + w_row + cc);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) hp[q] = make_uint4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
+          }
+        }
         const uint32_t tile = store_smem + (uint32_t)((cc >> 5) & 1) * (BM * 128);
         if (issuer) tma_store_wait_read<1>();  // the store before last has read this staging tile
         named_bar_sync(1, 128);
@@ -480,6 +518,7 @@ cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArg
   if (plain && out_cols % 4 == 0 && (!g.partial || g.M % BM == 0 || g.M == 64) &&
       make_tiled_map_2d_f32(&mc, target, (uint64_t)out_rows, (uint64_t)out_cols, g.M == 64 ? 64 : BM))
     g.tma_store = 1;
+  if (g.sgd_copy && !g.tma_store) return cudaErrorInvalidValue;  // the folded update lives in that epilogue only
   constexpr int kBudget = 227 * 1024 - 3072 - kStoreStagingBytes;
   constexpr int max_stages = kBudget / STAGE > kMaxStages ? kMaxStages : kBudget / STAGE;
   static bool configured = false;
@@ -592,13 +631,15 @@ cudaError_t tc_dense_dx(const bf16* dY, const bf16* Wt, const bf16* mask, bf16* 
 
 // dW = dY^T X: dY [M][Out], X [M][In] -> dW fp32 [Out][In]
 cudaError_t tc_dense_dw(const bf16* dY, const bf16* X, float* dW, int M, int In, int Out, int* dev_error,
-                        cudaStream_t st) {
+                        cudaStream_t st, bf16* sgd_copy, const float* sgd_lr) {
+  if ((sgd_copy != nullptr) && (sgd_lr == nullptr || In % 32 != 0)) return cudaErrorInvalidValue;
   CUtensorMap ma, mb;
   if (!make_tiled_map_2d(&ma, dY, (uint64_t)M, (uint64_t)Out, 64)) return cudaErrorInvalidValue;
   if (!make_tiled_map_2d(&mb, X, (uint64_t)M, (uint64_t)In, 64)) return cudaErrorInvalidValue;
   GemmArgs g{};
   g.M = Out; g.N = In; g.k_blocks = (M + BK - 1) / BK; g.kb_per_split = g.k_blocks;
   g.dev_error = dev_error; g.ldc = In; g.out_f = dW;
+  g.sgd_copy = sgd_copy; g.sgd_lr = sgd_lr;
   const int m_tiles = (Out + BM - 1) / BM;
   if (In % 256 == 0) {
     g.n_tiles = In / 256;

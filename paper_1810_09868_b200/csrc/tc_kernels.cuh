@@ -82,8 +82,11 @@ cudaError_t tc_dense_forward(const bf16* X, const bf16* W, const float* bias, bf
                              float* partial, int M, int In, int Out, bool relu, int* dev_error, cudaStream_t st);
 cudaError_t tc_dense_dx(const bf16* dY, const bf16* W, const bf16* mask, bf16* dX, float* partial, int M, int In,
                         int Out, int* dev_error, cudaStream_t st);
+// With sgd_copy and sgd_lr (a device scalar) the gradient is not stored: dW then points at the layer's fp32
+// master weights, which become w - lr * gradient in the GEMM's epilogue, and sgd_copy (their bf16 copy)
+// receives the rounded result - the parameter update of a training step folded into the filter-gradient GEMM.
 cudaError_t tc_dense_dw(const bf16* dY, const bf16* X, float* dW, int M, int In, int Out, int* dev_error,
-                        cudaStream_t st);
+                        cudaStream_t st, bf16* sgd_copy = nullptr, const float* sgd_lr = nullptr);
 
 // First layer (3 input channels, 64 output channels) on tensor cores, through an
 // 8-channel zero-padded copy x8 [N][H][W][8] of the image and a padded filter
