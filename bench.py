@@ -546,7 +546,7 @@ def run_native(args):
         "warmup": args.warmup, "ms_per_step": fwd_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "image": [H, W, 3],
-                   "l2": "no explicit flush: each step writes and re-reads 3.4 GB of activations, 27x the 126 MB L2",
+                   "l2": "no explicit flush: each step writes and re-reads 2.1 GB of activations, 16x the 126 MB L2",
                    "weights": "He-normal seed 0, biases 0", "graph": "one CUDA graph per pass"},
         "clocks": clocks,
         "e2e": {"value": world * BATCH * args.steps / (e2e_ms * 1e-3), "unit": "images/s",
