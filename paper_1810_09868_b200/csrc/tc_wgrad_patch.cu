@@ -190,42 +190,58 @@ wgrad_patch_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
 }
 
 // dW[k][r][s][c] = sum over splits of the tile (c / 64, k / 64)'s partial sums; db[k] likewise from the
-// tiles of input-channel block 0.  Threads run over (r, s, c, k) with k fastest, so that the reads of a
-// warp are contiguous; splits are added in order.
+// tiles of input-channel block 0.  A block is 32 outputs (k fastest, so that a warp's reads are
+// contiguous) x 8 groups of splits: with up to 148 splits and only 9 * Cin * Cout outputs one thread per
+// output would add its splits as a chain of dependent loads.  Each group adds its range of splits in
+// order, the groups are added in order through shared memory: a fixed order, whatever the launch.
+constexpr int kFinishGroups = 8;
 __global__ void wgrad_patch_finish_kernel(const float* __restrict__ partial, int splits, int tiles, int Cin, int Cout,
                                           float* __restrict__ dW, float* __restrict__ db) {
-  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  __shared__ float part[kFinishGroups][33];
+  const int g = threadIdx.y;
+  const long i = (long)blockIdx.x * 32 + threadIdx.x;
   const long total = 9L * Cin * Cout;
-  if (db && i < Cout) {
+  const int per = (splits + kFinishGroups - 1) / kFinishGroups;
+  const int z0 = g * per, z1 = min(splits, z0 + per);
+  if (db && g == 0 && i < Cout) {
     const int kb = (int)(i / 64), kl = (int)(i % 64);  // tile (cb = 0, kb), column sums row, group Z_0
     float s = 0.f;
     for (int z = 0; z < splits; ++z)
       s += partial[((size_t)z * tiles + kb) * kPartialFloats + 128 * 192 + 64 * 192 + 128 + kl];
     db[i] = s;
   }
-  if (i >= total) return;
-  const int k = (int)(i % Cout);
-  long t = i / Cout;
-  const int c = (int)(t % Cin); t /= Cin;
-  const int s9 = (int)(t % 3), r = (int)(t / 3);
-  const int kb = k / 64, kl = k % 64, cb = c / 64, cl = c % 64;
-  const int tile = cb * (Cout / 64) + kb;
-  const int col = (2 - s9) * 64 + kl;
-  const size_t off = r < 2 ? (size_t)(r * 64 + cl) * 192 + col : (size_t)128 * 192 + (size_t)cl * 192 + col;
-  // independent loads, issued several at a time; the additions stay in split order
   float sum = 0.f;
-  const float* src = partial + (size_t)tile * kPartialFloats + off;
-  const size_t stride = (size_t)tiles * kPartialFloats;
-  int z = 0;
-  for (; z + 8 <= splits; z += 8) {
-    float v[8];
+  long out = -1;
+  if (i < total) {
+    const int k = (int)(i % Cout);
+    long t = i / Cout;
+    const int c = (int)(t % Cin); t /= Cin;
+    const int s9 = (int)(t % 3), r = (int)(t / 3);
+    const int kb = k / 64, kl = k % 64, cb = c / 64, cl = c % 64;
+    const int tile = cb * (Cout / 64) + kb;
+    const int col = (2 - s9) * 64 + kl;
+    const size_t off = r < 2 ? (size_t)(r * 64 + cl) * 192 + col : (size_t)128 * 192 + (size_t)cl * 192 + col;
+    out = ((long)k * 9 + r * 3 + s9) * Cin + c;
+    const float* src = partial + (size_t)tile * kPartialFloats + off;
+    const size_t stride = (size_t)tiles * kPartialFloats;
+    int z = z0;
+    for (; z + 4 <= z1; z += 4) {  // independent loads, issued together; the additions stay in split order
+      float v[4];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) v[u] = src[(size_t)(z + u) * stride];
+      for (int u = 0; u < 4; ++u) v[u] = src[(size_t)(z + u) * stride];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) sum += v[u];
+      for (int u = 0; u < 4; ++u) sum += v[u];
+    }
+    for (; z < z1; ++z) sum += src[(size_t)z * stride];
   }
-  for (; z < splits; ++z) sum += src[(size_t)z * stride];
-  dW[((size_t)k * 9 + r * 3 + s9) * Cin + c] = sum;
+  part[g][threadIdx.x] = sum;
+  __syncthreads();
+  if (g == 0 && out >= 0) {
+    float tot = part[0][threadIdx.x];
+#pragma unroll
+    for (int q = 1; q < kFinishGroups; ++q) tot += part[q][threadIdx.x];
+    dW[out] = tot;
+  }
 }
 
 int patch_sm_count() {
@@ -290,7 +306,8 @@ cudaError_t tc_conv3x3_wgrad_patch(const bf16* x, const bf16* dz, float* dW, flo
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const long total = 9L * s.Cin * s.Cout;
-  wgrad_patch_finish_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(partial, splits, tiles, s.Cin, s.Cout, dW, db);
+  wgrad_patch_finish_kernel<<<(unsigned)((total + 31) / 32), dim3(32, kFinishGroups), 0, st>>>(partial, splits, tiles, s.Cin, s.Cout, dW,
+                                                                                                   db);
   return cudaGetLastError();
 }
 

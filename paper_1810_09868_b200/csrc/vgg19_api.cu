@@ -229,6 +229,7 @@ struct Pass {
   // summation order of the images in those tiles with the batch size, so a training pass, whose ReLU and
   // pooling decisions should not depend on what else is in the batch, keeps it off for its forward half.
   bool forward_tail_split = true;
+  const void *x8_of = nullptr;  // the image whose 8-channel copy this pass has already made
   // Training step on one GPU: the learning rate (device scalar).  Where a filter-gradient kernel can
   // apply the update itself (the dense layers' GEMM: 86 % of the parameters at 224x224) the gradient is
   // never stored; `folded` tells the caller which parameter ranges are already updated.
@@ -263,6 +264,7 @@ struct Pass {
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
     if (first_tc_ok(l, s)) {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
+      x8_of = x;
       ok(tc_first_conv((const bf16 *)buf(p.x8), n->w8, n->params + c.b_off, (bf16 *)y, s, true, n->dev_error, st), 1);
     } else if (n->use_tc && tc_conv3x3_rowshift_supported(s)) {
       ok(tc_conv3x3_rowshift((const bf16 *)x, n->tap_fwd + c.dgrad_off, n->params + c.b_off, nullptr,
@@ -302,7 +304,7 @@ struct Pass {
     if (!dW) {
       // input gradient only (per-layer entry point)
     } else if (first_tc_ok(l, s)) {
-      ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
+      if (x8_of != x) ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);  // the forward half's copy serves
       ok(tc_first_wgrad((const bf16 *)buf(p.x8), (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st), 2);
     } else if (n->use_tc && tc_wgrad_patch_supported(s)) {
       ok(tc_conv3x3_wgrad_patch((const bf16 *)x, (const bf16 *)dz, dW, db, fbuf(p.partial), s, n->dev_error, st), 2);
@@ -531,8 +533,15 @@ int run_pass(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st) {
   GraphEntry e{};
   size_t n_nodes = 0;
   if (cudaGraphGetNodes(graph, nullptr, &n_nodes) == cudaSuccess && n_nodes > 0) {
-    launches = (int)n_nodes;  // every node of the captured pass is a kernel launch
-    n->launches[mode] = launches;
+    // kernel launches of the captured pass (it also holds a few memset and event-record nodes)
+    std::vector<cudaGraphNode_t> nodes(n_nodes);
+    int kernels = 0;
+    if (cudaGraphGetNodes(graph, nodes.data(), &n_nodes) == cudaSuccess)
+      for (size_t i = 0; i < n_nodes; ++i) {
+        cudaGraphNodeType t;
+        if (cudaGraphNodeGetType(nodes[i], &t) == cudaSuccess && t == cudaGraphNodeTypeKernel) ++kernels;
+      }
+    if (kernels > 0) { launches = kernels; n->launches[mode] = launches; }
   }
   e.mode = mode; e.batch = a.batch; memcpy(e.p, key, sizeof key); e.n_kernels = launches;
   cudaError_t ie = cudaGraphInstantiate(&e.exec, graph, 0);
