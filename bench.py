@@ -673,6 +673,30 @@ def run_profile_layer(args):
     print(f"profiled conv layer {L} ({args.profile_kind}), batch {B}: {s}x{s}, {ci}->{co}")
 
 
+def run_profile_pass(args):
+    """Three forward passes, then three forward+backward passes at the benchmark's batch, and nothing else:
+    the launch list of `ncu --metrics gpu__time_duration.sum` on this is the per-kernel share of a pass
+    (prints nothing the driver parses)."""
+    import torch
+    import seeded_inputs as si
+    import paper_1810_09868_b200 as pkg
+    params = si.vgg19_params(H, W, seed=0, bf16_exact=True)
+    net = pkg.Net(H, W, BATCH, pkg.VGG19_BF16, params=params)
+    x = torch.from_numpy(si.images(BATCH, H, W, seed=1, bf16_exact=True)).cuda().to(torch.bfloat16)
+    y = torch.from_numpy(si.labels(BATCH, seed=2)).cuda()
+    logits = torch.empty(BATCH, 1000, dtype=torch.float32, device="cuda")
+    grads = torch.empty(net.n_params, dtype=torch.float32, device="cuda")
+    loss = torch.empty(1, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    for _ in range(3):
+        pkg.vgg19_forward(net.handle, x, BATCH, logits, None, stream)
+    for _ in range(3):
+        pkg.vgg19_backward(net.handle, x, y, BATCH, grads, loss, None, stream)
+    net.sync_status(stream)
+    print(f"profiled 3 forward passes ({pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_FORWARD)} kernels each) and 3 "
+          f"forward+backward passes ({pkg.vgg19_launch_count(net.handle, pkg.VGG19_MODE_BACKWARD)} kernels each)")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -684,11 +708,15 @@ def main():
     ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"])
     ap.add_argument("--dry", action="store_true", help="multi-rank plumbing only, on CPU ranks (needs --backend gloo)")
     ap.add_argument("--profile-layer", type=int, default=0, help="run only this conv layer (1..16) a few times and exit")
+    ap.add_argument("--profile-pass", action="store_true", help="run three forward and three forward+backward passes and exit")
     ap.add_argument("--profile-batch", type=int, default=16)
     ap.add_argument("--profile-kind", default="fwd", choices=["fwd", "bwd"])
     args = ap.parse_args()
     if args.profile_layer:
         run_profile_layer(args)
+        return
+    if args.profile_pass:
+        run_profile_pass(args)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     if args.impl == "reference":

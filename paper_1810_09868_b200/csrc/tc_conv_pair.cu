@@ -31,14 +31,19 @@ constexpr int A_BYTES = BM * BK * 2;
 constexpr int kThreads = 192;
 constexpr int kSmemLimit = 227 * 1024;
 
-template <int BN>
+// MASK: the kernel applies a ReLU mask and keeps a mask tile in shared memory (one stage fewer).
+template <int BN, bool MASK>
 struct PairTile {
   static constexpr int B_BYTES = (BN / 2) * BK * 2;  // this CTA's half of the filter slice
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int OUT_BYTES = BM * 64 * 2;      // staging tile of the TMA store
-  static constexpr int STAGES = (kSmemLimit - 4608 - 2 * OUT_BYTES) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608 - 2 * OUT_BYTES) / STAGE_BYTES;
+  static constexpr int TILES = MASK ? 2 : 1;         // staging tile, mask tile
+  // beside the dynamic shared memory: alignment slack and barriers (1280 B) and the static part, which is the
+  // 2 KB bias table unless MASK (an input gradient has no bias)
+  static constexpr int kOther = MASK ? 1792 : 4608;
+  static constexpr int STAGES = (kSmemLimit - kOther - TILES * OUT_BYTES) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - kOther - TILES * OUT_BYTES) / STAGE_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;           // double-buffered accumulator
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_BYTES + 1024 + 256;  // staging tile + mask tile
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TILES * OUT_BYTES + 1024 + 256;
 };
 
 struct PairArgs {
@@ -84,16 +89,16 @@ __device__ __forceinline__ void red_max_bf16x8(bf16* dst, uint32_t a, uint32_t b
   asm volatile("red.global.max.noftz.v4.bf16x2 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-template <int BN, bool POOL>
+template <int BN, bool POOL, bool MASK>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_m, PairArgs a) {
-  using T = PairTile<BN>;
+  using T = PairTile<BN, MASK>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t out_smem = smem_base + T::STAGES * T::STAGE_BYTES;
   const uint32_t mask_smem = out_smem + T::OUT_BYTES;  // ReLU-mask tile of the chunk being finished (input gradient)
-  const uint32_t bars = mask_smem + T::OUT_BYTES;
+  const uint32_t bars = mask_smem + (MASK ? T::OUT_BYTES : 0);
   auto full_bar = [&](int s) { return bars + 8u * s; };                       // used in the even CTA
   auto empty_bar = [&](int s) { return bars + 8u * (T::STAGES + s); };        // both CTAs
   auto acc_full_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + b); };       // both CTAs
@@ -102,7 +107,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const uint32_t mask_bar = bars + 8u * (2 * T::STAGES + 5);  // this CTA's own
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ __align__(16) float bias_s[512];
+  __shared__ __align__(16) float bias_s[MASK ? 4 : 512];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -111,7 +116,8 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const int k_blocks = 9 * a.cin_blocks;
   const int total_work = a.main_tiles + (a.m_pairs * a.n_tiles - a.main_tiles) * a.tail_splits;
 
-  for (int i = threadIdx.x; i < a.Cout; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
+  if (!MASK)
+    for (int i = threadIdx.x; i < a.Cout; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < T::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -245,7 +251,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         return;
       }
     };
-    if (a.mask && issuer) request_mask(pair, 0);
+    if (MASK && issuer) request_mask(pair, 0);
     for (int w = pair; w < total_work; w += n_pairs, ++local) {
       const Work wk = get_work(w, a, k_blocks);
       const int buf = local & 1;
@@ -302,7 +308,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
-            x0 += bias_s[c_base + cc + j]; x1 += bias_s[c_base + cc + j + 1];
+            if (!MASK) { x0 += bias_s[c_base + cc + j]; x1 += bias_s[c_base + cc + j + 1]; }
             if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
             __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
             packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
@@ -315,7 +321,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             }
             continue;
           }
-          if (a.mask) {
+          if (MASK) {
             if (!mask_ready) {  // a failed wait leaves the chunk unmasked; the error word says so
               mbar_wait(mask_bar, mask_phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull);
               mask_phase ^= 1;
@@ -350,7 +356,7 @@ conv3x3_pair_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           // rows past the end of the tensor (last tile) are clipped by the copy engine
           tma_store_2d(&map_y, out_smem, c_base + c64, m_tile * BM);
           tma_store_commit();
-          if (a.mask) {
+          if (MASK) {
             mask_pending = false;
             if (c64 + 64 < BN) request_mask(w, c64 + 64); else request_mask(w + n_pairs, 0);
           }
@@ -429,12 +435,12 @@ __global__ void pair_tail_finish_kernel(const float* __restrict__ partial, int s
 }
 
 // CTA pairs of this kernel that can be resident at once (one pair per two SMs at most)
-template <int BN, bool POOL>
+template <int BN, bool POOL, bool MASK>
 cudaError_t resident_pairs(int* out) {
-  using T = PairTile<BN>;
+  using T = PairTile<BN, MASK>;
   static int max_pairs = 0;
   if (!max_pairs) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_pair_tc_kernel<BN, POOL>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_pair_tc_kernel<BN, POOL, MASK>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
@@ -448,7 +454,7 @@ cudaError_t resident_pairs(int* out) {
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr; cfg.numAttrs = 1;
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, conv3x3_pair_tc_kernel<BN, POOL>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, conv3x3_pair_tc_kernel<BN, POOL, MASK>, &cfg);
     if (e != cudaSuccess || n < 1) { cudaGetLastError(); n = sms / 2; }
     max_pairs = n < sms / 2 ? n : sms / 2;
     if (max_pairs < 1) max_pairs = 1;
@@ -476,9 +482,9 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
   if (launches) *launches = 0;
   if (!tc_conv3x3_pair_supported(s)) return cudaErrorInvalidValue;
   if (pooled && (mask || !relu || (s.H & 1) || (s.W & 1))) return cudaErrorInvalidValue;  // maxima of ReLU outputs only
+  if (mask && bias) return cudaErrorInvalidValue;  // a masked result is an input gradient: no bias
   if (!pooled && !out) return cudaErrorInvalidValue;
   constexpr int BN = 256;
-  using T = PairTile<BN>;
   CUtensorMap mx, mw, my, mm;
   if (!make_im2col_map(&mx, in, s.N, s.H, s.W, s.Cin, BM)) return cudaErrorInvalidValue;
   if (!make_tiled_map_2d(&mw, wt, (uint64_t)s.Cout, (uint64_t)9 * s.Cin, BN / 2)) return cudaErrorInvalidValue;
@@ -496,7 +502,8 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
   a.relu = relu ? 1 : 0;
   a.bias = bias; a.mask = mask; a.dev_error = dev_error; a.pooled = pooled;
   int cap = 0;
-  cudaError_t e = pooled ? resident_pairs<BN, true>(&cap) : resident_pairs<BN, false>(&cap);
+  cudaError_t e = pooled ? resident_pairs<BN, true, false>(&cap)
+                         : (mask ? resident_pairs<BN, false, true>(&cap) : resident_pairs<BN, false, false>(&cap));
   if (e != cudaSuccess) return e;
   if (pooled) {
     e = cudaMemsetAsync(pooled, 0, (size_t)s.N * (s.H / 2) * (s.W / 2) * s.Cout * sizeof(bf16), st);
@@ -524,8 +531,9 @@ cudaError_t tc_conv3x3_pair(const bf16* in, const bf16* wt, const float* bias, c
   }
   const int work = a.main_tiles + (tiles - a.main_tiles) * a.tail_splits;
   const int pairs = work < cap ? work : cap;
-  if (pooled) conv3x3_pair_tc_kernel<BN, true><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
-  else conv3x3_pair_tc_kernel<BN, false><<<2 * pairs, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
+  if (pooled) conv3x3_pair_tc_kernel<BN, true, false><<<2 * pairs, kThreads, PairTile<BN, false>::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
+  else if (mask) conv3x3_pair_tc_kernel<BN, false, true><<<2 * pairs, kThreads, PairTile<BN, true>::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
+  else conv3x3_pair_tc_kernel<BN, false, false><<<2 * pairs, kThreads, PairTile<BN, false>::SMEM_BYTES, st>>>(mx, mw, my, mm, a);
   e = cudaGetLastError();
   if (launches) *launches = 1;
   if (e != cudaSuccess || !a.partial) return e;

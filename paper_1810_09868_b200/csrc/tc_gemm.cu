@@ -641,10 +641,8 @@ cudaError_t tc_dense_dw(const bf16* dY, const bf16* X, float* dW, int M, int In,
   g.dev_error = dev_error; g.ldc = In; g.out_f = dW;
   g.sgd_copy = sgd_copy; g.sgd_lr = sgd_lr;
   const int m_tiles = (Out + BM - 1) / BM;
-  if (In % 256 == 0) {
-    g.n_tiles = In / 256;
-    return launch_gemm_tc<256, kMnMajor, kMnMajor>(ma, mb, g, m_tiles, 1, st);
-  }
+  // 128-column tiles: two of these one-tile CTAs fit an SM (98 KB of shared memory, 128 tensor-memory
+  // columns each), so one's prologue and loads hide behind the other's 64 KB store
   g.n_tiles = (In + 127) / 128;
   return launch_gemm_tc<128, kMnMajor, kMnMajor>(ma, mb, g, m_tiles, 1, st);
 }
