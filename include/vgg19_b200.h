@@ -54,7 +54,8 @@ typedef enum {
 enum {
   VGG19_FLAG_NO_GRAPH = 1,        /* enqueue kernels directly instead of replaying a CUDA graph */
   VGG19_FLAG_NO_TENSOR_CORES = 2, /* bf16 only: use the CUDA-core kernels for every layer */
-  VGG19_FLAG_NO_CTA_PAIRS = 4     /* one CTA per tile everywhere: no two-CTA (cta_group::2) kernels */
+  VGG19_FLAG_NO_CTA_PAIRS = 4,    /* one CTA per tile everywhere: no two-CTA (cta_group::2) kernels */
+  VGG19_FLAG_FIRST_FUSION = 8     /* forward-only passes run conv1_1 and conv1_2 as one kernel (vgg19_first_block_forward) */
 };
 
 typedef enum {
@@ -216,6 +217,20 @@ int vgg19_conv_layer_forward(vgg19_t *net, int32_t layer, const void *x, int32_t
  * is then never written; VGG19_ERR_ARG where it cannot. */
 int vgg19_conv_layer_forward_ex(vgg19_t *net, int32_t layer, const void *x, int32_t batch, void *y, void *pooled,
                                 uint8_t *pool_code, void *stream);
+
+/* The first block, conv1_1 -> conv1_2 (-> max-pool), as ONE kernel that never
+ * writes conv1_1's activation (the paper's point about the forward pass is
+ * that the whole of it fuses into one executable, section 7.2; here the two
+ * layers whose intermediate is the largest tensor of the network share a
+ * kernel: the second layer's input patches are computed on the fly from image
+ * patches).  Same result, bit for bit, as the two layers run one after the
+ * other.  A forward-only pass runs layers 1 and 2 this way when the network
+ * was created with VGG19_FLAG_FIRST_FUSION (off by default: on a B200 at batch
+ * 100 the one kernel takes 0.55 ms, the two it replaces 0.51 ms).  bf16 only,
+ * width a multiple of 14, height of 8; else VGG19_ERR_SHAPE.  images: device
+ * [batch][H][W][3] bf16; y2 (or NULL): conv1_2's output [batch][H][W][64];
+ * pooled (or NULL): its 2x2 max-pool.  Needs the forward workspace. */
+int vgg19_first_block_forward(vgg19_t *net, const void *images, int32_t batch, void *y2, void *pooled, void *stream);
 
 /* Gradients of that layer given dz = d(loss)/d(pre-activation) already
  * masked by the ReLU: dw fp32 [Cout][3][3][Cin], db fp32 [Cout], and (unless

@@ -15,7 +15,7 @@ VGG19_OK = 0
 VGG19_ERR_ARG, VGG19_ERR_SHAPE, VGG19_ERR_WORKSPACE = -1, -2, -3
 VGG19_ERR_CUDA, VGG19_ERR_DEVICE_TIMEOUT, VGG19_ERR_UNSUPPORTED_ARCH = -4, -5, -6
 VGG19_FP32, VGG19_BF16 = 0, 1
-VGG19_FLAG_NO_GRAPH, VGG19_FLAG_NO_TENSOR_CORES, VGG19_FLAG_NO_CTA_PAIRS = 1, 2, 4
+VGG19_FLAG_NO_GRAPH, VGG19_FLAG_NO_TENSOR_CORES, VGG19_FLAG_NO_CTA_PAIRS, VGG19_FLAG_FIRST_FUSION = 1, 2, 4, 8
 VGG19_MODE_FORWARD, VGG19_MODE_BACKWARD, VGG19_MODE_TRAIN = 0, 1, 2
 
 EXPORTS = (
@@ -23,7 +23,7 @@ EXPORTS = (
     "vgg19_get_params", "vgg19_set_params", "vgg19_workspace_bytes", "vgg19_bind_workspace",
     "vgg19_forward", "vgg19_backward", "vgg19_sgd_step", "vgg19_train_step", "vgg19_train_steps",
     "vgg19_set_dense_grads_event", "vgg19_io_bytes", "vgg19_forward_host", "vgg19_forward_host_async", "vgg19_backward_host",
-    "vgg19_conv_layer_forward", "vgg19_conv_layer_forward_ex", "vgg19_conv_layer_backward", "vgg19_conv_layer_backward_ex", "vgg19_saved_tensor", "vgg19_conv_wgrad_static", "vgg19_sync_status", "vgg19_selftest_wait_timeout", "vgg19_launch_count",
+    "vgg19_conv_layer_forward", "vgg19_conv_layer_forward_ex", "vgg19_first_block_forward", "vgg19_conv_layer_backward", "vgg19_conv_layer_backward_ex", "vgg19_saved_tensor", "vgg19_conv_wgrad_static", "vgg19_sync_status", "vgg19_selftest_wait_timeout", "vgg19_launch_count",
     "vgg19_describe", "vgg19_last_error",
 )
 
@@ -81,6 +81,7 @@ def load():
         "vgg19_conv_layer_forward": ([vp, i32, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_backward": ([vp, i32, vp, vp, i32, vp, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_forward_ex": ([vp, i32, vp, i32, vp, vp, vp, vp], ctypes.c_int),
+        "vgg19_first_block_forward": ([vp, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_backward_ex": ([vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp], ctypes.c_int),
         "vgg19_saved_tensor": ([vp, i32, i32, i32, ctypes.POINTER(sz), ctypes.POINTER(ctypes.c_int64)], ctypes.c_int),
         "vgg19_conv_wgrad_static": ([vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, ctypes.POINTER(sz), vp], ctypes.c_int),
@@ -231,6 +232,10 @@ def vgg19_conv_layer_backward(net, layer, x, dz, batch, dw, db, dx=None, stream=
 def vgg19_conv_layer_forward_ex(net, layer, x, batch, y, pooled=None, pool_code=None, stream=None):
     return _check(net, load().vgg19_conv_layer_forward_ex(net, layer, _ptr(x), batch, _ptr(y), _ptr(pooled),
                                                            _ptr(pool_code), _stream(stream)))
+
+
+def vgg19_first_block_forward(net, images, batch, y2=None, pooled=None, stream=None):
+    return _check(net, load().vgg19_first_block_forward(net, _ptr(images), batch, _ptr(y2), _ptr(pooled), _stream(stream)))
 
 
 def vgg19_conv_layer_backward_ex(net, layer, x, dz, batch, dw=None, db=None, dx=None, relu_mask=None, pool_code=None,

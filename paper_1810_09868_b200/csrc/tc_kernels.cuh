@@ -101,6 +101,14 @@ size_t tc_first_wgrad_scratch_elems(ConvShape s);
 cudaError_t tc_first_wgrad(const bf16* x8, const bf16* dz, float* dW, float* db, float* partial, ConvShape s, int* dev_error,
                            cudaStream_t st);
 
+// conv1_1 and conv1_2 (3 -> 64 -> 64 channels, bias and ReLU each) as one kernel that never writes conv1_1's
+// output (tc_conv_fused12.cu).  x8 from tc_pad_to8, w8 from tc_make_first_filter, wt2_tap_major the second
+// layer's tap-major filter; out (or null) the second layer's output, pooled (or null) its 2x2 max-pool.
+// s describes the first layer (Cin 3, Cout 64); W must be a multiple of 14 and H of 8.
+bool tc_conv12_fused_supported(ConvShape s);
+cudaError_t tc_conv12_fused(const bf16* x8, const bf16* w8, const float* bias1, const bf16* wt2_tap_major, const float* bias2,
+                            bf16* out, bf16* pooled, ConvShape s, int* dev_error, cudaStream_t st);
+
 // Self-test of the bounded-wait plumbing: one CTA of 32 threads initialises an mbarrier in shared
 // memory on which nothing ever arrives and waits for it with a limit of `limit_cycles` SM cycles; the
 // wait runs out, kDevTimeoutTest lands in dev_error and the kernel returns normally.  No TMA, no

@@ -375,11 +375,33 @@ struct Pass {
     }
   }
 
+  // conv1_1 -> conv1_2 as one kernel (neither layer's full-resolution output is stored): forward-only passes
+  bool first_block_fused_ok(int B) const {
+    const ConvLayer &c0 = n->conv[0], &c1 = n->conv[1];
+    return n->use_tc && p.valid && c1.Cin == 64 && c1.Cout == 64 &&
+           tc_conv12_fused_supported(ConvShape{B, c0.H, c0.W, c0.Cin, c0.Cout});
+  }
+  void first_block_fused(const T *x, int B, T *y2, T *pooled) {
+    const ConvLayer &c0 = n->conv[0], &c1 = n->conv[1];
+    ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c0.H * c0.W, st), 1);
+    x8_of = x;
+    ok(tc_conv12_fused((const bf16 *)buf(p.x8), n->w8, n->params + c0.b_off, n->tap_fwd + c1.dgrad_off, n->params + c1.b_off,
+                       (bf16 *)y2, (bf16 *)pooled, ConvShape{B, c0.H, c0.W, c0.Cin, c0.Cout}, n->dev_error, st), 1);
+  }
+
   void forward(const PassArgs &a) {
     const int B = a.batch;
     const T *x = static_cast<const T *>(a.images);
     int pi = 0;
-    for (int l = 0; l < kConvLayers; ++l) {
+    int first = 0;
+    // (opt-in: at batch 100 the fused kernel measures 0.55 ms against 0.51 ms for the two kernels it replaces)
+    if (!keep_activations && !a.grads && (n->cfg.flags & VGG19_FLAG_FIRST_FUSION) && n->conv[1].pool_after &&
+        first_block_fused_ok(B)) {
+      first_block_fused(x, B, nullptr, buf(p.pooled[0]));
+      x = buf(p.pooled[0]);
+      pi = 1; first = 2;
+    }
+    for (int l = first; l < kConvLayers; ++l) {
       T *y = buf(p.act[l]);
       T *pooled = n->conv[l].pool_after ? buf(p.pooled[pi]) : nullptr;
       // a pass that will run backward stores, with each pooled tensor, where every window's maximum sat
@@ -976,6 +998,22 @@ int vgg19_conv_layer_forward_ex(vgg19_t *n, int32_t layer, const void *x, int32_
     e = ps.err;
   }
   if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  return VGG19_OK;
+}
+
+int vgg19_first_block_forward(vgg19_t *n, const void *images, int32_t batch, void *y2, void *pooled, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (!images || (!y2 && !pooled)) return fail(n, VGG19_ERR_ARG, "null images, or neither output asked for");
+  int rc = check_batch(n, batch, VGG19_MODE_FORWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  if (n->cfg.dtype != VGG19_BF16) return fail(n, VGG19_ERR_ARG, "the fused first block exists for the bf16 configuration only");
+  n->other_pass = true;
+  Pass<bf16> ps{n, make_plan(n, batch, VGG19_MODE_FORWARD), static_cast<cudaStream_t>(stream)};
+  if (!ps.first_block_fused_ok(batch))
+    return fail(n, VGG19_ERR_SHAPE, "no fused first block at %dx%d (width a multiple of 14, height of 8)", n->cfg.height,
+                n->cfg.width);
+  ps.first_block_fused((const bf16 *)images, batch, (bf16 *)y2, (bf16 *)pooled);
+  if (ps.err != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(ps.err));
   return VGG19_OK;
 }
 

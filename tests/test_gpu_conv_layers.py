@@ -211,3 +211,60 @@ def test_block_ending_layers_pool_in_their_epilogue(net224, layer, S, Cin, Cout)
     Wt, b = layer_params(p, net, params, layer)
     ref = oracle.maxpool2x2_fwd(oracle.round_bf16(oracle.relu_fwd(oracle.conv3x3_fwd(x[:1], Wt, b))))
     assert rel_l2(pooled[:1].float().cpu().numpy(), ref) <= 1e-3
+
+
+def test_first_block_as_one_kernel(net224):
+    """conv1_1 -> conv1_2 (-> pool) in one kernel that never stores conv1_1's activation (what a forward-only
+    pass runs): against the checker's two convolutions with the bf16 store between them, and against the two
+    separate kernels."""
+    p, net, params = net224
+    B = 3
+    x = si.images(B, 224, 224, seed=1, bf16_exact=True)
+    xd = torch.from_numpy(x).to(DEV).to(torch.bfloat16)
+    st = torch.cuda.current_stream()
+    y2 = torch.full((B, 224, 224, 64), float("nan"), dtype=torch.bfloat16, device=DEV)
+    pooled = torch.full((B, 112, 112, 64), float("nan"), dtype=torch.bfloat16, device=DEV)
+    p.vgg19_first_block_forward(net.handle, xd, B, y2, pooled, st)
+    pooled_only = torch.full((B, 112, 112, 64), float("nan"), dtype=torch.bfloat16, device=DEV)
+    p.vgg19_first_block_forward(net.handle, xd, B, None, pooled_only, st)
+    net.sync_status()
+    # the two separate kernels
+    y1 = torch.empty((B, 224, 224, 64), dtype=torch.bfloat16, device=DEV)
+    y2_two = torch.empty_like(y2)
+    p.vgg19_conv_layer_forward(net.handle, 1, xd, B, y1, None, st)
+    p.vgg19_conv_layer_forward(net.handle, 2, y1, B, y2_two, None, st)
+    net.sync_status()
+    assert torch.isfinite(y2.float()).all()
+    same = torch.equal(y2, y2_two)
+    print(f"fused first block vs two kernels: {'bit-identical' if same else 'rel-L2 %.2e' % rel_l2(y2.float().cpu().numpy(), y2_two.float().cpu().numpy())}")
+    assert same or rel_l2(y2.float().cpu().numpy(), y2_two.float().cpu().numpy()) <= 1e-3
+    want_pool = torch.nn.functional.max_pool2d(y2.float().permute(0, 3, 1, 2), 2).permute(0, 2, 3, 1)
+    assert torch.equal(pooled.float(), want_pool) and torch.equal(pooled_only, pooled)
+    # the checker, on one image (edges and corners of the image included)
+    W1, b1 = layer_params(p, net, params, 1)
+    W2, b2 = layer_params(p, net, params, 2)
+    r1 = oracle.round_bf16(oracle.relu_fwd(oracle.conv3x3_fwd(x[:1], W1, b1)))
+    r2 = oracle.round_bf16(oracle.relu_fwd(oracle.conv3x3_fwd(r1, W2, b2)))
+    got = y2[:1].float().cpu().numpy()
+    assert rel_l2(got, r2) <= 1e-3
+    for sl in (np.s_[0, 0, :, :], np.s_[0, -1, :, :], np.s_[0, :, 0, :], np.s_[0, :, -1, :]):
+        assert rel_l2(got[sl], r2[sl]) <= 2e-3
+
+
+def test_forward_pass_with_the_fused_first_block_is_bit_identical(net224):
+    """A network created with VGG19_FLAG_FIRST_FUSION runs layers 1 and 2 of a forward-only pass as the one fused
+    kernel; the logits must equal, bit for bit, those of the default schedule."""
+    p, net, params = net224
+    B = 2
+    xd = torch.from_numpy(si.images(B, 224, 224, seed=7, bf16_exact=True)).to(DEV).to(torch.bfloat16)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        want = net.forward(xd, stream=s).clone()
+    net.sync_status(s)
+    fused = p.Net(224, 224, B, p.VGG19_BF16, params=params, flags=p.VGG19_FLAG_FIRST_FUSION, mode=p.VGG19_MODE_FORWARD)
+    with torch.cuda.stream(s):
+        got = fused.forward(xd, stream=s).clone()
+    fused.sync_status(s)
+    assert p.vgg19_launch_count(fused.handle, p.VGG19_MODE_FORWARD) == p.vgg19_launch_count(net.handle, p.VGG19_MODE_FORWARD) - 1
+    assert torch.equal(got, want)
+    fused.close()
