@@ -69,22 +69,28 @@ constexpr int kStoreStagingBytes = 2 * BM * 128;  // two tiles of 128 rows x 32 
 
 // PAIR: two CTAs (a cluster, tcgen05 cta_group::2) compute a 256 x BN tile with one MMA stream; each
 // stages its own 128 rows of A and half of the B tile.
-template <int BN, bool PAIR>
+// WIDE (pairs only): a second accumulator of 128 columns beside the BN = 256 one, fed by the same A tile - the
+// pair's tile is 256 x 384, and the A operand, half of what a pair loads per K block, is loaded once for both.
+template <int BN, bool PAIR, bool WIDE = false>
 __host__ __device__ constexpr int stage_bytes() {
   // BN = 80 is the 8-channel form, whose K blocks are 128 pixels: ten taps x 128 pixels x 16 bytes
-  return BN == 80 ? A_BYTES + 10 * 2048 : A_BYTES + (PAIR ? BN / 2 : BN) * BK * 2;
+  return BN == 80 ? A_BYTES + 10 * 2048 : A_BYTES + (PAIR ? (BN + (WIDE ? 128 : 0)) / 2 : BN) * BK * 2;
 }
 
-template <int BN, int AMODE, int BMODE, bool PAIR>
+template <int BN, int AMODE, int BMODE, bool PAIR, bool WIDE = false>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, GemmArgs g) {
   static_assert(!PAIR || (AMODE == kMnMajor && BMODE == kMnMajorIm2col && BN % 128 == 0), "pairs: filter gradient only");
-  constexpr int STAGE = stage_bytes<BN, PAIR>();
-  constexpr int B_GROUPS = (PAIR ? BN / 2 : BN) / 64;  // 64-column groups of B this CTA stages
+  static_assert(!WIDE || (PAIR && BN == 256), "the second accumulator goes with the 256-column pair tile");
+  constexpr int BN2 = WIDE ? 128 : 0;   // columns of the second accumulator
+  constexpr int BNT = BN + BN2;         // columns of the whole tile
+  constexpr int STAGE = stage_bytes<BN, PAIR, WIDE>();
+  constexpr int B_GROUPS1 = (PAIR ? BN / 2 : BN) / 64;  // 64-column groups of B this CTA stages for the first accumulator
+  constexpr int B_GROUPS = B_GROUPS1 + BN2 / 128;       // ... and in all (one more for the second)
   // filter gradient: 32 spare columns after the tile where the column sums of A can accumulate.  The
   // dense layers need none, and with 256 columns instead of 512 two of their CTAs share an SM.
-  constexpr int COLS = BN + (BMODE == kMnMajorIm2col ? 32 : 0);
+  constexpr int COLS = BNT + (BMODE == kMnMajorIm2col ? 32 : 0);
   constexpr int TMEM_COLS = COLS <= 64 ? 64 : (COLS <= 128 ? 128 : (COLS <= 256 ? 256 : 512));
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -102,7 +108,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // position in the pair; rank 0 issues the MMAs
   const int tile_index = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int m_tile = (tile_index / g.n_tiles) * (PAIR ? 2 : 1) + (int)rank, n_tile = tile_index % g.n_tiles;
-  const int m0 = m_tile * BM, n0 = n_tile * BN;
+  const int m0 = m_tile * BM, n0 = n_tile * BNT;
   const int kb0 = blockIdx.y * g.kb_per_split;
   const int kb1 = min(g.k_blocks, kb0 + g.kb_per_split);
   // K blocks kb = n_tile (mod n_tiles) are the ones whose column sums this CTA adds
@@ -158,7 +164,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (BMODE == kMnMajorIm2col) {
 #pragma unroll
           for (int q = 0; q < B_GROUPS; ++q) {
-            const int j = n0 + 64 * ((int)rank * B_GROUPS + q), tap = j / g.Cin;
+            // first accumulator: this CTA's half of its BN columns; second: its 64 of the 128 columns that follow
+            const int j = q < B_GROUPS1 ? n0 + 64 * ((int)rank * B_GROUPS1 + q) : n0 + BN + 64 * (int)rank, tap = j / g.Cin;
             grp_c[q] = j - tap * g.Cin; grp_r[q] = tap / 3; grp_s[q] = tap - 3 * (tap / 3);
           }
         }
@@ -260,11 +267,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
           for (int k = 1; k < BK / 16; ++k)
             umma_bf16_pair_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), idesc);
-          if (kb == db_next) {
-            umma_bf16_pair(tmem_base + BN, da, d_ones, idesc_ones, kb != db_first ? 1u : 0u);
+          if (WIDE) {
+            // the same A tile against this pair's other 128 columns (one 64-column group per CTA, behind
+            // the first accumulator's groups in the stage)
+            constexpr uint32_t idesc2 = umma_idesc_bf16(2 * BM, 128, AMODE != kKMajor, BMODE != kKMajor);
+            const uint64_t db2 = smem_desc_sw128(sb + B_GROUPS1 * GROUP_BYTES, GROUP_BYTES);
+            umma_bf16_pair(tmem_base + BN, da, db2, idesc2, kb > kb0 ? 1u : 0u);
 #pragma unroll
             for (int k = 1; k < BK / 16; ++k)
-              umma_bf16_pair_acc(tmem_base + BN, desc_advance(da, k * a_step), d_ones, idesc_ones);
+              umma_bf16_pair_acc(tmem_base + BN, desc_advance(da, k * a_step), desc_advance(db2, k * b_step), idesc2);
+          }
+          if (kb == db_next) {
+            umma_bf16_pair(tmem_base + BNT, da, d_ones, idesc_ones, kb != db_first ? 1u : 0u);
+#pragma unroll
+            for (int k = 1; k < BK / 16; ++k)
+              umma_bf16_pair_acc(tmem_base + BNT, desc_advance(da, k * a_step), d_ones, idesc_ones);
             db_next += g.n_tiles;
           }
           umma_commit_pair(empty_bar(stage), 3);  // frees the stage in both CTAs
@@ -318,7 +335,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       };
       if (fold) fetch(0);
 #pragma unroll 1
-      for (int cc = 0; cc < BN; cc += 32) {
+      for (int cc = 0; cc < BNT; cc += 32) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)cc, v);
         tmem_ld_wait();
@@ -326,7 +343,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           float4 w[8];
 #pragma unroll
           for (int q = 0; q < 8; ++q) w[q] = w_next[q];
-          if (cc + 32 < BN) fetch(cc + 32);
+          if (cc + 32 < BNT) fetch(cc + 32);
           if (row_ok && n0 + cc < g.N) {
             uint32_t h[16];
 #pragma unroll
@@ -362,7 +379,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (got_acc && !g.tma_store) {
       tc_fence_after();
 #pragma unroll 1
-      for (int cc = 0; cc < BN; cc += 32) {
+      for (int cc = 0; cc < BNT; cc += 32) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)cc, v);
         tmem_ld_wait();
@@ -415,7 +432,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (got_acc) {
       if (BMODE == kMnMajorIm2col && g.db_partial) {
         uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)BN, v);
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)BNT, v);
         tmem_ld_wait();
         if (row_ok)
           g.db_partial[((long)blockIdx.y * g.n_tiles + n_tile) * g.M + m] = db_first < kb1 ? __uint_as_float(v[0]) : 0.f;
@@ -500,10 +517,10 @@ void plan_split(int mn_tiles, int k_blocks, int* splits, int* kb_per_split, int 
 }
 
 // m_tiles counts tiles of 128 rows, or of 256 rows (CTA pairs) with PAIR
-template <int BN, int AMODE, int BMODE, bool PAIR = false>
+template <int BN, int AMODE, int BMODE, bool PAIR = false, bool WIDE = false>
 cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArgs g, int m_tiles, int splits,
                            cudaStream_t st) {
-  constexpr int STAGE = stage_bytes<BN, PAIR>();
+  constexpr int STAGE = stage_bytes<BN, PAIR, WIDE>();
   constexpr int kExtra = 1024 + 256 + 1024;  // alignment slack, barriers, block of ones
   // Raw fp32 output (split-K partial sums, or a result without bias / ReLU / mask) leaves by TMA store
   // where whole 128-row boxes cannot run into rows that belong to someone else: a single result
@@ -523,7 +540,7 @@ cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArg
   constexpr int max_stages = kBudget / STAGE > kMaxStages ? kMaxStages : kBudget / STAGE;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, AMODE, BMODE, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, AMODE, BMODE, PAIR, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          max_stages * STAGE + kExtra + kStoreStagingBytes);
     if (e != cudaSuccess) return e;
     configured = true;
@@ -540,10 +557,10 @@ cudaError_t launch_gemm_tc(const CUtensorMap& ma, const CUtensorMap& mb, GemmArg
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, AMODE, BMODE, PAIR>, ma, mb, mc, g);
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, AMODE, BMODE, PAIR, WIDE>, ma, mb, mc, g);
   }
   dim3 grid(m_tiles * g.n_tiles, splits);
-  gemm_tc_kernel<BN, AMODE, BMODE, PAIR><<<grid, kThreads, smem, st>>>(ma, mb, mc, g);
+  gemm_tc_kernel<BN, AMODE, BMODE, PAIR, WIDE><<<grid, kThreads, smem, st>>>(ma, mb, mc, g);
   return cudaGetLastError();
 }
 
@@ -654,14 +671,15 @@ namespace {
 // 192 columns (three 64-channel groups) divide 9*Cin for every Cin that is a multiple of 64; with 128
 // input channels they measured faster than 128-column tiles, CTA pairs included (0.43 -> 0.34 ms on layer 4)
 int wgrad_bn(int Cin) { return Cin % 256 == 0 ? 256 : 192; }
-// CTA pairs take 256 output channels per tile
-bool wgrad_pair(ConvShape s, bool pairs) { return pairs && s.Cout % 256 == 0 && s.Cin % 256 == 0; }
+// CTA pairs take 256 output channels and 384 columns per tile (two accumulators, 256 and 128 columns wide, fed by
+// one dz tile); 9 * Cin divides into such tiles when Cin is a multiple of 128
+bool wgrad_pair(ConvShape s, bool pairs) { return pairs && s.Cout % 256 == 0 && s.Cin % 128 == 0; }
 // m_tiles: tiles of 128 output channels, or of 256 with CTA pairs
 void wgrad_plan(ConvShape s, bool pairs, int* m_tiles, int* n_tiles, int* k_blocks, int* splits, int* per) {
   const long P = (long)s.N * s.H * s.W;
   const bool pair = wgrad_pair(s, pairs);
   *m_tiles = pair ? s.Cout / 256 : (s.Cout + BM - 1) / BM;
-  *n_tiles = 9 * s.Cin / wgrad_bn(s.Cin);
+  *n_tiles = pair ? 9 * s.Cin / 384 : 9 * s.Cin / wgrad_bn(s.Cin);
   *k_blocks = (int)((P + BK - 1) / BK);
   plan_split(*m_tiles * *n_tiles, *k_blocks, splits, per, pair ? 2 : 1);
 }
@@ -703,13 +721,9 @@ cudaError_t tc_conv3x3_wgrad(const bf16* x, const bf16* dz, float* dW, float* db
   if (db) g.db_partial = partial + (splits == 1 ? 0 : (size_t)splits * s.Cout * 9 * s.Cin);
   cudaError_t e;
   const bool pair = wgrad_pair(s, pairs);
-  switch (BN) {
-    case 256:
-      e = pair ? launch_gemm_tc<256, kMnMajor, kMnMajorIm2col, true>(ma, mb, g, m_tiles, splits, st)
-               : launch_gemm_tc<256, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st);
-      break;
-    default: e = launch_gemm_tc<192, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st); break;
-  }
+  if (pair) e = launch_gemm_tc<256, kMnMajor, kMnMajorIm2col, true, true>(ma, mb, g, m_tiles, splits, st);
+  else if (BN == 256) e = launch_gemm_tc<256, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st);
+  else e = launch_gemm_tc<192, kMnMajor, kMnMajorIm2col>(ma, mb, g, m_tiles, splits, st);
   if (e != cudaSuccess) return e;
   if (splits == 1) {
     if (!db) return e;

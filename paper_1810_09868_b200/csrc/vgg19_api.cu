@@ -1135,7 +1135,7 @@ int vgg19_describe(const vgg19_t *n, char *out, size_t cap) {
     const char *wgrad = !n->use_tc ? "simt"
                         : l == 0 ? (tc_first_conv_supported(sh) ? "tcgen05:gemm-8ch" : "simt")
                         : tc_wgrad_patch_supported(sh) ? "tcgen05:patch"
-                        : tc_wgrad_supported(sh) ? (n->use_pair && c.Cin % 256 == 0 && c.Cout % 256 == 0 ? "tcgen05:gemm-pair" : "tcgen05:gemm")
+                        : tc_wgrad_supported(sh) ? (n->use_pair && c.Cin % 128 == 0 && c.Cout % 256 == 0 ? "tcgen05:gemm-pair" : "tcgen05:gemm")
                         : "simt";
     snprintf(line, sizeof line, "conv%-2d %3dx%-3d %3d->%-3d +bias +relu%s  fwd=%s dgrad=%s wgrad=%s\n",
              l + 1, c.H, c.W, c.Cin, c.Cout, c.pool_after ? " +maxpool2x2" : "", fwd, dgrad, wgrad);
