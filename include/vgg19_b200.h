@@ -43,7 +43,8 @@ typedef enum {
   VGG19_ERR_WORKSPACE = -3,       /* no workspace bound, or too small */
   VGG19_ERR_CUDA = -4,            /* a CUDA runtime/driver call failed */
   VGG19_ERR_DEVICE_TIMEOUT = -5,  /* a bounded device-side wait ran out */
-  VGG19_ERR_UNSUPPORTED_ARCH = -6 /* the device is not compute capability 10.x */
+  VGG19_ERR_UNSUPPORTED_ARCH = -6,/* the device is not compute capability 10.x */
+  VGG19_ERR_RANGE = -7            /* VGG19_FLAG_SPLIT_F16: an activation beyond fp16's range (reported by vgg19_sync_status) */
 } vgg19_status;
 
 typedef enum {
@@ -55,7 +56,14 @@ enum {
   VGG19_FLAG_NO_GRAPH = 1,        /* enqueue kernels directly instead of replaying a CUDA graph */
   VGG19_FLAG_NO_TENSOR_CORES = 2, /* bf16 only: use the CUDA-core kernels for every layer */
   VGG19_FLAG_NO_CTA_PAIRS = 4,    /* one CTA per tile everywhere: no two-CTA (cta_group::2) kernels */
-  VGG19_FLAG_FIRST_FUSION = 8     /* forward-only passes run conv1_1 and conv1_2 as one kernel (vgg19_first_block_forward) */
+  VGG19_FLAG_FIRST_FUSION = 8,    /* forward-only passes run conv1_1 and conv1_2 as one kernel (vgg19_first_block_forward) */
+  /* fp32 only: forward-only passes (vgg19_forward*, vgg19_conv_layer_forward*) run layers 2..16 and the dense
+   * layers on tensor cores, every fp32 value carried as two fp16 terms (hi = fp16(v), lo = fp16(v - hi)) and
+   * every product formed as hi*hi + hi*lo + lo*hi in an fp32 accumulator: 22 of fp32's 24 mantissa bits per
+   * operand.  Activations must stay within fp16's range (65504): one beyond it makes vgg19_sync_status
+   * return VGG19_ERR_RANGE.  Backward and training passes keep the CUDA-core kernels.  The paper runs its
+   * fp32 network (section 7.2) on CPU and GPU back ends and has no counterpart of this. */
+  VGG19_FLAG_SPLIT_F16 = 16
 };
 
 typedef enum {

@@ -13,9 +13,10 @@ from . import build as _build
 
 VGG19_OK = 0
 VGG19_ERR_ARG, VGG19_ERR_SHAPE, VGG19_ERR_WORKSPACE = -1, -2, -3
-VGG19_ERR_CUDA, VGG19_ERR_DEVICE_TIMEOUT, VGG19_ERR_UNSUPPORTED_ARCH = -4, -5, -6
+VGG19_ERR_CUDA, VGG19_ERR_DEVICE_TIMEOUT, VGG19_ERR_UNSUPPORTED_ARCH, VGG19_ERR_RANGE = -4, -5, -6, -7
 VGG19_FP32, VGG19_BF16 = 0, 1
 VGG19_FLAG_NO_GRAPH, VGG19_FLAG_NO_TENSOR_CORES, VGG19_FLAG_NO_CTA_PAIRS, VGG19_FLAG_FIRST_FUSION = 1, 2, 4, 8
+VGG19_FLAG_SPLIT_F16 = 16
 VGG19_MODE_FORWARD, VGG19_MODE_BACKWARD, VGG19_MODE_TRAIN = 0, 1, 2
 
 EXPORTS = (

@@ -28,6 +28,7 @@ enum DeviceError : int {
   kDevTimeoutTmemFree = 4,  // MMA issuer waited too long for a drained accumulator
   kDevTimeoutTest = 5,      // the self-test kernel's wait on a barrier nobody arrives on
   kDevBadLabel = 64,        // a label outside [0, classes): not a timeout, reported as a bad argument
+  kDevSplitRange = 65,      // fp32 configuration on tensor cores: an activation beyond fp16's range
 };
 
 // ---- CUDA-core kernels (simt_kernels.cu) ---------------------------------
@@ -130,5 +131,21 @@ cudaError_t sgd_update(float* params, const float* grads, T* params_t, float lr,
 cudaError_t set_scalar(float* dst, float v, cudaStream_t st);
 template <typename T>
 cudaError_t make_dgrad_filter(const float* w, T* wt_t, int Cin, int Cout, cudaStream_t st);
+
+// fp32 tensors as pairs of fp16 terms (split_kernels.cu): a row of C values as [hi | lo], hi = fp16(v),
+// lo = fp16(v - hi), the same bytes as the fp32 row (the 16-bit words are passed as `half16`).  split_rows /
+// merge_rows convert between the forms (dst may be src); C must divide 4096; a value beyond fp16's range sets
+// kDevSplitRange in *dev_error.  maxpool_split pools [N][H][W][2C]; with rows_per_image the output is one row
+// [all hi | all lo] per image, the form a dense layer reads.  split_weights turns rows of K weights, scaled
+// by kSplitWeightScale, into rows [hi | lo | hi] of 3K.
+typedef unsigned short half16;
+// Weights are split after scaling by this power of two (exact), so that the lo terms of weights around 1e-2
+// stay above fp16's smallest normal number; the kernels that multiply by them scale their sums back.
+constexpr float kSplitWeightScale = 64.f;
+bool split_rows_supported(int C);
+cudaError_t split_rows(const float* src, half16* dst, long rows, int C, int* dev_error, cudaStream_t st);
+cudaError_t merge_rows(const half16* src, float* dst, long rows, int C, cudaStream_t st);
+cudaError_t maxpool_split(const half16* x, half16* y, int N, int H, int W, int C, bool rows_per_image, cudaStream_t st);
+cudaError_t split_weights(const float* w, half16* out, long rows, int K, cudaStream_t st);
 
 }  // namespace vgg

@@ -64,6 +64,10 @@ struct GemmArgs {
   // w - lr * D, and sgd_copy receives their bf16 rounding.  lr is read from device memory.
   bf16* sgd_copy;
   const float* sgd_lr;
+  // fp32 product from split operands (K-major A, fp16 terms): A holds [hi | lo] per row, a_wrap K blocks each; B
+  // holds [hi | lo | hi] of the weights times kSplitWeightScale.  K blocks [0, 2 * a_wrap) read A's hi term (the
+  // second group wraps back), the rest its lo term; the sum is scaled back before the bias is added.
+  int a_wrap;
 };
 constexpr int kStoreStagingBytes = 2 * BM * 128;  // two tiles of 128 rows x 32 fp32
 
@@ -195,7 +199,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         mbar_expect_tx(full_bar(stage), BMODE == kMnMajorIm2colC8 ? A_BYTES + 9 * 2048 : STAGE);
         if (AMODE == kKMajor) {
-          tma_load_2d(sa, &map_a, full_bar(stage), kb * BK, m0);
+          tma_load_2d(sa, &map_a, full_bar(stage), (g.a_wrap && kb >= g.a_wrap ? kb - g.a_wrap : kb) * BK, m0);
         } else if (BMODE == kMnMajorIm2colC8) {
           tma_load_2d(sa, &map_a, full_bar(stage), m0, kb * 2 * BK);
           tma_load_2d(sa + GROUP_BYTES, &map_a, full_bar(stage), m0, kb * 2 * BK + BK);
@@ -287,10 +291,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           umma_commit_pair(empty_bar(stage), 3);  // frees the stage in both CTAs
         } else {
           constexpr int k_steps = BMODE == kMnMajorIm2colC8 ? 2 * BK / 16 : BK / 16;
-          umma_bf16(tmem_base, da, db, idesc, kb > kb0 ? 1u : 0u);
+          // split operands are fp16 (the instruction takes the element type from the descriptor)
+          const uint32_t id = g.a_wrap ? umma_idesc_f16(BM, BN, AMODE != kKMajor, BMODE != kKMajor) : idesc;
+          umma_bf16(tmem_base, da, db, id, kb > kb0 ? 1u : 0u);
 #pragma unroll
           for (int k = 1; k < k_steps; ++k)
-            umma_bf16_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), idesc);
+            umma_bf16_acc(tmem_base, desc_advance(da, k * a_step), desc_advance(db, k * b_step), id);
           if (kb == db_next) {
             umma_bf16(tmem_base + BN, da, d_ones, idesc_ones, kb != db_first ? 1u : 0u);
 #pragma unroll
@@ -401,6 +407,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               x[e] = __uint_as_float(v[j + e]);
+              if (g.a_wrap) x[e] *= 1.f / kSplitWeightScale;
               if (g.bias) x[e] += __ldg(g.bias + n + j + e);
               if (g.relu) x[e] = fmaxf(x[e], 0.f);
             }
@@ -456,7 +463,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 __global__ void splitk_finish_kernel(const float* __restrict__ partial, int splits, long MN, int N,
                                      const float* __restrict__ bias, int relu, const bf16* __restrict__ mask,
                                      bf16* out_h, float* out_f, const float* __restrict__ db_partial, int db_parts,
-                                     int M, float* db) {
+                                     int M, float* db, float scale) {
   const long t = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (db && t < M) {
     float s = 0.f;
@@ -483,6 +490,7 @@ __global__ void splitk_finish_kernel(const float* __restrict__ partial, int spli
   const int n = (int)(i % N);
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
+    x[e] *= scale;  // 1 except for sums of split operands
     if (bias) x[e] += bias[n + e];
     if (relu) x[e] = fmaxf(x[e], 0.f);
     if (mask && !(__bfloat162float(mask[i + e]) > 0.f)) x[e] = 0.f;
@@ -569,7 +577,8 @@ cudaError_t finish(const GemmArgs& g, int splits, const float* bias, bool relu, 
   const long MN = (long)g.M * g.N;
   splitk_finish_kernel<<<(unsigned)((MN / 4 + 255) / 256), 256, 0, st>>>(g.partial, splits, MN, g.N, bias, relu ? 1 : 0,
                                                                           mask, out_h, out_f, g.db_partial,
-                                                                          splits * g.n_tiles, g.M, db);
+                                                                          splits * g.n_tiles, g.M, db,
+                                                                          g.a_wrap ? 1.f / kSplitWeightScale : 1.f);
   return cudaGetLastError();
 }
 
@@ -622,6 +631,34 @@ cudaError_t tc_dense_forward(const bf16* X, const bf16* Wt, const float* bias, b
   cudaError_t e = launch_gemm_tc<128, kKMajor, kKMajor>(ma, mb, g, m_tiles, splits, st);
   if (e != cudaSuccess) return e;
   return finish(g, splits, bias, relu, nullptr, out_h, out_f, st);
+}
+
+constexpr int kSplitChunkBlocks = 8;
+// fp32 Y = [relu](X W^T + b) from split operands: X [M][2 * In] = [x_hi | x_lo], Ws [Out][3 * In] =
+// [w_hi | w_lo | w_hi] (fp16 terms); three products x_hi w_hi + x_hi w_lo + x_lo w_hi in one fp32 accumulator
+cudaError_t tc_dense_forward_split(const half16* X, const half16* Ws, const float* bias, float* out_f, float* partial,
+                                   int M, int In, int Out, bool relu, int* dev_error, cudaStream_t st) {
+  if (In % BK != 0) return cudaErrorInvalidValue;
+  CUtensorMap ma, mb;
+  if (!make_tiled_map_2d(&ma, X, (uint64_t)M, (uint64_t)2 * In, BM)) return cudaErrorInvalidValue;
+  if (!make_tiled_map_2d(&mb, Ws, (uint64_t)Out, (uint64_t)3 * In, 128)) return cudaErrorInvalidValue;
+  GemmArgs g{};
+  g.M = M; g.N = Out; g.k_blocks = 3 * In / BK; g.n_tiles = (Out + 127) / 128; g.a_wrap = In / BK;
+  g.dev_error = dev_error; g.ldc = Out;
+  const int m_tiles = (M + BM - 1) / BM;
+  // The tensor core's fp32 accumulation truncates, an error that grows with the length of the chain: K is cut
+  // into splits of kSplitChunkBlocks blocks (32 MMAs) whatever the tile count, and the finishing kernel adds
+  // the partial sums with round-to-nearest fp32 additions.
+  g.kb_per_split = kSplitChunkBlocks;
+  const int splits = (g.k_blocks + kSplitChunkBlocks - 1) / kSplitChunkBlocks;
+  g.partial = partial;
+  cudaError_t e = launch_gemm_tc<128, kKMajor, kKMajor>(ma, mb, g, m_tiles, splits, st);
+  if (e != cudaSuccess) return e;
+  return finish(g, splits, bias, relu, nullptr, nullptr, out_f, st);
+}
+
+size_t tc_dense_split_scratch_elems(int M, int In, int Out) {
+  return (size_t)((3 * In / BK + kSplitChunkBlocks - 1) / kSplitChunkBlocks) * M * Out;
 }
 
 // dX = (dY W) [* (mask > 0)]: dY [M][Out], W [Out][In]

@@ -29,6 +29,8 @@
 
 #include <mutex>
 
+#include <cuda_fp16.h>
+
 #include "tc_common.cuh"
 
 namespace vgg {
@@ -172,6 +174,7 @@ constexpr int BK = 64;              // channels per K block (one 128-byte swizzl
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int kThreads = 192;
 constexpr int kSmemLimit = 227 * 1024;
+constexpr int kSplitChunk = 8;      // SPLIT: K blocks (of 64) per accumulation chain in tensor memory: 32 MMAs
 
 template <int BN>
 struct ConvTile {
@@ -197,11 +200,19 @@ struct ConvArgs {
   const bf16* mask;
   bf16* out;
   int* dev_error;
+  int split_blocks;  // SPLIT: 64-channel blocks of one term of the input (logical Cin / 64)
 };
 
 constexpr int PW = 16, PH = 8;  // patch of a tile in patch mode (PW * PH = BM)
 
-template <int BN>
+// SPLIT: fp32 convolution as three fp16 products.  Every fp32 value v travels as two fp16 terms, hi = fp16(v) and
+// lo = fp16(v - hi), stored per pixel as [hi of all channels | lo of all channels].  The K loop runs over three
+// groups of channel blocks per tap: x_hi * w_hi, x_hi * w_lo, x_lo * w_hi (the filter copy holds [w_hi | w_lo | w_hi]
+// per tap, of the weights times kSplitWeightScale; the input's channel block wraps back by one term after the
+// first group), all into the same fp32 accumulator; the epilogue scales the sum back, adds the bias, applies
+// the ReLU, splits the result again and stores the two terms.  A result beyond fp16's range is reported in
+// *dev_error (kDevSplitRange).
+template <int BN, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                   const __grid_constant__ CUtensorMap map_y, ConvArgs a) {
@@ -271,10 +282,12 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
               if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_flag, a.dev_error, kDevTimeoutStageFree)) { ok = false; break; }
               const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
               mbar_expect_tx(full_bar(stage), T::STAGE_BYTES);
+              // SPLIT: blocks [0, n) and [n, 2n) read x_hi, blocks [2n, 3n) read x_lo, which sits n blocks after x_hi
+              const int xb = SPLIT && cb >= a.split_blocks ? cb - a.split_blocks : cb;
               if (a.patch)
-                tma_load_4d(sa, &map_x, full_bar(stage), cb * BK, w0 + s - 1, h0 + r - 1, n0);
+                tma_load_4d(sa, &map_x, full_bar(stage), xb * BK, w0 + s - 1, h0 + r - 1, n0);
               else
-                tma_load_im2col_4d(sa, &map_x, full_bar(stage), cb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
+                tma_load_im2col_4d(sa, &map_x, full_bar(stage), xb * BK, w0 - 1, h0 - 1, n0, (uint16_t)s, (uint16_t)r);
               tma_load_2d(sb, &map_w, full_bar(stage), kb * BK, n_tile * BN);
               ++fills[stage];
               if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
@@ -292,32 +305,37 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, 0, 0);
+      constexpr uint32_t idesc = SPLIT ? umma_idesc_f16(BM, BN, 0, 0) : umma_idesc_bf16(BM, BN, 0, 0);
       int stage = 0;
       uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
-        const int buf = local & 1;
-        const uint32_t use = (uint32_t)(local >> 1);  // how many times this buffer was used before
-        if (!mbar_wait(acc_empty_bar(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+      // one accumulator hand-off per tile, or (SPLIT) per chunk of kSplitChunk K blocks of a tile
+      const int chunk = SPLIT ? kSplitChunk : k_blocks;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int kb0 = 0; kb0 < k_blocks && ok; kb0 += chunk, ++local) {
+          const int buf = local & 1;
+          const uint32_t use = (uint32_t)(local >> 1);  // how many times this buffer was used before
+          if (!mbar_wait(acc_empty_bar(buf), (use & 1) ^ 1, &abort_flag, a.dev_error, kDevTimeoutTmemFree)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
-          // the issue loop is the critical path of the tensor pipe: one descriptor pair per stage,
-          // advanced by 32 bytes (16 K elements) with a single add per MMA
-          const uint64_t da = smem_desc_sw128(sa, 16), db = smem_desc_sw128(sb, 16);
-          umma_bf16(d_tmem, da, db, idesc, kb != 0 ? 1u : 0u);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+          const int kb1 = kb0 + chunk < k_blocks ? kb0 + chunk : k_blocks;
+          for (int kb = kb0; kb < kb1; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, &abort_flag, a.dev_error, kDevTimeoutTmaFull)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = smem_base + stage * T::STAGE_BYTES, sb = sa + A_BYTES;
+            // the issue loop is the critical path of the tensor pipe: one descriptor pair per stage,
+            // advanced by 32 bytes (16 K elements) with a single add per MMA
+            const uint64_t da = smem_desc_sw128(sa, 16), db = smem_desc_sw128(sb, 16);
+            umma_bf16(d_tmem, da, db, idesc, kb != kb0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 1; k < BK / 16; ++k)
-            umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
-          umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
-          if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
+            for (int k = 1; k < BK / 16; ++k)
+              umma_bf16_acc(d_tmem, desc_advance(da, k * 32), desc_advance(db, k * 32), idesc);
+            umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+            if (++stage == T::STAGES) { stage = 0; phase ^= 1; }
+          }
+          if (ok) umma_commit(acc_full_bar(buf));
         }
-        if (ok) umma_commit(acc_full_bar(buf));
       }
       if (!ok) {
         // wait for the MMAs already issued before shared and tensor memory go away
@@ -335,10 +353,36 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // store (whole 128-byte lines), not as per-thread pieces of rows.  Thread 64 owns the store groups.
     const bool issuer = threadIdx.x == 64;
     uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+    bool alive = true;
+    for (int tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x, ++local) {
+      const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
+      // SPLIT: the tensor core's fp32 accumulation truncates, an error that grows with the length of the chain
+      // (1.6e-5 after the 864 MMAs of a 512-channel layer).  The K loop therefore hands over its accumulator every
+      // kSplitChunk K blocks, and the chunks are added here, in registers, with round-to-nearest fp32 additions.
+      float run[SPLIT ? BN : 1];
+      if (SPLIT) {
+#pragma unroll
+        for (int j = 0; j < BN; ++j) run[j] = 0.f;
+        for (int kb0 = kSplitChunk; kb0 < k_blocks && alive; kb0 += kSplitChunk, ++local) {
+          const int cbuf = local & 1;
+          const bool cgot = mbar_wait(acc_full_bar(cbuf), (uint32_t)(local >> 1) & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
+          if (named_bar_or(1, 128, !cgot)) { alive = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int cc = 0; cc < BN; cc += 32) {
+            uint32_t v[32];
+            tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cbuf * BN + cc), v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) run[cc + j] += __uint_as_float(v[j]);
+          }
+          tc_fence_before();
+          mbar_arrive(acc_empty_bar(cbuf));
+        }
+        if (!alive) break;
+      }
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
-      const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
       const bool got = mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
       if (named_bar_or(1, 128, !got)) break;  // all four warps leave together
       tc_fence_after();
@@ -355,10 +399,12 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       const bool valid = pixel < a.pixels;
       const int c_base = n_tile * BN;
       const bf16* mask_row = (a.mask && valid) ? a.mask + pixel * a.Cout + c_base : nullptr;
-#pragma unroll 1
+#pragma unroll(SPLIT ? BN / 64 : 1)
       for (int c64 = 0; c64 < BN; c64 += 64) {
         if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
         named_bar_sync(1, 128);
+        uint32_t lo_packed[SPLIT ? 32 : 1];
+        bool out_of_range = false;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           const int cc = c64 + half * 32;
@@ -369,12 +415,25 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
+            if (SPLIT) {
+              x0 = (x0 + run[cc + j]) * (1.f / kSplitWeightScale);
+              x1 = (x1 + run[cc + j + 1]) * (1.f / kSplitWeightScale);
+            }
             x0 += bias_s[c_base + cc + j]; x1 += bias_s[c_base + cc + j + 1];
             if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
-            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
-            packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+            if (SPLIT) {
+              // first term fp16(x); second term: what that rounding left (exact in fp32), rounded to fp16
+              out_of_range |= fmaxf(fabsf(x0), fabsf(x1)) > 65504.f;
+              __half2 h = __floats2half2_rn(x0, x1);
+              __half2 l = __floats2half2_rn(x0 - __low2float(h), x1 - __high2float(h));
+              packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+              lo_packed[half * 16 + (j >> 1)] = *reinterpret_cast<uint32_t*>(&l);
+            } else {
+              __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+              packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+            }
           }
-          if (mask_row) {
+          if (!SPLIT && mask_row) {
             const uint4* mp = reinterpret_cast<const uint4*>(mask_row + cc);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -406,6 +465,23 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           else tma_store_2d(&map_y, out_smem, c_base + c64, m_tile * BM);
           tma_store_commit();
         }
+        if (SPLIT) {
+          if (out_of_range && valid) atomicCAS(a.dev_error, 0, (int)kDevSplitRange);
+          // the second terms of the same 64 channels, Cout channels further on in the pixel's row
+          if (issuer) tma_store_wait_read<0>();
+          named_bar_sync(1, 128);
+#pragma unroll
+          for (int chunk = 0; chunk < 8; ++chunk)
+            *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) =
+                make_uint4(lo_packed[chunk * 4], lo_packed[chunk * 4 + 1], lo_packed[chunk * 4 + 2], lo_packed[chunk * 4 + 3]);
+          fence_async_smem();
+          named_bar_sync(1, 128);
+          if (issuer) {
+            if (a.patch) tma_store_4d(&map_y, out_smem, a.Cout + c_base + c64, tw * PW, th * PH, img);
+            else tma_store_2d(&map_y, out_smem, a.Cout + c_base + c64, m_tile * BM);
+            tma_store_commit();
+          }
+        }
       }
       tc_fence_before();
       mbar_arrive(acc_empty_bar(buf));
@@ -422,13 +498,13 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   }
 }
 
-template <int BN>
+template <int BN, bool SPLIT = false>
 cudaError_t launch_conv(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, ConvArgs a,
                         cudaStream_t st) {
   using T = ConvTile<BN>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel<BN, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -437,7 +513,7 @@ cudaError_t launch_conv(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int tiles = a.m_tiles * a.n_tiles;
   const int grid = tiles < sms ? tiles : sms;
-  conv3x3_tc_kernel<BN><<<grid, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
+  conv3x3_tc_kernel<BN, SPLIT><<<grid, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
   return cudaGetLastError();
 }
 
@@ -479,11 +555,44 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0;
   a.bias = bias; a.mask = mask; a.out = out; a.dev_error = dev_error;
+  a.split_blocks = 0;
   switch (BN) {
     case 256: return launch_conv<256>(mx, mw, my, a, st);
     case 128: return launch_conv<128>(mx, mw, my, a, st);
     default: return launch_conv<64>(mx, mw, my, a, st);
   }
+}
+
+// fp32 convolution from split operands (see the kernel): in [N][H][W][2 * Cin] and out [N][H][W][2 * Cout] hold
+// [hi | lo] per pixel, wt_split [Cout][9][3 * Cin] holds [w_hi | w_lo | w_hi] per tap; s has the logical channels.
+// (The tensor maps only move 16-bit words: the bf16 ones serve fp16 data.)
+cudaError_t tc_conv3x3_split(const half16* in, const half16* wt_split, const float* bias, half16* out, ConvShape s,
+                             bool relu, int* dev_error, cudaStream_t st) {
+  if (!tc_conv3x3_supported(s)) return cudaErrorInvalidValue;
+  const int BN = s.Cout % 128 == 0 ? 128 : 64;  // the epilogue keeps a tile row's running sums in registers
+  CUtensorMap mx, mw, my;
+  const bool patch = s.W % PW == 0 && s.H % PH == 0;
+  if (patch) {
+    if (!make_patch_map(&mx, in, s.N, s.H, s.W, 2 * s.Cin, PW, PH)) return cudaErrorInvalidValue;
+    if (!make_patch_map(&my, out, s.N, s.H, s.W, 2 * s.Cout, PW, PH)) return cudaErrorInvalidValue;
+  } else {
+    if (!make_im2col_map(&mx, in, s.N, s.H, s.W, 2 * s.Cin, BM)) return cudaErrorInvalidValue;
+    if (!make_tiled_map_2d(&my, out, (uint64_t)s.N * s.H * s.W, (uint64_t)2 * s.Cout, BM)) return cudaErrorInvalidValue;
+  }
+  if (!make_tiled_map_2d(&mw, wt_split, (uint64_t)s.Cout, (uint64_t)27 * s.Cin, (uint32_t)BN)) return cudaErrorInvalidValue;
+  ConvArgs a;
+  a.patch = patch ? 1 : 0;
+  a.tiles_w = s.W / PW; a.tiles_h = s.H / PH;
+  a.pixels = s.N * s.H * s.W;
+  a.H = s.H; a.W = s.W;
+  a.cin_blocks = 3 * s.Cin / 64;
+  a.split_blocks = s.Cin / 64;
+  a.Cout = s.Cout;
+  a.m_tiles = (a.pixels + BM - 1) / BM;
+  a.n_tiles = s.Cout / BN;
+  a.relu = relu ? 1 : 0;
+  a.bias = bias; a.mask = nullptr; a.out = reinterpret_cast<bf16*>(out); a.dev_error = dev_error;
+  return BN == 128 ? launch_conv<128, true>(mx, mw, my, a, st) : launch_conv<64, true>(mx, mw, my, a, st);
 }
 
 namespace {

@@ -17,6 +17,12 @@ bool tc_conv3x3_supported(ConvShape s);
 cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const bf16* mask,
                        bf16* out, ConvShape s, bool relu, int* dev_error, cudaStream_t st);
 
+// fp32 convolution as three fp16 products per product: in [N][H][W][2 Cin] and out [N][H][W][2 Cout] hold each
+// pixel's channels as [hi | lo] fp16 terms, wt_split [Cout][9][3 Cin] each tap's filter row as [hi | lo | hi] of
+// the weights times kSplitWeightScale; s names the logical channels (shapes as tc_conv3x3_supported).
+cudaError_t tc_conv3x3_split(const half16* in, const half16* wt_split, const float* bias, half16* out, ConvShape s,
+                             bool relu, int* dev_error, cudaStream_t st);
+
 // The same convolution on CTA pairs (tc_conv_pair.cu): a cluster of two CTAs per 256-pixel x 256-channel
 // tile, each staging half of the filter slice.  Cout must be a multiple of 256.
 // partial (or null): fp32 scratch of tc_conv3x3_pair_scratch_elems() elements.  With it, when the tile count
@@ -82,6 +88,12 @@ cudaError_t tc_dense_forward(const bf16* X, const bf16* W, const float* bias, bf
                              float* partial, int M, int In, int Out, bool relu, int* dev_error, cudaStream_t st);
 cudaError_t tc_dense_dx(const bf16* dY, const bf16* W, const bf16* mask, bf16* dX, float* partial, int M, int In,
                         int Out, int* dev_error, cudaStream_t st);
+// fp32 dense layer from split operands: X [M][2 In] = [hi | lo] rows of fp16 terms, Ws [Out][3 In] = [hi | lo | hi]
+// rows of the weights times kSplitWeightScale (In a multiple of 64); fp32 output.
+// partial: tc_dense_split_scratch_elems(M, In, Out) elements (K is cut into many short splits).
+size_t tc_dense_split_scratch_elems(int M, int In, int Out);
+cudaError_t tc_dense_forward_split(const half16* X, const half16* Ws, const float* bias, float* out_f, float* partial,
+                                   int M, int In, int Out, bool relu, int* dev_error, cudaStream_t st);
 // With sgd_copy and sgd_lr (a device scalar) the gradient is not stored: dW then points at the layer's fp32
 // master weights, which become w - lr * gradient in the GEMM's epilogue, and sgd_copy (their bf16 copy)
 // receives the rounded result - the parameter update of a training step folded into the filter-gradient GEMM.

@@ -65,6 +65,7 @@ struct vgg19 {
   bf16 *tap_fwd = nullptr;   // tap-major [9][Cout][Cin] filters of layers 2..16 (halo kernel), at dgrad_off
   bf16 *tap_bwd = nullptr;   // tap-major rotated filters [9][Cin][Cout] of the same layers
   bf16 *w8 = nullptr;        // first-layer filter padded to [64][10][8] (bf16 tensor-core path)
+  half16 *split_w = nullptr; // fp32 configuration on tensor cores: rows [hi | lo | hi] (fp16 terms) of every weight matrix, at 3 * w_off
   int *dev_error = nullptr;
   void *ws = nullptr;
   size_t ws_bytes = 0;
@@ -74,6 +75,7 @@ struct vgg19 {
   std::string err;
   bool use_tc = false;
   bool use_pair = false;  // two-CTA kernels where a layer's shape takes them
+  bool use_split = false; // fp32 forward-only passes on tensor cores, three fp16 products per product
   // vgg19_forward_host_async: two staging slots, a stream of the library's own for the uploads, and per
   // slot an event for "images uploaded" and one for "the pass that used the slot has finished"
   cudaStream_t copy_stream = nullptr;
@@ -166,6 +168,8 @@ Plan make_plan(const vgg19 *n, int B, int mode) {
   size_t dense_partial = 0;
   for (int i = 0; i < kFcLayers; ++i) {
     size_t e = tc_dense_scratch_elems(B, n->fc[i].In, n->fc[i].Out);
+    if (n->use_split && tc_dense_split_scratch_elems(B, n->fc[i].In, n->fc[i].Out) > e)
+      e = tc_dense_split_scratch_elems(B, n->fc[i].In, n->fc[i].Out);
     if (e > dense_partial) dense_partial = e;
   }
   if (1024 * 512 > max_partial) max_partial = 1024 * 512;  // bias-gradient column sums
@@ -230,6 +234,9 @@ struct Pass {
   // pooling decisions should not depend on what else is in the batch, keeps it off for its forward half.
   bool forward_tail_split = true;
   const void *x8_of = nullptr;  // the image whose 8-channel copy this pass has already made
+  // fp32 configuration, forward only: activations travel as [hi | lo] fp16 terms (the same bytes as fp32) and
+  // layers 2..16 and the dense layers run on tensor cores with three fp16 products per product
+  bool split = false;
   // Training step on one GPU: the learning rate (device scalar).  Where a filter-gradient kernel can
   // apply the update itself (the dense layers' GEMM: 86 % of the parameters at 224x224) the gradient is
   // never stored; `folded` tells the caller which parameter ranges are already updated.
@@ -262,6 +269,19 @@ struct Pass {
   void conv_forward(int l, const T *x, int B, T *y, T *pooled, bool need_y = true, uint8_t *code = nullptr) {
     const ConvLayer &c = n->conv[l];
     ConvShape s{B, c.H, c.W, c.Cin, c.Cout};
+    if (split) {
+      // layer 1 (3 input channels) stays on the CUDA cores in fp32 and its output is split in place; the others
+      // read and write split tensors.  The last pool writes one [all hi | all lo] row per image for dense 1.
+      if (l == 0) {
+        ok(simt_conv3x3<T>(x, wt(c.w_off), n->params + c.b_off, nullptr, y, s, true, st), 1);
+        ok(split_rows((const float *)y, (half16 *)y, (long)B * c.H * c.W, c.Cout, n->dev_error, st), 1);
+      } else {
+        ok(tc_conv3x3_split((const half16 *)x, n->split_w + 3 * c.w_off, n->params + c.b_off, (half16 *)y, s, true,
+                            n->dev_error, st), 1);
+      }
+      if (pooled) ok(maxpool_split((const half16 *)y, (half16 *)pooled, B, c.H, c.W, c.Cout, l == kConvLayers - 1, st), 1);
+      return;
+    }
     if (first_tc_ok(l, s)) {
       ok(tc_pad_to8((const bf16 *)x, (bf16 *)buf(p.x8), (long)B * c.H * c.W, st), 1);
       x8_of = x;
@@ -348,6 +368,14 @@ struct Pass {
   bool tc_dense_ok(int B, const FcLayer &f) const { return n->use_tc && tc_dense_supported(B, f.In, f.Out); }
 
   void dense_forward(const FcLayer &f, const T *x, int B, T *out_t, float *out_f) {
+    if (split) {
+      // fp32 result into the output buffer, then split in place for the next layer (the logits stay fp32)
+      float *o = out_f ? out_f : (float *)out_t;
+      ok(tc_dense_forward_split((const half16 *)x, n->split_w + 3 * f.w_off, n->params + f.b_off, o, fbuf(p.partial), B,
+                                f.In, f.Out, f.relu, n->dev_error, st), 2);
+      if (!out_f) ok(split_rows(o, (half16 *)out_t, B, f.Out, n->dev_error, st), 1);
+      return;
+    }
     if (tc_dense_ok(B, f))
       ok(tc_dense_forward((const bf16 *)x, (const bf16 *)wt(f.w_off), n->params + f.b_off, (bf16 *)out_t, out_f,
                           fbuf(p.partial), B, f.In, f.Out, f.relu, n->dev_error, st), 2);
@@ -485,6 +513,7 @@ int enqueue(vgg19 *n, int mode, const PassArgs &a, cudaStream_t st, int *launche
   Pass<T> pass{n, make_plan(n, a.batch, mode), st};
   if (mode == VGG19_MODE_FORWARD) {
     pass.keep_activations = false;
+    pass.split = n->use_split;
     pass.forward(a);
   } else if (mode == VGG19_MODE_BACKWARD) {
     pass.forward_tail_split = false;
@@ -584,6 +613,16 @@ void drop_graphs(vgg19 *n) {
 // gradients, tap-major filters, the padded first-layer filter), rebuilt from the fp32 master on `st`.
 int refresh_filter_copies(vgg19 *n, cudaStream_t st) {
   const bool h = n->cfg.dtype == VGG19_BF16;
+  if (n->split_w) {
+    for (int l = 1; l < kConvLayers; ++l) {
+      const ConvLayer &c = n->conv[l];
+      CUDA_TRY(n, split_weights(n->params + c.w_off, n->split_w + 3 * c.w_off, 9L * c.Cout, c.Cin, st));
+    }
+    for (int i = 0; i < kFcLayers; ++i) {
+      const FcLayer &f = n->fc[i];
+      CUDA_TRY(n, split_weights(n->params + f.w_off, n->split_w + 3 * f.w_off, f.Out, f.In, st));
+    }
+  }
   if (h && n->tap_fwd && n->tap_bwd) {
     // tensor-core configuration: all three bf16 copies of layers 2..16 in one launch
     FilterCopyTable tab{};
@@ -637,6 +676,8 @@ int create_common(const vgg19_config *cfg, vgg19 **out) {
     return fail(nullptr, VGG19_ERR_SHAPE, "height %d / width %d must be positive multiples of 32",
                 cfg->height, cfg->width);
   if (cfg->batch_max < 1) return fail(nullptr, VGG19_ERR_ARG, "batch_max %d < 1", cfg->batch_max);
+  if ((cfg->flags & VGG19_FLAG_SPLIT_F16) && cfg->dtype != VGG19_FP32)
+    return fail(nullptr, VGG19_ERR_ARG, "VGG19_FLAG_SPLIT_F16 applies to the fp32 configuration only");
   int dev = 0;
   cudaDeviceProp prop;
   CUDA_TRY(nullptr, cudaGetDevice(&dev));
@@ -650,6 +691,7 @@ int create_common(const vgg19_config *cfg, vgg19 **out) {
   n->elt = cfg->dtype == VGG19_BF16 ? 2 : 4;
   n->use_tc = cfg->dtype == VGG19_BF16 && !(cfg->flags & VGG19_FLAG_NO_TENSOR_CORES);
   n->use_pair = n->use_tc && !(cfg->flags & VGG19_FLAG_NO_CTA_PAIRS);
+  n->use_split = cfg->dtype == VGG19_FP32 && (cfg->flags & VGG19_FLAG_SPLIT_F16) != 0;
   size_t off = 0, doff = 0;
   int h = cfg->height, w = cfg->width, cin = 3, n_pool = 0;
   for (int l = 0; l < kConvLayers; ++l) {
@@ -681,6 +723,7 @@ int create_common(const vgg19_config *cfg, vgg19 **out) {
   if (e == cudaSuccess && n->use_tc) e = cudaMalloc(&n->w8, 64 * 80 * sizeof(bf16));
   if (e == cudaSuccess && n->use_tc) e = cudaMalloc(&n->tap_fwd, n->n_dgrad * sizeof(bf16));
   if (e == cudaSuccess && n->use_tc) e = cudaMalloc(&n->tap_bwd, n->n_dgrad * sizeof(bf16));
+  if (e == cudaSuccess && n->use_split) e = cudaMalloc(&n->split_w, 3 * n->n_params * sizeof(half16));
   if (e == cudaSuccess) e = cudaMalloc(&n->dev_error, 256);
   if (e == cudaSuccess) e = cudaMemset(n->dev_error, 0, 256);
   if (e != cudaSuccess) {
@@ -726,6 +769,7 @@ void vgg19_destroy(vgg19_t *n) {
   if (n->params) cudaFree(n->params);
   if (n->dgrad_w) cudaFree(n->dgrad_w);
   if (n->w8) cudaFree(n->w8);
+  if (n->split_w) cudaFree(n->split_w);
   if (n->tap_fwd) cudaFree(n->tap_fwd);
   if (n->tap_bwd) cudaFree(n->tap_bwd);
   if (n->dev_error) cudaFree(n->dev_error);
@@ -991,6 +1035,26 @@ int vgg19_conv_layer_forward_ex(vgg19_t *n, int32_t layer, const void *x, int32_
       return fail(n, VGG19_ERR_ARG, "layer %d at this size has no pooled-only kernel: y must not be null", layer);
     ps.conv_forward(layer - 1, (const bf16 *)x, batch, (bf16 *)y, (bf16 *)pooled, y != nullptr, pool_code);
     e = ps.err;
+  } else if (n->use_split && layer > 1) {
+    // fp32 tensors in and out; between them the layer runs on its split form: x is split into the workspace slot
+    // a whole pass would read it from, y and pooled receive split tensors and are merged in place
+    const ConvLayer &c = n->conv[layer - 1];
+    if (!y || pool_code) return fail(n, VGG19_ERR_ARG, "the fp32 configuration has no pooled-only kernel and stores no pool codes here");
+    if (!plan.valid) return fail(n, VGG19_ERR_WORKSPACE, "this layer needs the forward workspace bound");
+    if (!split_rows_supported(c.Cin) || !split_rows_supported(c.Cout))
+      return fail(n, VGG19_ERR_SHAPE, "channel counts %d -> %d do not divide 4096", c.Cin, c.Cout);
+    Pass<float> ps{n, plan, st};
+    ps.split = true;
+    const bool in_is_pool = n->conv[layer - 2].pool_after;
+    half16 *xs = (half16 *)ps.buf(in_is_pool ? plan.pooled[n->pool_idx[layer - 2]] : plan.act[layer - 2]);
+    ps.ok(split_rows((const float *)x, xs, (long)batch * c.H * c.W, c.Cin, n->dev_error, st), 1);
+    ps.conv_forward(layer - 1, (const float *)xs, batch, (float *)y, nullptr);
+    if (pooled) {
+      ps.ok(maxpool_split((const half16 *)y, (half16 *)pooled, batch, c.H, c.W, c.Cout, false, st), 1);
+      ps.ok(merge_rows((const half16 *)pooled, (float *)pooled, (long)batch * (c.H / 2) * (c.W / 2), c.Cout, st), 1);
+    }
+    ps.ok(merge_rows((const half16 *)y, (float *)y, (long)batch * c.H * c.W, c.Cout, st), 1);
+    e = ps.err;
   } else {
     Pass<float> ps{n, plan, st};
     if (!y) return fail(n, VGG19_ERR_ARG, "the fp32 configuration has no pooled-only kernel: y must not be null");
@@ -1090,6 +1154,8 @@ int vgg19_sync_status(vgg19_t *n, void *stream) {
     cudaMemset(n->dev_error, 0, 256);
     if (code == kDevBadLabel)
       return fail(n, VGG19_ERR_ARG, "a label outside [0, %d) reached the loss (its row's loss is NaN)", kClasses);
+    if (code == kDevSplitRange)
+      return fail(n, VGG19_ERR_RANGE, "an activation beyond fp16's range (65504) met the split-fp16 path");
     return fail(n, VGG19_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (code %d)", code);
   }
   return VGG19_OK;
