@@ -526,9 +526,18 @@ def run_native(args):
             row["dgrad_ms"] = round(dg, 4)
             row["dgrad_tflops"] = round(f / (dg * 1e-3) / 1e12, 1)
             row["dgrad_frac"] = round(f / (dg * 1e-3) / 1e12 / peak, 3)
+            # an input gradient reads dz and the ReLU mask of the layer below and writes dx: where those bytes at the
+            # measured copy bandwidth take longer than the FLOPs at the tensor peak, that is the kernel's roofline
+            s_, ci, co = CONV[l - 1]
+            hbm_ms = BATCH * s_ * s_ * (co + 2 * ci) * 2 / (pk["hbm_gbs"] * 1e9) * 1e3
+            if hbm_ms > f / (peak * 1e12) * 1e3:
+                row["dgrad_bound"] = "hbm"
+                row["dgrad_hbm_floor_ms"] = round(hbm_ms, 4)
+                row["dgrad_frac_of_hbm"] = round(hbm_ms / dg, 3)
             for kind in ("wgrad", "dgrad"):
                 if row[kind + "_frac"] < 0.6:
-                    below.append(f"conv{l} {kind} {row[kind + '_frac']:.2f}")
+                    hb = f" (hbm-bound: {row['dgrad_frac_of_hbm']:.2f} of its byte floor)" if kind == "dgrad" and "dgrad_bound" in row else ""
+                    below.append(f"conv{l} {kind} {row[kind + '_frac']:.2f}{hb}")
         per_layer_bwd[f"conv{l}"] = row
     for l, ms, f, path in layers:
         if f / (ms * 1e-3) / 1e12 / peak < 0.6:

@@ -1186,7 +1186,8 @@ int vgg19_describe(const vgg19_t *n, char *out, size_t cap) {
     ConvShape sh{n->cfg.batch_max, c.H, c.W, c.Cin, c.Cout};
     ConvShape sd{n->cfg.batch_max, c.H, c.W, c.Cout, c.Cin};
     // the kernel each pass picks for this layer, in the order the scheduler tries them
-    const char *fwd = !n->use_tc ? "simt"
+    const char *fwd = n->use_split ? (l == 0 ? "simt" : "tcgen05:im2col-split-fp16 (forward-only passes; else simt)")
+                      : !n->use_tc ? "simt"
                       : l == 0 ? (tc_first_conv_supported(sh) ? "tcgen05:first-layer" : "simt")
                       : tc_conv3x3_rowshift_supported(sh) ? "tcgen05:row-shift"
                       : tc_conv3x3_halo_supported(sh) ? (n->use_pair && c.Cout == 128 ? "tcgen05:halo-pair" : "tcgen05:halo")
@@ -1209,7 +1210,8 @@ int vgg19_describe(const vgg19_t *n, char *out, size_t cap) {
   }
   for (int i = 0; i < kFcLayers; ++i) {
     const FcLayer &f = n->fc[i];
-    snprintf(line, sizeof line, "dense%d %5d->%-4d +bias%s\n", i + 1, f.In, f.Out, f.relu ? " +relu" : "");
+    snprintf(line, sizeof line, "dense%d %5d->%-4d +bias%s%s\n", i + 1, f.In, f.Out, f.relu ? " +relu" : "",
+             n->use_split ? "  fwd=tcgen05:gemm-split-fp16 (forward-only passes; else simt)" : "");
     s += line;
   }
   s += "softmax 1000\n";

@@ -129,6 +129,32 @@ def test_split_reports_an_activation_beyond_fp16_range():
     net.close()
 
 
+def test_split_network_through_the_host_entry_point_and_beside_a_backward_pass():
+    """The host-buffer call runs the same split pass (same bits as the device call); a backward pass of the same
+    network keeps the CUDA-core fp32 kernels (the flag covers forward-only passes) and still matches the checker."""
+    p = pkg()
+    B = 2
+    params = si.vgg19_params(32, 32, seed=0, bias_std=0.05)
+    images, labels = si.images(B, 32, 32, seed=1), si.labels(B, seed=2)
+    net = p.Net(32, 32, B, p.VGG19_FP32, params=params, flags=p.VGG19_FLAG_SPLIT_F16, host_io=True)
+    assert "split-fp16" in p.vgg19_describe(net.handle)
+    x = torch.from_numpy(images)
+    logits_host = torch.empty(B, 1000, dtype=torch.float32).pin_memory()
+    s = torch.cuda.Stream()
+    p.vgg19_forward_host(net.handle, x.pin_memory(), B, logits_host, None, s)
+    dev_logits = net.forward(x.to(DEV)).clone()
+    net.sync_status()
+    assert torch.equal(dev_logits.cpu(), logits_host)
+    bl = torch.empty(B, 1000, dtype=torch.float32, device=DEV)
+    grads, loss = net.backward(x.to(DEV), torch.from_numpy(labels).to(DEV), logits=bl)
+    net.sync_status()
+    o_loss, o_grads, o_logits = oracle.vgg19_backward(params.astype(np.float64), images, labels, chunk=B)
+    assert rel_l2(bl.cpu().numpy(), o_logits) <= 1e-4 and rel_l2(dev_logits.cpu().numpy(), o_logits) <= 3e-5
+    assert rel_l2(grads.cpu().numpy(), o_grads) <= 2e-4
+    assert abs(float(loss) - o_loss) <= 1e-4 * abs(o_loss)
+    net.close()
+
+
 def test_split_flag_needs_fp32():
     p = pkg()
     with pytest.raises(Exception):
