@@ -210,7 +210,10 @@ int vgg19_forward_host_async(vgg19_t *net, const void *host_images, int32_t batc
  * config's dtype; the per-layer building block of section 7.2, exposed for
  * per-layer parity and timing.  layer in 1..16 selects shape and weights;
  * x: [batch][h][w][Cin]; y: [batch][h][w][Cout]; pooled (or NULL):
- * [batch][h/2][w/2][Cout]. */
+ * [batch][h/2][w/2][Cout].  On a network created with VGG19_FLAG_SPLIT_F16
+ * layers 2..16 run on the split-fp16 tensor-core kernel: x, y and pooled are
+ * fp32 as always (y and pooled also serve as scratch for their two-term
+ * forms), and the forward workspace must be bound (VGG19_ERR_WORKSPACE). */
 int vgg19_conv_layer_forward(vgg19_t *net, int32_t layer, const void *x, int32_t batch,
                              void *y, void *pooled, void *stream);
 
