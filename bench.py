@@ -43,6 +43,10 @@ METRIC = "VGG19 fwd images/s @batch 100, 224x224 bf16"
 WORKLOAD = "configs[3]: full VGG19 forward, 224x224x3, batch 100, bf16 storage, fp32 accumulate"
 H = W = 224
 BATCH = 100
+# Idle time after each kernel of the per-kernel timings: seven launches of one kernel are a millisecond or two of
+# full load; without a pause the whole table runs as one stretch of tens of milliseconds and, on some boxes, at the
+# power cap's clock, while the peaks it is compared with are burst figures taken on an idle GPU.
+KERNEL_GAP_S = 0.05
 CONV = [(224, 3, 64), (224, 64, 64), (112, 64, 128), (112, 128, 128), (56, 128, 256), (56, 256, 256),
         (56, 256, 256), (56, 256, 256), (28, 256, 512), (28, 512, 512), (28, 512, 512), (28, 512, 512),
         (14, 512, 512), (14, 512, 512), (14, 512, 512), (14, 512, 512)]
@@ -79,7 +83,7 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def stop(self, t_begin=None, t_end=None, extra_window=None):
+    def stop(self, t_begin=None, t_end=None, extra_window=None, kernel_window=None):
         """Summary of the samples taken between the two wall-clock times (all samples if none fall inside);
         with extra_window=(t0, t1) also {"extra": summary of the samples inside that second window}."""
         if self.proc is None:
@@ -116,6 +120,8 @@ class ClockSampler:
         out = summary(t_begin, t_end, "timed region")
         if extra_window:
             out["extra"] = summary(extra_window[0], extra_window[1], "sustained region")
+        if kernel_window:
+            out["kernels"] = summary(kernel_window[0], kernel_window[1], "per-kernel timings")
         return out
 
 
@@ -261,6 +267,7 @@ def time_conv_layers(pkg, net, torch, stream, reps=5):
                 pkg.vgg19_conv_layer_forward(net.handle, l + 1, x, BATCH, scratch, None, stream)
                 b.record(stream)
         stream.synchronize()
+        time.sleep(KERNEL_GAP_S)
         ms = sum(a.elapsed_time(b) for a, b in evs) / reps
         out.append((l + 1, ms, 2.0 * BATCH * s * s * co * 9 * ci, path))
     return out
@@ -305,8 +312,46 @@ def time_conv_layers_backward(pkg, net, torch, stream, images, reps=5):
                     fn()
                     b.record(stream)
             stream.synchronize()
+            time.sleep(KERNEL_GAP_S)
             ms[name] = sum(a.elapsed_time(b) for a, b in evs) / reps
         out.append((l + 1, ms.get("dgrad"), ms["wgrad"], 2.0 * BATCH * s * s * co * 9 * ci))
+    return out
+
+
+def time_dense_layers(pkg, net, torch, stream, reps=5):
+    """Per-layer CUDA-event timing of the dense layers at batch 100 through the per-layer entry points: forward
+    (GEMM + finishing kernel) and backward (bias gradient, input gradient with its ReLU mask, filter gradient).
+    Both stream the layer's weights once and are bound by that: algorithmic bytes = bf16 weights read (forward;
+    input gradient) + fp32 filter gradient written.  Returns {name: {...}}."""
+    dims = [(7 * 7 * 512, 4096), (4096, 4096), (4096, 1000)]
+    out = {}
+    for i, (In, Out) in enumerate(dims):
+        x = torch.randn(BATCH, In, device=net.device).abs().to(torch.bfloat16)
+        dy = (torch.randn(BATCH, Out, device=net.device) * 1e-3).to(torch.bfloat16)
+        y = torch.empty(BATCH, Out, dtype=torch.bfloat16, device=net.device)
+        yf = torch.empty(BATCH, Out, dtype=torch.float32, device=net.device)
+        dx = torch.empty(BATCH, In, dtype=torch.bfloat16, device=net.device)
+        dw = torch.empty(Out * In, dtype=torch.float32, device=net.device)
+        db = torch.empty(Out, dtype=torch.float32, device=net.device)
+        calls = {"fwd": lambda: pkg.vgg19_dense_layer_forward(net.handle, i + 1, x, BATCH, y if i < 2 else None, yf if i == 2 else None, stream),
+                 "bwd": lambda: pkg.vgg19_dense_layer_backward(net.handle, i + 1, x, dy, BATCH, dw, db, dx, x if i > 0 else None, stream)}
+        row = {}
+        for name, fn in calls.items():
+            with torch.cuda.stream(stream):
+                for _ in range(2):
+                    fn()
+                evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+                for a, b in evs:
+                    a.record(stream)
+                    fn()
+                    b.record(stream)
+            stream.synchronize()
+            time.sleep(KERNEL_GAP_S)
+            row[name] = sum(a.elapsed_time(b) for a, b in evs) / reps
+        w = In * Out
+        out[f"dense{i + 1}"] = {"fwd_ms": row["fwd"], "fwd_bytes": 2 * w + 2 * BATCH * (In + Out),
+                                "bwd_ms": row["bwd"], "bwd_bytes": 2 * w + 4 * w + 2 * BATCH * (2 * In + 2 * Out)}
+        del x, dy, y, yf, dx, dw, db
     return out
 
 
@@ -438,14 +483,18 @@ def run_native(args):
     # compared with burst peaks (a best-of-10 GEMM and copy on an idle GPU), and the seconds of sustained
     # load further down pull the SM clock to the power cap's level.  Rank 0 only; the others wait at the
     # next barrier.
-    layers = bwd_layers = None
+    layers = bwd_layers = dense_layers = None
+    t_k0 = time.time()
     if rank == 0:
         with torch.cuda.stream(stream):
             bwd()  # leaves the batch-100 activations of every layer in the workspace
         stream.synchronize()
+        time.sleep(0.3)
         layers = time_conv_layers(pkg, net, torch, stream)
         first_ms, first_bytes = time_first_layer(pkg, net, torch, stream, x)
         bwd_layers = time_conv_layers_backward(pkg, net, torch, stream, x)
+        dense_layers = time_dense_layers(pkg, net, torch, stream)
+        t_k1 = time.time()
         time.sleep(1.0)  # let the power budget recover before the next timed region
     bwd_steps = max(3, args.steps // 2)
     t_begin_bwd = time.time()
@@ -460,8 +509,9 @@ def run_native(args):
     t_sus1 = time.time()
     net.sync_status(stream)
     # the clock record of the headline number: the samples inside the forward passes' timed region
-    clocks = sampler.stop(t_begin, t_end_fwd, extra_window=(t_sus0, t_sus1)) if sampler else None
+    clocks = sampler.stop(t_begin, t_end_fwd, extra_window=(t_sus0, t_sus1), kernel_window=(t_k0, t_k1)) if sampler else None
     sustained_clocks = clocks.pop("extra", None) if clocks else None
+    kernel_clocks = clocks.pop("kernels", None) if clocks else None
 
     # training step last: it moves the weights (by a learning rate small enough to keep them sane)
     if world > 1:
@@ -542,6 +592,13 @@ def run_native(args):
     for l, ms, f, path in layers:
         if f / (ms * 1e-3) / 1e12 / peak < 0.6:
             below.append(f"conv{l} fwd {f / (ms * 1e-3) / 1e12 / peak:.2f}")
+    # dense layers: bound by streaming their weights (and, backward, writing the fp32 filter gradient)
+    per_dense = {}
+    for name, d in dense_layers.items():
+        per_dense[name] = {"fwd_ms": round(d["fwd_ms"], 4), "fwd_gbs": round(d["fwd_bytes"] / (d["fwd_ms"] * 1e-3) / 1e9, 1),
+                           "fwd_frac_of_hbm": round(d["fwd_bytes"] / (d["fwd_ms"] * 1e-3) / 1e9 / pk["hbm_gbs"], 3),
+                           "bwd_ms": round(d["bwd_ms"], 4), "bwd_gbs": round(d["bwd_bytes"] / (d["bwd_ms"] * 1e-3) / 1e9, 1),
+                           "bwd_frac_of_hbm": round(d["bwd_bytes"] / (d["bwd_ms"] * 1e-3) / 1e9 / pk["hbm_gbs"], 3)}
     bwd_conv_ms = sum((dg or 0.0) + wg for _, dg, wg, _ in bwd_layers)
     bwd_conv_flop = sum(f * (2 if l > 1 else 0) for l, _, _, f in bwd_layers)
     roof_ms = forward_roofline_ms(pk)
@@ -595,10 +652,12 @@ def run_native(args):
                                               "frac": all_flop / (all_ms * 1e-3) / 1e12 / peak},
                      "per_layer": per_layer,
                      "per_layer_bwd": per_layer_bwd,
+                     "per_dense_layer": per_dense,
+                     "per_kernel_clocks": kernel_clocks,
                      "bwd_conv_kernels": {"ms": bwd_conv_ms, "tflops": bwd_conv_flop / (bwd_conv_ms * 1e-3) / 1e12,
                                           "note": "input- and filter-gradient kernels of layers 1..16, each timed alone"},
                      "below_60pct_of_bf16_peak": below,
-                     "hbm_bound_not_listed_above": "conv1 fwd and wgrad (3 input channels) and the dense layers at batch "
+                     "hbm_bound_not_listed_above": "conv1 fwd and wgrad (3 input channels) and the dense layers (per_dense_layer) at batch "
                                                    "100 are bound by HBM, see hbm_bound and per_layer_bwd.conv1"},
         "hbm_bound": {"kernel": "conv1_1 forward (pad_to8_kernel + conv3x3_c8_tc_kernel): 3-channel image in, 64-channel activation out",
                       "ms": round(first_ms, 4), "achieved": first_bytes / (first_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"],

@@ -277,6 +277,21 @@ int vgg19_conv_layer_backward_ex(vgg19_t *net, int32_t layer, const void *x, con
  * Element type is the config's dtype.  A forward-only pass does not write the
  * pre-pool output of a layer whose max-pool is fused into the convolution
  * (layers 2 and 4 at 224x224); a backward pass stores everything. */
+/* Single dense layer (section 7.2's last three layers; the appendix table's `dot` rows), exposed like the
+ * convolution layers for per-layer parity and timing.  layer in 1..3.  x: device [batch][In] in the config's
+ * dtype (for layer 1 the flattened last pooling output, [batch][h][w][512] order).  y (or NULL): device
+ * [batch][Out] in the config's dtype; y_f32 (or NULL): the same values as fp32 (how layer 3's logits leave); at
+ * least one.  Bias added; ReLU applied for layers 1 and 2.  Needs the forward workspace. */
+int vgg19_dense_layer_forward(vgg19_t *net, int32_t layer, const void *x, int32_t batch, void *y, float *y_f32,
+                              void *stream);
+
+/* Backward of one dense layer: dw fp32 [Out][In] and db fp32 [Out] from (x, dy); dx (or NULL) device
+ * [batch][In] in the config's dtype = dy W, multiplied by (relu_mask > 0) when relu_mask (the layer's input,
+ * itself a ReLU output; or NULL) is given.  dy: device [batch][Out] in the config's dtype, the gradient at the
+ * layer's pre-activation.  Needs the backward workspace. */
+int vgg19_dense_layer_backward(vgg19_t *net, int32_t layer, const void *x, const void *dy, int32_t batch, float *dw,
+                               float *db, void *dx, const void *relu_mask, void *stream);
+
 int vgg19_saved_tensor(const vgg19_t *net, int32_t batch, int32_t mode, int32_t index,
                        size_t *offset_bytes, int64_t dims[4]);
 

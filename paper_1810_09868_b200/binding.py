@@ -24,7 +24,7 @@ EXPORTS = (
     "vgg19_get_params", "vgg19_set_params", "vgg19_workspace_bytes", "vgg19_bind_workspace",
     "vgg19_forward", "vgg19_backward", "vgg19_sgd_step", "vgg19_train_step", "vgg19_train_steps",
     "vgg19_set_dense_grads_event", "vgg19_io_bytes", "vgg19_forward_host", "vgg19_forward_host_async", "vgg19_backward_host",
-    "vgg19_conv_layer_forward", "vgg19_conv_layer_forward_ex", "vgg19_first_block_forward", "vgg19_conv_layer_backward", "vgg19_conv_layer_backward_ex", "vgg19_saved_tensor", "vgg19_conv_wgrad_static", "vgg19_sync_status", "vgg19_selftest_wait_timeout", "vgg19_launch_count",
+    "vgg19_conv_layer_forward", "vgg19_conv_layer_forward_ex", "vgg19_first_block_forward", "vgg19_conv_layer_backward", "vgg19_conv_layer_backward_ex", "vgg19_dense_layer_forward", "vgg19_dense_layer_backward", "vgg19_saved_tensor", "vgg19_conv_wgrad_static", "vgg19_sync_status", "vgg19_selftest_wait_timeout", "vgg19_launch_count",
     "vgg19_describe", "vgg19_last_error",
 )
 
@@ -84,6 +84,8 @@ def load():
         "vgg19_conv_layer_forward_ex": ([vp, i32, vp, i32, vp, vp, vp, vp], ctypes.c_int),
         "vgg19_first_block_forward": ([vp, vp, i32, vp, vp, vp], ctypes.c_int),
         "vgg19_conv_layer_backward_ex": ([vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp], ctypes.c_int),
+        "vgg19_dense_layer_forward": ([vp, i32, vp, i32, vp, vp, vp], ctypes.c_int),
+        "vgg19_dense_layer_backward": ([vp, i32, vp, vp, i32, vp, vp, vp, vp, vp], ctypes.c_int),
         "vgg19_saved_tensor": ([vp, i32, i32, i32, ctypes.POINTER(sz), ctypes.POINTER(ctypes.c_int64)], ctypes.c_int),
         "vgg19_conv_wgrad_static": ([vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, ctypes.POINTER(sz), vp], ctypes.c_int),
         "vgg19_sync_status": ([vp, vp], ctypes.c_int),
@@ -228,6 +230,15 @@ def vgg19_conv_layer_forward(net, layer, x, batch, y, pooled=None, stream=None):
 def vgg19_conv_layer_backward(net, layer, x, dz, batch, dw, db, dx=None, stream=None):
     return _check(net, load().vgg19_conv_layer_backward(net, layer, _ptr(x), _ptr(dz), batch, _ptr(dw), _ptr(db),
                                                          _ptr(dx), _stream(stream)))
+
+
+def vgg19_dense_layer_forward(net, layer, x, batch, y=None, y_f32=None, stream=None):
+    return _check(net, load().vgg19_dense_layer_forward(net, layer, _ptr(x), batch, _ptr(y), _ptr(y_f32), _stream(stream)))
+
+
+def vgg19_dense_layer_backward(net, layer, x, dy, batch, dw, db, dx=None, relu_mask=None, stream=None):
+    return _check(net, load().vgg19_dense_layer_backward(net, layer, _ptr(x), _ptr(dy), batch, _ptr(dw), _ptr(db),
+                                                          _ptr(dx), _ptr(relu_mask), _stream(stream)))
 
 
 def vgg19_conv_layer_forward_ex(net, layer, x, batch, y, pooled=None, pool_code=None, stream=None):

@@ -1122,6 +1122,56 @@ int vgg19_conv_layer_backward(vgg19_t *n, int32_t layer, const void *x, const vo
   return vgg19_conv_layer_backward_ex(n, layer, x, dz, batch, dw, db, dx, nullptr, nullptr, stream);
 }
 
+int vgg19_dense_layer_forward(vgg19_t *n, int32_t layer, const void *x, int32_t batch, void *y, float *y_f32,
+                              void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (layer < 1 || layer > kFcLayers || !x || (!y && !y_f32))
+    return fail(n, VGG19_ERR_ARG, "bad dense layer (%d) or null tensor", layer);
+  int rc = check_batch(n, batch, VGG19_MODE_FORWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  n->other_pass = true;
+  Plan p = make_plan(n, batch, VGG19_MODE_FORWARD);
+  cudaError_t e;
+  if (n->cfg.dtype == VGG19_BF16) {
+    Pass<bf16> ps{n, p, st};
+    ps.dense_forward(n->fc[layer - 1], (const bf16 *)x, batch, (bf16 *)y, y_f32);
+    e = ps.err;
+  } else {
+    Pass<float> ps{n, p, st};
+    ps.dense_forward(n->fc[layer - 1], (const float *)x, batch, (float *)y, y_f32);
+    e = ps.err;
+  }
+  if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  return VGG19_OK;
+}
+
+int vgg19_dense_layer_backward(vgg19_t *n, int32_t layer, const void *x, const void *dy, int32_t batch, float *dw,
+                               float *db, void *dx, const void *relu_mask, void *stream) {
+  if (!n) return VGG19_ERR_ARG;
+  if (layer < 1 || layer > kFcLayers || !x || !dy || !dw || !db || (relu_mask && !dx))
+    return fail(n, VGG19_ERR_ARG, "bad dense layer (%d) or null tensor", layer);
+  int rc = check_batch(n, batch, VGG19_MODE_BACKWARD, 0);
+  if (rc != VGG19_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  n->other_pass = true;
+  Plan p = make_plan(n, batch, VGG19_MODE_BACKWARD);
+  cudaError_t e;
+  if (n->cfg.dtype == VGG19_BF16) {
+    Pass<bf16> ps{n, p, st};
+    ps.dense_backward(n->fc[layer - 1], (const bf16 *)x, (const bf16 *)dy, batch, dw, db,
+                      dx ? (bf16 *)dx : ps.buf(p.dflat), (const bf16 *)relu_mask);
+    e = ps.err;
+  } else {
+    Pass<float> ps{n, p, st};
+    ps.dense_backward(n->fc[layer - 1], (const float *)x, (const float *)dy, batch, dw, db,
+                      dx ? (float *)dx : ps.buf(p.dflat), (const float *)relu_mask);
+    e = ps.err;
+  }
+  if (e != cudaSuccess) return fail(n, VGG19_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  return VGG19_OK;
+}
+
 int vgg19_saved_tensor(const vgg19_t *n, int32_t batch, int32_t mode, int32_t index,
                        size_t *offset_bytes, int64_t dims[4]) {
   if (!n || !offset_bytes || !dims || batch < 1 || batch > n->cfg.batch_max || mode < 0 || mode > 2 ||
