@@ -263,6 +263,34 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
       tc_fence_after();
       const int tw = tile % a.tiles_w, t = tile / a.tiles_w;
       const int w0 = tw * TW, h0 = (t % a.tiles_h) * TH, img = t / a.tiles_h;
+      // Phase 1: the accumulator into registers (three partial sums per value, added across lanes), bias, ReLU,
+      // bf16 - and the accumulator goes back to the MMA thread at once: everything that can make this group wait
+      // (its previous store still reading the staging tile, the mask tile's copy) comes after.
+      uint32_t packed[16];
+#pragma unroll
+      for (int pass = 0; pass < 2; ++pass) {
+        const int c16 = c_first + 16 * pass;
+        uint32_t v0[16], v1[16], v2[16];
+        tmem_ld_32x16(t_row + (uint32_t)c16, v0);
+        tmem_ld_32x16(t_row + (uint32_t)(64 + c16), v1);
+        tmem_ld_32x16(t_row + (uint32_t)(128 + c16), v2);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) {
+          // out(ph, j) = D(ph, j)[s = 0] + D(ph, j + 1)[s = 1] + D(ph, j + 2)[s = 2]
+          float x0 = __uint_as_float(v0[i]) + __shfl_down_sync(0xffffffffu, __uint_as_float(v1[i]), 1) +
+                     __shfl_down_sync(0xffffffffu, __uint_as_float(v2[i]), 2);
+          float x1 = __uint_as_float(v0[i + 1]) + __shfl_down_sync(0xffffffffu, __uint_as_float(v1[i + 1]), 1) +
+                     __shfl_down_sync(0xffffffffu, __uint_as_float(v2[i + 1]), 2);
+          x0 += bias_s[c16 + i]; x1 += bias_s[c16 + i + 1];
+          if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
+          __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+          packed[pass * 8 + (i >> 1)] = *reinterpret_cast<uint32_t*>(&hh);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty(group));
+      // Phase 2: mask, staging tile, pooled output
       if (a.out) {
         // the group's previous store has read the staging tile, and (barrier above) every thread of
         // the group is done with the previous mask tile
@@ -275,33 +303,16 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
                                 : nullptr;
       uint8_t* code_row = (MODE == 1 && a.code) ? a.code + (((long)img * (a.H / 2) + (h0 + ph) / 2) * (a.W / 2) + (w0 + j) / 2) * 64
                                  : nullptr;
-      // pool scatter: this thread's 32 code bytes, requested before the tensor-memory loads
+      // pool scatter: this thread's 32 code bytes
       uint4 sc[2];
       if (MODE == 2 && col_ok) {
         const uint4* cp = reinterpret_cast<const uint4*>(a.scatter_code + (((long)img * a.H + h0 + ph) * a.W + w0 + j) * 64 + c_first);
         sc[0] = __ldg(cp); sc[1] = __ldg(cp + 1);
       }
-      uint32_t kept[16];  // pool scatter: the tile's values (bf16 pairs) of this thread's 32 channels
 #pragma unroll
-      for (int c16 = c_first; c16 < c_first + 32; c16 += 16) {
-        uint32_t v0[16], v1[16], v2[16];
-        tmem_ld_32x16(t_row + (uint32_t)c16, v0);
-        tmem_ld_32x16(t_row + (uint32_t)(64 + c16), v1);
-        tmem_ld_32x16(t_row + (uint32_t)(128 + c16), v2);
-        tmem_ld_wait();
-        uint32_t packed[8];
-#pragma unroll
-        for (int i = 0; i < 16; i += 2) {
-          // out(ph, j) = D(ph, j)[s = 0] + D(ph, j + 1)[s = 1] + D(ph, j + 2)[s = 2]
-          float x0 = __uint_as_float(v0[i]) + __shfl_down_sync(0xffffffffu, __uint_as_float(v1[i]), 1) +
-                     __shfl_down_sync(0xffffffffu, __uint_as_float(v2[i]), 2);
-          float x1 = __uint_as_float(v0[i + 1]) + __shfl_down_sync(0xffffffffu, __uint_as_float(v1[i + 1]), 1) +
-                     __shfl_down_sync(0xffffffffu, __uint_as_float(v2[i + 1]), 2);
-          x0 += bias_s[c16 + i]; x1 += bias_s[c16 + i + 1];
-          if (a.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); }
-          __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-          packed[i >> 1] = *reinterpret_cast<uint32_t*>(&hh);
-        }
+      for (int pass = 0; pass < 2; ++pass) {
+        const int c16 = c_first + 16 * pass;
+        uint32_t (&pk)[8] = reinterpret_cast<uint32_t (&)[8]>(packed[pass * 8]);
         const int chunk0 = c16 >> 3;  // first of this pass's two 16-byte chunks of the 128-byte row
         if (a.mask && col_ok) {
 #pragma unroll
@@ -315,36 +326,30 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
               uint32_t keep = 0;
               if (lo != 0 && !(lo & 0x8000u)) keep |= 0x0000FFFFu;
               if (hi != 0 && !(hi & 0x8000u)) keep |= 0xFFFF0000u;
-              packed[q * 4 + e] &= keep;
+              pk[q * 4 + e] &= keep;
             }
           }
-        }
-        if (MODE == 2) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) kept[((c16 - c_first) >> 1) + i] = packed[i];
         }
         if (a.out && col_ok) {
 #pragma unroll
           for (int q = 0; q < 2; ++q)
             *reinterpret_cast<uint4*>(stage_row + (((chunk0 + q) ^ (rr & 7)) << 4)) =
-                make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+                make_uint4(pk[q * 4], pk[q * 4 + 1], pk[q * 4 + 2], pk[q * 4 + 3]);
         }
         if (a.pooled) {
-          // 2x2 window: columns j, j + 1 (next lane) of rows ph, ph + 1 (16 lanes on)
+          // 2x2 window: columns j, j + 1 (next lane) of rows ph, ph + 1 (16 lanes on); in place (the tile is
+          // already in the staging tile, and the pool scatter, which reads these values again, has no pooled output)
           uint32_t codes[4];
-          if (MODE == 1) pool2x2_codes<8>(packed, 1, 16, codes);
-          else pool2x2<8>(packed, 1, 16);
+          if (MODE == 1) pool2x2_codes<8>(pk, 1, 16, codes);
+          else pool2x2<8>(pk, 1, 16);
           if (pool_lane) {
             uint4* pp = reinterpret_cast<uint4*>(pool_row + c16);
-            pp[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            pp[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+            pp[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            pp[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
             if (code_row) *reinterpret_cast<uint4*>(code_row + c16) = make_uint4(codes[0], codes[1], codes[2], codes[3]);
           }
         }
       }
-      // the accumulator has been read: hand it back before the store is issued
-      tc_fence_before();
-      mbar_arrive(acc_empty(group));
       if (a.out) {
         fence_async_smem();
         named_bar_sync(bar_id, kGroupThreads);  // the staging tile is complete, and the group has read its mask tile
@@ -376,7 +381,7 @@ conv3x3_rowshift_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __gr
                 uint32_t keep = 0;
                 if ((k2 & 0xFFu) == q) keep |= 0x0000FFFFu;
                 if (((k2 >> 8) & 0xFFu) == q) keep |= 0xFFFF0000u;
-                o[e] = kept[ch * 4 + e] & keep;
+                o[e] = packed[ch * 4 + e] & keep;
               }
               *reinterpret_cast<uint4*>(stage_row + ((((c_first >> 3) + ch) ^ (rr & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
             }
