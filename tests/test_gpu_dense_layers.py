@@ -85,6 +85,35 @@ def test_dense_layer_backward(net224, layer, In, Out, relu, B):
     assert rel_l2(dx.float().cpu().numpy(), oracle.round_bf16(o_dx)) <= 1e-3
 
 
+def test_dense_layers_fp32_configuration():
+    """The fp32 configuration's dense kernels (CUDA cores) through the same entry points, 32x32 network:
+    512 -> 4096 -> 4096 -> 1000, bar 1e-5."""
+    import paper_1810_09868_b200 as p
+    B = 3
+    params = si.vgg19_params(32, 32, seed=0, bias_std=0.1)
+    net = p.Net(32, 32, B, p.VGG19_FP32, params=params)
+    for layer, In, Out, relu in [(1, 512, 4096, True), (2, 4096, 4096, True), (3, 4096, 1000, False)]:
+        x = si.normal(B * In, seed=700 + layer, take_abs=True).reshape(B, In).astype(np.float32)
+        dy = si.normal(B * Out, seed=800 + layer, stddev=1e-3).reshape(B, Out).astype(np.float32)
+        Wt, b = layer_params(p, net, params, layer)
+        xd, dyd = torch.from_numpy(x).to(DEV), torch.from_numpy(dy).to(DEV)
+        y = torch.full((B, Out), float("nan"), dtype=torch.float32, device=DEV)
+        p.vgg19_dense_layer_forward(net.handle, layer, xd, B, y, None, torch.cuda.current_stream())
+        dw = torch.full((Out, In), float("nan"), dtype=torch.float32, device=DEV)
+        db = torch.full((Out,), float("nan"), dtype=torch.float32, device=DEV)
+        dx = torch.full((B, In), float("nan"), dtype=torch.float32, device=DEV)
+        p.vgg19_dense_layer_backward(net.handle, layer, xd, dyd, B, dw, db, dx, None, torch.cuda.current_stream())
+        net.sync_status()
+        ref = oracle.dense_fwd(x.astype(np.float64), Wt, b)
+        if relu:
+            ref = oracle.relu_fwd(ref)
+        o_dx, o_dw, o_db = oracle.dense_bwd(x.astype(np.float64), Wt, dy.astype(np.float64))
+        assert rel_l2(y.cpu().numpy(), ref) <= 1e-5
+        assert rel_l2(dw.cpu().numpy(), o_dw) <= 1e-5 and rel_l2(db.cpu().numpy(), o_db) <= 1e-5
+        assert rel_l2(dx.cpu().numpy(), o_dx) <= 1e-5
+    net.close()
+
+
 def test_dense_layer_arguments():
     import paper_1810_09868_b200 as p
     net = p.Net(32, 32, 2, p.VGG19_BF16, seed=0)
