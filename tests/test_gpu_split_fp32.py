@@ -71,13 +71,14 @@ def test_split_conv_layer_forward(net224, layer, S, Cin, Cout):
     assert np.array_equal(pooled.cpu().numpy(), oracle.maxpool2x2_fwd(got.astype(np.float64)).astype(np.float32))
 
 
-@pytest.mark.parametrize("H,B", [(32, 1), (64, 3)])
-def test_split_forward_small(H, B):
-    """Section 7.2's fp32 configuration (32x32, batch 1) and a larger one, whole pass, bar 1e-4."""
+@pytest.mark.parametrize("H,B,extra", [(32, 1, 0), (64, 3, 0), (32, 2, 1)])
+def test_split_forward_small(H, B, extra):
+    """Section 7.2's fp32 configuration (32x32, batch 1) and a larger one, whole pass, bar 1e-4; also without a
+    recorded graph (extra = VGG19_FLAG_NO_GRAPH)."""
     p = pkg()
     params = si.vgg19_params(H, H, seed=0, bias_std=0.05)
     images = si.images(B, H, H, seed=1)
-    net = p.Net(H, H, B, p.VGG19_FP32, params=params, flags=p.VGG19_FLAG_SPLIT_F16, mode=p.VGG19_MODE_FORWARD)
+    net = p.Net(H, H, B, p.VGG19_FP32, params=params, flags=p.VGG19_FLAG_SPLIT_F16 | extra, mode=p.VGG19_MODE_FORWARD)
     x = torch.from_numpy(images).to(DEV)
     probs = torch.empty(B, 1000, dtype=torch.float32, device=DEV)
     logits = net.forward(x, probs=probs).clone()
