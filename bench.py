@@ -720,6 +720,18 @@ def run_profile_layer(args):
     import paper_1810_09868_b200 as pkg
     L, B = args.profile_layer, args.profile_batch
     s, ci, co = CONV[L - 1]
+    if args.profile_kind == "split":
+        # the fp32 configuration's tensor-core path: fp32 tensors in and out, split-fp16 kernel between
+        params = si.vgg19_params(H, W, seed=0)
+        net = pkg.Net(H, W, B, pkg.VGG19_FP32, params=params, flags=pkg.VGG19_FLAG_SPLIT_F16, mode=pkg.VGG19_MODE_FORWARD)
+        x = torch.from_numpy(si.normal(B * s * s * ci, seed=100 + L, take_abs=True).reshape(B, s, s, ci)).cuda().float()
+        y = torch.empty(B, s, s, co, dtype=torch.float32, device="cuda")
+        stream = torch.cuda.Stream()
+        for _ in range(3):
+            pkg.vgg19_conv_layer_forward(net.handle, L, x, B, y, None, stream)
+        net.sync_status(stream)
+        print(f"profiled conv layer {L} (split-fp16), batch {B}: {s}x{s}, {ci}->{co}")
+        return
     params = si.vgg19_params(H, W, seed=0, bf16_exact=True)
     net = pkg.Net(H, W, B, pkg.VGG19_BF16, params=params)
     x = torch.from_numpy(si.normal(B * s * s * ci, seed=100 + L, take_abs=True, bf16_exact=True)
@@ -778,7 +790,7 @@ def main():
     ap.add_argument("--profile-layer", type=int, default=0, help="run only this conv layer (1..16) a few times and exit")
     ap.add_argument("--profile-pass", action="store_true", help="run three forward and three forward+backward passes and exit")
     ap.add_argument("--profile-batch", type=int, default=16)
-    ap.add_argument("--profile-kind", default="fwd", choices=["fwd", "bwd"])
+    ap.add_argument("--profile-kind", default="fwd", choices=["fwd", "bwd", "split"])
     args = ap.parse_args()
     if args.profile_layer:
         run_profile_layer(args)
