@@ -248,6 +248,23 @@ def test_mid_size_image_takes_every_convolution_kernel():
     net.close()
 
 
+def test_wide_image_takes_the_large_image_kernels_with_unequal_sides():
+    # 96 rows x 224 columns: the row-shift kernel at 96x224 and the halo kernel at 48x112 (height and width enter
+    # their tile arithmetic separately), the pair kernels at 24x56, 12x28 and 6x14 with ragged last tiles, and a
+    # first dense layer of 3 x 7 x 512 inputs; forward + backward against the checker
+    p = pkg()
+    params, images, labels = make_inputs(96, 224, 2, True, bias_std=0.05)
+    net = p.Net(96, 224, 2, p.VGG19_BF16, params=params)
+    logits, grads, loss = run_backward(net, images, labels)
+    check_bf16_backward(net, params, images, labels, logits, grads, loss)
+    # and the forward-only pass (pools in the epilogues, no pre-pool activation stored) gives the same logits
+    x = torch.from_numpy(images).to(DEV).to(torch.bfloat16)
+    fwd = net.forward(x).clone()
+    net.sync_status()
+    assert rel_l2(fwd.cpu().numpy(), logits) <= 1e-3
+    net.close()
+
+
 def test_graph_replay_is_bit_identical_and_matches_direct_launch():
     p = pkg()
     params, images, _ = make_inputs(32, 32, 2, True)
