@@ -265,6 +265,18 @@ def test_wide_image_takes_the_large_image_kernels_with_unequal_sides():
     net.close()
 
 
+@pytest.mark.parametrize("B", [1, 3])
+def test_full_resolution_odd_batches(B):
+    # 224x224 at batch 1 and 3: odd tile counts in the pair kernels (a last pair with one idle CTA), tail rounds
+    # of other sizes than at batch 100, a dense M tile of 1 or 3 rows
+    p = pkg()
+    params, images, labels = make_inputs(224, 224, B, True, bias_std=0.05)
+    net = p.Net(224, 224, B, p.VGG19_BF16, params=params)
+    logits, grads, loss = run_backward(net, images, labels)
+    check_bf16_backward(net, params, images, labels, logits, grads, loss)
+    net.close()
+
+
 def test_graph_replay_is_bit_identical_and_matches_direct_launch():
     p = pkg()
     params, images, _ = make_inputs(32, 32, 2, True)
