@@ -277,6 +277,25 @@ def test_full_resolution_odd_batches(B):
     net.close()
 
 
+@pytest.mark.parametrize("H,W", [(256, 256), (448, 448)])
+def test_other_resolutions_forward(H, W):
+    # 256x256: a width that is no multiple of 14, so conv1_2 leaves the row-shift kernel for the halo kernel;
+    # 448x448: four times the benchmark's pixels (first dense layer 14 x 14 x 512 = 100352 inputs).  Forward-only
+    # pass (pools in the epilogues) and training-mode forward give logits within the bf16 bar of the checker.
+    p = pkg()
+    params, images, labels = make_inputs(H, W, 1, True, bias_std=0.05)
+    net = p.Net(H, W, 1, p.VGG19_BF16, params=params)
+    x = torch.from_numpy(images).to(DEV).to(torch.bfloat16)
+    fwd = net.forward(x).clone()
+    net.sync_status()
+    ref = oracle.forward(oracle.vgg19_steps(), params.astype(np.float64), images)
+    assert np.isfinite(fwd.cpu().numpy()).all()
+    assert rel_l2(fwd.cpu().numpy(), ref) <= 2e-2
+    logits, grads, loss = run_backward(net, images, labels)
+    assert rel_l2(logits, ref) <= 2e-2 and np.isfinite(grads).all()
+    net.close()
+
+
 def test_graph_replay_is_bit_identical_and_matches_direct_launch():
     p = pkg()
     params, images, _ = make_inputs(32, 32, 2, True)
