@@ -60,7 +60,7 @@ enum {
   /* fp32 only: forward-only passes (vgg19_forward*, vgg19_conv_layer_forward*) run layers 2..16 and the dense
    * layers on tensor cores, every fp32 value carried as two fp16 terms (hi = fp16(v), lo = fp16(v - hi)) and
    * every product formed as hi*hi + hi*lo + lo*hi in an fp32 accumulator: 22 of fp32's 24 mantissa bits per
-   * operand.  Activations must stay within fp16's range (65504): one beyond it makes vgg19_sync_status
+   * operand (an absolute 3e-8 for activations below 0.25).  Activations must stay within fp16's range (65504): one beyond it makes vgg19_sync_status
    * return VGG19_ERR_RANGE.  Backward and training passes keep the CUDA-core kernels.  The paper runs its
    * fp32 network (section 7.2) on CPU and GPU back ends and has no counterpart of this. */
   VGG19_FLAG_SPLIT_F16 = 16

@@ -2,8 +2,10 @@
 //
 // A value v is carried as hi = fp16(v) and lo = fp16(v - hi): v - hi is exact in fp32, and hi + lo keeps
 // 22 bits of v's mantissa (two bf16 terms would keep 16 at the same cost of three products).  The price is
-// fp16's range: values beyond 65504 are reported (kDevSplitRange), values below 6e-5 lose bits of their lo
-// term, which is why weights are scaled by a power of two before they are split.
+// fp16's range: values beyond 65504 are reported (kDevSplitRange); where the lo term falls among fp16's subnormal
+// numbers (|v| below about 0.25) the pair keeps an absolute 2^-25 rather than 22 bits - nothing beside activations of
+// order one, but weights around 1e-2 would lose five bits, which is why they are scaled by a power of two before
+// they are split.
 // A row of C values (a pixel's channels, a dense layer's row) is stored as [hi_0 .. hi_{C-1} | lo_0 .. lo_{C-1}]:
 // 4 C bytes, the size of the fp32 row, so a buffer planned for fp32 holds either form.  The kernels here move
 // tensors between the two forms, pool the split form, and build the filter copies [w_hi | w_lo | w_hi] whose
