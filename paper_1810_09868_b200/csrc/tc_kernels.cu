@@ -172,20 +172,24 @@ using namespace tc;
 constexpr int BM = 128;             // pixels per tile (TMEM lanes)
 constexpr int BK = 64;              // channels per K block (one 128-byte swizzle row)
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int kThreads = 192;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kSplitChunk = 8;      // SPLIT: K blocks (of 64) per accumulation chain in tensor memory: 32 MMAs
 
-template <int BN>
+// EPI: epilogue groups of four warps, each with its own staging tile and BN / EPI of the tile's columns
+template <int BN, int EPI = 1>
 struct ConvTile {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int OUT_BYTES = BM * 64 * 2;  // staging tile of the TMA store: 128 rows x 64 channels
-  // leaves room for the staging tile, barriers, bias and alignment
-  static constexpr int STAGES = (kSmemLimit - 4608 - OUT_BYTES) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608 - OUT_BYTES) / STAGE_BYTES;
+  // leaves room for the staging tiles, barriers, bias and alignment
+  static constexpr int STAGES = (kSmemLimit - 4608 - EPI * OUT_BYTES) / STAGE_BYTES > 8 ? 8 : (kSmemLimit - 4608 - EPI * OUT_BYTES) / STAGE_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;  // 128, 256 or 512: powers of two
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI * OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
+// SPLIT with 256-column tiles: two epilogue groups of 128 columns each (the running sums of a tile row live in
+// registers: 128 per thread is what fits), 320 threads
+template <int BN, bool SPLIT> __host__ __device__ constexpr int conv_epi_groups() { return SPLIT && BN == 256 ? 2 : 1; }
+template <int BN, bool SPLIT> __host__ __device__ constexpr int conv_threads() { return 64 + 128 * conv_epi_groups<BN, SPLIT>(); }
 
 struct ConvArgs {
   int pixels;     // N*H*W
@@ -213,15 +217,17 @@ constexpr int PW = 16, PH = 8;  // patch of a tile in patch mode (PW * PH = BM)
 // the ReLU, splits the result again and stores the two terms.  A result beyond fp16's range is reported in
 // *dev_error (kDevSplitRange).
 template <int BN, bool SPLIT>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__((conv_threads<BN, SPLIT>()), 1)
 conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                   const __grid_constant__ CUtensorMap map_y, ConvArgs a) {
-  using T = ConvTile<BN>;
+  constexpr int EPI = conv_epi_groups<BN, SPLIT>();
+  constexpr int CW = BN / EPI;  // columns of an epilogue group
+  using T = ConvTile<BN, EPI>;
   extern __shared__ uint8_t smem_raw[];
   // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t out_smem = smem_base + T::STAGES * T::STAGE_BYTES;  // 1024-byte aligned
-  const uint32_t bars = out_smem + T::OUT_BYTES;
+  const uint32_t bars = out_smem + EPI * T::OUT_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (T::STAGES + s); };
   auto acc_full_bar = [&](int b) { return bars + 8u * (2 * T::STAGES + b); };
@@ -235,11 +241,11 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   const int k_blocks = 9 * a.cin_blocks;
   const int total_tiles = a.m_tiles * a.n_tiles;
 
-  for (int i = threadIdx.x; i < a.Cout; i += kThreads) bias_s[i] = a.bias ? a.bias[i] : 0.f;
+  for (int i = threadIdx.x; i < a.Cout; i += (int)blockDim.x) bias_s[i] = a.bias ? a.bias[i] : 0.f;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < T::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 128); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 128 * EPI); }
     mbar_init(drain_bar, 1);
     mbar_fence_init();
     tma_prefetch_desc(&map_x);
@@ -348,30 +354,34 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // -------------------------------- epilogue --------------------------------
     const int quarter = warp & 3;  // the TMEM lane quarter this warp may read
     const int row = quarter * 32 + lane;
+    const int grp = EPI == 1 ? 0 : (warp - 2) >> 2;  // epilogue group: columns [grp * CW, (grp + 1) * CW) of the tile
+    const int col_base = grp * CW;
+    const int bar_id = 1 + grp;
+    const uint32_t my_out = out_smem + grp * T::OUT_BYTES;
     int local = 0;
     // The tile leaves 64 channels at a time through a 128-byte-swizzled staging tile and one TMA
-    // store (whole 128-byte lines), not as per-thread pieces of rows.  Thread 64 owns the store groups.
-    const bool issuer = threadIdx.x == 64;
-    uint8_t* stage_row = smem_raw + (out_smem - smem_u32(smem_raw)) + row * 128;
+    // store (whole 128-byte lines), not as per-thread pieces of rows.  The group's first thread owns its store groups.
+    const bool issuer = threadIdx.x == 64 + 128 * grp;
+    uint8_t* stage_row = smem_raw + (my_out - smem_u32(smem_raw)) + row * 128;
     bool alive = true;
     for (int tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x, ++local) {
       const int m_tile = tile / a.n_tiles, n_tile = tile - m_tile * a.n_tiles;
       // SPLIT: the tensor core's fp32 accumulation truncates, an error that grows with the length of the chain
       // (1.6e-5 after the 864 MMAs of a 512-channel layer).  The K loop therefore hands over its accumulator every
       // kSplitChunk K blocks, and the chunks are added here, in registers, with round-to-nearest fp32 additions.
-      float run[SPLIT ? BN : 1];
+      float run[SPLIT ? CW : 1];
       if (SPLIT) {
 #pragma unroll
-        for (int j = 0; j < BN; ++j) run[j] = 0.f;
+        for (int j = 0; j < CW; ++j) run[j] = 0.f;
         for (int kb0 = kSplitChunk; kb0 < k_blocks && alive; kb0 += kSplitChunk, ++local) {
           const int cbuf = local & 1;
           const bool cgot = mbar_wait(acc_full_bar(cbuf), (uint32_t)(local >> 1) & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
-          if (named_bar_or(1, 128, !cgot)) { alive = false; break; }
+          if (named_bar_or(bar_id, 128, !cgot)) { alive = false; break; }
           tc_fence_after();
 #pragma unroll
-          for (int cc = 0; cc < BN; cc += 32) {
+          for (int cc = 0; cc < CW; cc += 32) {
             uint32_t v[32];
-            tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cbuf * BN + cc), v);
+            tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cbuf * BN + col_base + cc), v);
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) run[cc + j] += __uint_as_float(v[j]);
@@ -384,7 +394,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
       const bool got = mbar_wait(acc_full_bar(buf), use & 1, &abort_flag, a.dev_error, kDevTimeoutAccum);
-      if (named_bar_or(1, 128, !got)) break;  // all four warps leave together
+      if (named_bar_or(bar_id, 128, !got)) break;  // the group's four warps leave together
       tc_fence_after();
       long pixel;
       int tw = 0, th = 0, img = 0;
@@ -397,19 +407,19 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         pixel = (long)m_tile * BM + row;
       }
       const bool valid = pixel < a.pixels;
-      const int c_base = n_tile * BN;
+      const int c_base = n_tile * BN + col_base;  // first output channel of this group's columns
       const bf16* mask_row = (a.mask && valid) ? a.mask + pixel * a.Cout + c_base : nullptr;
-#pragma unroll(SPLIT ? BN / 64 : 1)
-      for (int c64 = 0; c64 < BN; c64 += 64) {
+#pragma unroll(SPLIT ? CW / 64 : 1)
+      for (int c64 = 0; c64 < CW; c64 += 64) {
         if (issuer) tma_store_wait_read<0>();  // the previous store has read the staging tile
-        named_bar_sync(1, 128);
+        named_bar_sync(bar_id, 128);
         uint32_t lo_packed[SPLIT ? 32 : 1];
         bool out_of_range = false;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           const int cc = c64 + half * 32;
           uint32_t v[32];
-          tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cc), v);
+          tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + col_base + cc), v);
           tmem_ld_wait();
           uint32_t packed[16];
 #pragma unroll
@@ -458,27 +468,27 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           }
         }
         fence_async_smem();
-        named_bar_sync(1, 128);
+        named_bar_sync(bar_id, 128);
         if (issuer) {
           // rows past the end of the tensor (last tile) are clipped by the copy engine
-          if (a.patch) tma_store_4d(&map_y, out_smem, c_base + c64, tw * PW, th * PH, img);
-          else tma_store_2d(&map_y, out_smem, c_base + c64, m_tile * BM);
+          if (a.patch) tma_store_4d(&map_y, my_out, c_base + c64, tw * PW, th * PH, img);
+          else tma_store_2d(&map_y, my_out, c_base + c64, m_tile * BM);
           tma_store_commit();
         }
         if (SPLIT) {
           if (out_of_range && valid) atomicCAS(a.dev_error, 0, (int)kDevSplitRange);
           // the second terms of the same 64 channels, Cout channels further on in the pixel's row
           if (issuer) tma_store_wait_read<0>();
-          named_bar_sync(1, 128);
+          named_bar_sync(bar_id, 128);
 #pragma unroll
           for (int chunk = 0; chunk < 8; ++chunk)
             *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) =
                 make_uint4(lo_packed[chunk * 4], lo_packed[chunk * 4 + 1], lo_packed[chunk * 4 + 2], lo_packed[chunk * 4 + 3]);
           fence_async_smem();
-          named_bar_sync(1, 128);
+          named_bar_sync(bar_id, 128);
           if (issuer) {
-            if (a.patch) tma_store_4d(&map_y, out_smem, a.Cout + c_base + c64, tw * PW, th * PH, img);
-            else tma_store_2d(&map_y, out_smem, a.Cout + c_base + c64, m_tile * BM);
+            if (a.patch) tma_store_4d(&map_y, my_out, a.Cout + c_base + c64, tw * PW, th * PH, img);
+            else tma_store_2d(&map_y, my_out, a.Cout + c_base + c64, m_tile * BM);
             tma_store_commit();
           }
         }
@@ -501,7 +511,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 template <int BN, bool SPLIT = false>
 cudaError_t launch_conv(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, ConvArgs a,
                         cudaStream_t st) {
-  using T = ConvTile<BN>;
+  using T = ConvTile<BN, conv_epi_groups<BN, SPLIT>()>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel<BN, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES);
@@ -513,7 +523,7 @@ cudaError_t launch_conv(const CUtensorMap& mx, const CUtensorMap& mw, const CUte
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int tiles = a.m_tiles * a.n_tiles;
   const int grid = tiles < sms ? tiles : sms;
-  conv3x3_tc_kernel<BN, SPLIT><<<grid, kThreads, T::SMEM_BYTES, st>>>(mx, mw, my, a);
+  conv3x3_tc_kernel<BN, SPLIT><<<grid, conv_threads<BN, SPLIT>(), T::SMEM_BYTES, st>>>(mx, mw, my, a);
   return cudaGetLastError();
 }
 
@@ -569,7 +579,8 @@ cudaError_t tc_conv3x3(const bf16* in, const bf16* wt, const float* bias, const 
 cudaError_t tc_conv3x3_split(const half16* in, const half16* wt_split, const float* bias, half16* out, ConvShape s,
                              bool relu, int* dev_error, cudaStream_t st) {
   if (!tc_conv3x3_supported(s)) return cudaErrorInvalidValue;
-  const int BN = s.Cout % 128 == 0 ? 128 : 64;  // the epilogue keeps a tile row's running sums in registers
+  // the epilogue keeps a tile row's running sums in registers, 128 per thread: 256-column tiles take two groups of warps
+  const int BN = s.Cout % 256 == 0 ? 256 : s.Cout % 128 == 0 ? 128 : 64;
   CUtensorMap mx, mw, my;
   const bool patch = s.W % PW == 0 && s.H % PH == 0;
   if (patch) {
@@ -592,7 +603,8 @@ cudaError_t tc_conv3x3_split(const half16* in, const half16* wt_split, const flo
   a.n_tiles = s.Cout / BN;
   a.relu = relu ? 1 : 0;
   a.bias = bias; a.mask = nullptr; a.out = reinterpret_cast<bf16*>(out); a.dev_error = dev_error;
-  return BN == 128 ? launch_conv<128, true>(mx, mw, my, a, st) : launch_conv<64, true>(mx, mw, my, a, st);
+  return BN == 256 ? launch_conv<256, true>(mx, mw, my, a, st)
+         : BN == 128 ? launch_conv<128, true>(mx, mw, my, a, st) : launch_conv<64, true>(mx, mw, my, a, st);
 }
 
 namespace {
